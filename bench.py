@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the DeMo optimizer transform (compress x W + decode) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decoder_1b] [--impl ours|reference]
+
+One "step" is one optimizer step of the whole hot path: W x demo_compress + 1 x demo_decode_apply
+over a synthetic parameter set resident in HBM.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun)
+every rank runs an independent replica of the same workload -- the path has no exchange step on one
+GPU per replica -- and `value` is the work of all ranks over the slowest rank's time.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "optimizer-step params/s (compress+decode)"
+UNIT = "params/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, device-to-device copy)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+        med = sorted(self.samples)[len(self.samples) // 2] if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def algorithmic_bytes(wl, gbytes: int):
+    """Bytes the method must move per step: per worker read g and m, write m; once read and write x.
+    Payload traffic (written once, read once) is reported separately."""
+    P = wl.n_params
+    core = P * (wl.num_workers * (gbytes + 8) + 8)
+    payload = 2 * wl.num_workers * wl.records_per_worker() * 8
+    return core, payload
+
+
+def cpu_baseline(wl, target_s: float = 12.0):
+    """Time the oracle, as it stands, on a bounded sample: n chunks of 2-D tiles through W compress
+    passes and one decode.  Returns params/s on that sample."""
+    import numpy as np
+
+    from oracle import demo_oracle as orc
+
+    s, k, W = wl.chunk, wl.topk, wl.num_workers
+    M = s * s
+    rng = np.random.default_rng(0)
+
+    def run(n):
+        g = rng.standard_normal((W, n, M)) * 1e-3
+        m = rng.standard_normal((W, n, M)) * 1e-2
+        x = rng.standard_normal((n, M)) * 0.02
+        recs = np.zeros((W, n, min(k, M)), dtype=orc.RECORD_DTYPE)
+        t0 = time.perf_counter()
+        for w in range(W):
+            out = orc.compress_chunks(g[w], m[w], s, s, k, wl.beta)
+            recs[w]["idx"] = out["idx"]
+            recs[w]["val"] = out["val"].astype(np.float32)
+        orc.decode_chunks(recs, x, s, s, wl.lr, wl.weight_decay)
+        return time.perf_counter() - t0
+
+    cores = orc.max_threads()
+    n0 = max(cores, 16)
+    t_probe = run(n0)
+    n = int(min(max(n0, n0 * target_s / max(t_probe, 1e-6)), 1 << 16))
+    t = run(n)
+    return {"value": n * M / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d chunks of %dx%d (k=%d) through W=%d compress passes + 1 decode, %.1f s" % (n, s, s, k, W, t)}, n * M, t
+
+
+def run_reference(args, rank):
+    from paper_2411_19870_b200 import inputs
+
+    if rank != 0:
+        return
+    wl = inputs.by_name(args.workload)
+    times, units = [], 0
+    base = None
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        base, n_par, t = cpu_baseline(wl, target_s=per_step)
+        if i >= args.warmup:
+            times.append(t)
+            units += n_par
+    value = units / sum(times)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "chunk": wl.chunk, "topk": wl.topk, "num_workers": wl.num_workers,
+                   "note": "fp64 CPU oracle on a bounded chunk sample per step"},
+        "cpu_baseline": dict(base, value=value),
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def run_ours(args, rank, world):
+    import torch
+
+    import paper_2411_19870_b200 as demo
+    from paper_2411_19870_b200 import inputs
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = inputs.by_name(args.workload)
+    W, T = wl.num_workers, len(wl.shapes)
+    gbytes = 2 if wl.grad_dtype == torch.bfloat16 else 4
+    tr = demo.DemoTransform(wl.shapes, chunk=wl.chunk, topk=wl.topk, beta=wl.beta, lr=wl.lr,
+                            weight_decay=wl.weight_decay, num_workers=W,
+                            grad_dtype=demo.DEMO_BF16 if gbytes == 2 else demo.DEMO_F32, device=local)
+    if args.path == "generic":
+        tr.set_path(demo.DEMO_PATH_GENERIC)
+    params = inputs.make_params(wl, dev)
+    mom = [inputs.make_momentum(wl, dev) for _ in range(W)]
+    grads = [inputs.GradStream(wl, w, dev).next() for w in range(W)]  # one seeded set per worker, reused
+    payloads = [torch.empty(tr.payload_bytes, dtype=torch.uint8, device=dev) for _ in range(W)]
+    torch.cuda.synchronize()
+
+    def step(events=None):
+        for w in range(W):
+            if events is not None:
+                e0 = torch.cuda.Event(enable_timing=True)
+                e0.record()
+            tr.compress(w, grads[w], mom[w], payloads[w])
+            if events is not None:
+                e1 = torch.cuda.Event(enable_timing=True)
+                e1.record()
+                events["compress"].append((e0, e1))
+        if events is not None:
+            e0 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+        tr.decode_apply(payloads, params)
+        if events is not None:
+            e1 = torch.cuda.Event(enable_timing=True)
+            e1.record()
+            events["decode"].append((e0, e1))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = tr.launch_count
+    events = {"compress": [], "decode": []}
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for _ in range(args.steps):
+        step(events)
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = tr.launch_count - launches0
+    ms_total = t_start.elapsed_time(t_end)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    assert tr.device_status() == 0
+
+    P = wl.n_params
+    value = world * P / (ms_step * 1e-3)
+    core_bytes, payload_bytes = algorithmic_bytes(wl, gbytes)
+    peak, peak_src = _peaks()
+    c_ms = [a.elapsed_time(b) for a, b in events["compress"]]
+    d_ms = [a.elapsed_time(b) for a, b in events["decode"]]
+    c_avg = sum(c_ms) / len(c_ms)
+    d_avg = sum(d_ms) / len(d_ms)
+    compress_bytes = P * (gbytes + 8)  # read g, read m, write m for one worker
+    achieved = compress_bytes / (c_avg * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": "demo_compress (one worker: fused momentum+DCT+top-k+residual over all tensors)",
+        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+        "traffic": None, "algorithmic_bytes_per_launch": compress_bytes, "avg_launch_ms": c_avg,
+        "decode": {"avg_launch_ms": d_avg, "algorithmic_bytes_per_launch": P * 8 + payload_bytes // 2,
+                   "achieved": (P * 8 + payload_bytes // 2) / (d_avg * 1e-3) / 1e9},
+        "step": {"algorithmic_bytes": core_bytes, "payload_bytes": payload_bytes,
+                 "achieved": core_bytes / (ms_step * 1e-3) / 1e9, "frac_of_measured": core_bytes / (ms_step * 1e-3) / 1e9 / peak,
+                 "frac_of_nominal_8TBs": core_bytes / (ms_step * 1e-3) / 8e12},
+    }
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            with open(traffic_file) as f:
+                tj = json.load(f)
+            per_param = tj.get("compress_dram_bytes_per_param")
+            if per_param is not None:
+                roofline["traffic"] = per_param * P
+                roofline["traffic_source"] = tj.get("source")
+        except Exception:
+            pass
+
+    # end to end through the host-buffer entry point: H2D of every worker's gradients from pinned
+    # memory, the step, D2H of the W payloads
+    e2e = None
+    if not args.no_e2e:
+        try:
+            e2e = run_e2e(torch, tr, wl, grads, mom, payloads, params, dev, world, dist, gbytes, args)
+        except Exception as ex:  # pragma: no cover
+            e2e = {"value": None, "unit": UNIT, "error": repr(ex)}
+
+    base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        base, _, _ = cpu_baseline(wl)
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "n_params": P, "n_tensors": T, "chunk": wl.chunk, "topk": wl.topk,
+                       "num_workers": W, "beta": wl.beta, "grad_dtype": "bf16" if gbytes == 2 else "f32",
+                       "parallelism": "replicas only (one GPU per replica, no collective)" if world > 1 else "1 GPU",
+                       "worker_params_per_s": value * W, "l2": "inputs (%.1f GB resident in HBM) are larger than the 126 MB L2; no flush needed" % (
+                           (W * P * (gbytes + 4) + 4 * P + W * tr.payload_bytes) / 1e9), "kernel_path": args.path},
+            "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
+        }
+        if base is not None:
+            out["cpu_baseline"] = base
+        print(json.dumps(out), flush=True)
+    tr.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(torch, tr, wl, grads, mom, payloads, params, dev, world, dist, gbytes, args):
+    W = wl.num_workers
+    P = wl.n_params
+    import psutil
+
+    need = W * P * gbytes + W * tr.payload_bytes
+    distinct = psutil.virtual_memory().available > 2.5 * need * max(1, world)
+    if distinct:
+        host = [[g.cpu().pin_memory() for g in gw] for gw in grads]
+        note = "distinct pinned gradient set per worker"
+    else:
+        one = [g.cpu().pin_memory() for g in grads[0]]
+        host = [one for _ in range(W)]
+        note = "one pinned gradient set copied for every worker (host memory too small for W sets)"
+    out = torch.empty(W * tr.payload_bytes, dtype=torch.uint8).pin_memory()
+    steps = max(1, min(args.steps, args.e2e_steps))
+    tr.step_host(host, grads, mom, payloads, params, out)  # warm-up
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        tr.step_host(host, grads, mom, payloads, params, out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return {"value": world * P / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": W * P * gbytes, "d2h_bytes_per_step": W * tr.payload_bytes, "note": note}
+
+
+def aggregate_replicas(ms_per_rank, units_per_rank):
+    """Whole-job throughput of independent replicas: all units over the slowest rank's time."""
+    return sum(units_per_rank) / (max(ms_per_rank) * 1e-3)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decoder_1b")
+    ap.add_argument("--path", default="auto", choices=["auto", "generic"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = max(args.warmup, 1)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,163 @@
+/*
+ * demo.h -- C ABI of the B200-native DeMo optimizer transform (arXiv 2411.19870).
+ *
+ * One optimizer step of the paper's Algorithm 1 ("DeMo: Decoupled Momentum") is
+ *     for every simulated worker w:   demo_compress(ctx, w, grads_w, momentum_w, payload_w, stream)
+ *     once:                           demo_decode_apply(ctx, payloads, W, params, stream)
+ * All tensors live in device memory owned by the caller; the library owns only its context
+ * (DCT tables, chunk tables, pointer tables, one status word).  Every call enqueues work on the
+ * given CUDA stream and returns; argument errors are reported synchronously before any launch,
+ * device-side problems through demo_device_status().  No C++ exception crosses this boundary,
+ * there is no global state and no CPU fallback: without a CUDA device every compute entry point
+ * fails with DEMO_ERR_CUDA.
+ *
+ * Notation (the paper's): s chunk size, k coefficients kept per chunk, M = s*s (2-D tensors) or
+ * s (1-D tensors) elements per chunk, k_eff = min(k, M), W workers, beta momentum decay,
+ * lr learning rate (eta), weight_decay (lambda).
+ *
+ * Payload layout (part of the bit-exact contract; the paper leaves "encode" open, Section 2.1 and
+ * the appendix algorithm): for every tensor in descriptor order, for every chunk in row-major
+ * order over the chunk grid (c0, c1) of the blocking operator (appendix B.1.2), k_eff records of
+ *     struct { int32_t idx; float val; }      little-endian, 8 bytes
+ * with idx the flat position inside the chunk (i*s + j for 2-D tiles, j for 1-D segments),
+ * records sorted by ascending idx.  Ties at the k-th magnitude go to the lowest idx.
+ */
+#ifndef DEMO_H_
+#define DEMO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct demo_ctx demo_ctx; /* opaque, library-owned */
+
+typedef enum {
+    DEMO_OK = 0,
+    DEMO_ERR_INVALID_ARG = 1, /* null pointer, bad worker index, misaligned buffer, bad count     */
+    DEMO_ERR_SHAPE = 2,       /* ndim not in {1,2} or a dimension not a multiple of s              */
+    DEMO_ERR_K = 3,           /* k < 1 or k > s*s                                                  */
+    DEMO_ERR_UNSUPPORTED = 4, /* s not in {8,16,32,64,128}, unknown dtype, too many tensors        */
+    DEMO_ERR_ALLOC = 5,       /* host or device allocation failed                                  */
+    DEMO_ERR_CUDA = 6,        /* a CUDA runtime call failed (no device, launch error, ...)         */
+    DEMO_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired                                */
+    DEMO_ERR_PAYLOAD = 8      /* decode met a record whose idx is outside its chunk (skipped)      */
+} demo_status;
+
+typedef enum { DEMO_F32 = 0, DEMO_BF16 = 1 } demo_dtype;
+
+/* A contiguous row-major tensor: ndim 1 (shape[0] elements) or ndim 2 (shape[0] x shape[1]). */
+typedef struct {
+    int32_t ndim;
+    int64_t shape[2];
+} demo_tensor_desc;
+
+/* Hyper-parameters of Algorithm 1's "Require" line. */
+typedef struct {
+    float beta;            /* momentum decay, m <- beta*m + g                        */
+    int32_t chunk;         /* s: 2-D tensors use s x s tiles, 1-D tensors length-s    */
+    int32_t topk;          /* k per chunk, 1 <= k <= s*s                              */
+    float lr;              /* eta                                                     */
+    float weight_decay;    /* lambda, applied to every tensor                         */
+    int32_t num_workers;   /* W, number of payloads demo_decode_apply aggregates      */
+    int32_t grad_dtype;    /* demo_dtype of the gradient tensors (momentum/params: f32) */
+} demo_config;
+
+/* Kernel family used for 2-D tensors.  AUTO picks the register-resident fast-DCT kernels where
+ * they exist (s in {32, 64}) and the generic dense-contraction kernels elsewhere; GENERIC forces
+ * the latter everywhere (used by tests to cross-check the two).  Both are CUDA paths. */
+typedef enum { DEMO_PATH_AUTO = 0, DEMO_PATH_GENERIC = 1 } demo_path;
+
+/*
+ * demo_init -- validate the configuration and the tensor list, build the orthonormal DCT-II basis
+ * of dimension s (Section 2.1: "precomputed only once before training"), the chunk tables of the
+ * blocking operator (appendix B.1.2) and the payload offsets, and allocate the context's small
+ * device tables on `cuda_device`.
+ *   out        host pointer receiving the context (set to NULL on failure)
+ *   cfg        host pointer, read during the call
+ *   tensors    host array of n_tensors descriptors, read during the call
+ * Errors: INVALID_ARG (nulls, n_tensors < 1, W < 1, beta/lr/weight_decay not finite), SHAPE, K,
+ * UNSUPPORTED, ALLOC, CUDA.
+ */
+demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_desc *tensors,
+                      int32_t n_tensors, int32_t cuda_device);
+
+/* Bytes of one worker's payload: sum over tensors of n_chunks * k_eff * 8.  0 if ctx is NULL. */
+size_t demo_payload_bytes(const demo_ctx *ctx);
+
+/* Where tensor `tensor` sits inside a payload: index of its first record, its number of chunks
+ * and its k_eff.  Any output pointer may be NULL.  Errors: INVALID_ARG. */
+demo_status demo_payload_layout(const demo_ctx *ctx, int32_t tensor, int64_t *first_record,
+                                int64_t *n_chunks, int32_t *k_eff);
+
+/*
+ * demo_compress -- the worker side of Algorithm 1 / CompressChunks for worker `worker`, fused per
+ * chunk: m <- beta*m + g; Q = DCT(chunk); keep the k_eff largest |Q| as records;
+ * m <- m - IDCT(kept) (momentum subtraction with alpha = 1, Section 2.1 "Momentum Subtraction").
+ *   grads        host array of n_tensors DEVICE pointers (dtype cfg.grad_dtype), read-only
+ *   momentum     host array of n_tensors DEVICE pointers (fp32), updated in place
+ *   payload_out  DEVICE buffer of demo_payload_bytes() bytes, overwritten
+ *   cuda_stream  cudaStream_t (NULL = default stream)
+ * Device buffers must be 16-byte aligned and must not alias each other.  The pointer arrays are
+ * host memory, read during the call and not retained.  Calls on one context must be issued in
+ * stream order (one stream, or streams the caller orders).  Errors: INVALID_ARG, CUDA.
+ */
+demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grads,
+                          float *const *momentum, void *payload_out, void *cuda_stream);
+
+/*
+ * demo_decode_apply -- the server side of Algorithm 1 / Decompress&Aggregate plus the update,
+ * fused per chunk: S = sum over the n_payloads payloads (in the order given) of their records;
+ * R = IDCT(S); x <- x - lr * (sign(R) + weight_decay * x), with sign(0) = 0.
+ *   payloads     host array of n_payloads DEVICE pointers (each demo_payload_bytes() bytes)
+ *   n_payloads   must equal cfg.num_workers
+ *   params       host array of n_tensors DEVICE pointers (fp32), updated in place
+ * A record whose idx lies outside its chunk is skipped and DEMO_ERR_PAYLOAD becomes the sticky
+ * device status.  Errors: INVALID_ARG, CUDA.
+ */
+demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads,
+                              float *const *params, void *cuda_stream);
+
+/*
+ * demo_step_host -- one whole optimizer step driven from HOST gradient buffers: for every worker
+ * copy its gradients host->device into the caller's device staging tensors, compress, then decode
+ * and apply, then (if host_payloads_out is not NULL) copy all W payloads device->host.  Everything
+ * is enqueued on cuda_stream; the host buffers must stay valid until the stream has drained
+ * (use pinned memory for the copies to be asynchronous).
+ *   host_grads         host array [W * n_tensors] of HOST pointers (worker-major)
+ *   dev_grads          host array [W * n_tensors] of DEVICE pointers receiving the copies
+ *   momentum           host array [W * n_tensors] of DEVICE pointers (fp32)
+ *   payloads           host array [W] of DEVICE payload buffers
+ *   params             host array [n_tensors] of DEVICE pointers (fp32)
+ *   host_payloads_out  HOST buffer of W * demo_payload_bytes() bytes, or NULL
+ * Errors: as demo_compress / demo_decode_apply.
+ */
+demo_status demo_step_host(demo_ctx *ctx, const void *const *host_grads, void *const *dev_grads,
+                           float *const *momentum, void *const *payloads, float *const *params,
+                           void *host_payloads_out, void *cuda_stream);
+
+/* The learning rate is scheduled (eta_t in the update equation of Section 2.1): takes effect for
+ * the next demo_decode_apply.  Errors: INVALID_ARG (null ctx, non-finite lr). */
+demo_status demo_set_lr(demo_ctx *ctx, float lr);
+
+/* Select the kernel family (see demo_path).  Errors: INVALID_ARG. */
+demo_status demo_set_path(demo_ctx *ctx, int32_t path);
+
+/* Number of kernel launches this context has enqueued since demo_init (for accounting). */
+int64_t demo_launch_count(const demo_ctx *ctx);
+
+/* Synchronise cuda_stream and return (and clear) the sticky device status word: DEMO_OK,
+ * DEMO_ERR_TIMEOUT or DEMO_ERR_PAYLOAD; DEMO_ERR_CUDA if the synchronisation itself failed. */
+demo_status demo_device_status(demo_ctx *ctx, void *cuda_stream);
+
+const char *demo_status_string(demo_status status);
+
+/* Release the context's host and device memory.  NULL-safe.  Caller-owned tensors are untouched. */
+void demo_free(demo_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEMO_H_ */

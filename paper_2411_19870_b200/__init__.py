@@ -1,0 +1,18 @@
+"""B200-native DeMo optimizer transform (arXiv 2411.19870): thin Python binding over the C ABI.
+
+The product is ``libdemo_b200.so`` (hand-written CUDA for sm_100a behind ``include/demo.h``).
+This package only marshals arguments: every step of the path runs in the library's kernels.
+"""
+from .binding import (  # noqa: F401
+    DEMO_BF16,
+    DEMO_F32,
+    DEMO_PATH_AUTO,
+    DEMO_PATH_GENERIC,
+    DemoConfig,
+    DemoError,
+    DemoTensorDesc,
+    DemoTransform,
+    RECORD_BYTES,
+    demo_status_string,
+    load_library,
+)

@@ -1,0 +1,205 @@
+"""ctypes binding of the C ABI in ``include/demo.h`` -- argument marshalling only.
+
+``load_library()`` opens ``libdemo_b200.so`` (built in-tree by ``build.py``) and fails loudly if it
+is missing: there is no CPU or eager fallback.  ``DemoTransform`` wraps one ``demo_ctx`` and turns
+lists of torch tensors into the pointer arrays the ABI takes; method names follow the ABI
+(``compress`` = ``demo_compress``, ``decode_apply`` = ``demo_decode_apply``, ...).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdemo_b200.so")
+
+DEMO_F32, DEMO_BF16 = 0, 1
+DEMO_PATH_AUTO, DEMO_PATH_GENERIC = 0, 1
+RECORD_BYTES = 8
+
+EXPORTS = [
+    "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
+    "demo_step_host", "demo_set_lr", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_status_string", "demo_free",
+]
+
+
+class DemoTensorDesc(ctypes.Structure):
+    _fields_ = [("ndim", ctypes.c_int32), ("shape", ctypes.c_int64 * 2)]
+
+
+class DemoConfig(ctypes.Structure):
+    _fields_ = [
+        ("beta", ctypes.c_float), ("chunk", ctypes.c_int32), ("topk", ctypes.c_int32), ("lr", ctypes.c_float),
+        ("weight_decay", ctypes.c_float), ("num_workers", ctypes.c_int32), ("grad_dtype", ctypes.c_int32),
+    ]
+
+
+class DemoError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__("%s failed: status %d (%s)" % (where, status, demo_status_string(status)))
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Open the CUDA library and declare the ABI's signatures.  Raises if the library is absent."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(
+            "CUDA library %s is missing: build it with `python -m paper_2411_19870_b200.build` "
+            "(there is no CPU fallback)" % p)
+    lib = ctypes.CDLL(p)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    pvp = ctypes.POINTER(ctypes.c_void_p)
+    lib.demo_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(DemoConfig), ctypes.POINTER(DemoTensorDesc), i32, i32]
+    lib.demo_init.restype = i32
+    lib.demo_payload_bytes.argtypes = [vp]
+    lib.demo_payload_bytes.restype = ctypes.c_size_t
+    lib.demo_payload_layout.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i32)]
+    lib.demo_payload_layout.restype = i32
+    lib.demo_compress.argtypes = [vp, i32, pvp, pvp, vp, vp]
+    lib.demo_compress.restype = i32
+    lib.demo_decode_apply.argtypes = [vp, pvp, i32, pvp, vp]
+    lib.demo_decode_apply.restype = i32
+    lib.demo_step_host.argtypes = [vp, pvp, pvp, pvp, pvp, pvp, vp, vp]
+    lib.demo_step_host.restype = i32
+    lib.demo_set_lr.argtypes = [vp, ctypes.c_float]
+    lib.demo_set_lr.restype = i32
+    lib.demo_set_path.argtypes = [vp, i32]
+    lib.demo_set_path.restype = i32
+    lib.demo_launch_count.argtypes = [vp]
+    lib.demo_launch_count.restype = i64
+    lib.demo_device_status.argtypes = [vp, vp]
+    lib.demo_device_status.restype = i32
+    lib.demo_status_string.argtypes = [i32]
+    lib.demo_status_string.restype = ctypes.c_char_p
+    lib.demo_free.argtypes = [vp]
+    lib.demo_free.restype = None
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def demo_status_string(status: int) -> str:
+    return load_library().demo_status_string(int(status)).decode()
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    return (ctypes.c_void_p * len(ptrs))(*ptrs)
+
+
+def _tensor_ptrs(tensors) -> List[int]:
+    return [int(t.data_ptr()) for t in tensors]
+
+
+class DemoTransform:
+    """One ``demo_ctx``.  ``shapes`` is a list of 1-D / 2-D shapes in payload order."""
+
+    def __init__(self, shapes, *, chunk: int, topk: int, beta: float, lr: float, weight_decay: float,
+                 num_workers: int, grad_dtype: int = DEMO_BF16, device: int = 0):
+        self.lib = load_library()
+        self.shapes = [tuple(int(d) for d in s) for s in shapes]
+        descs = (DemoTensorDesc * len(self.shapes))()
+        for d, s in zip(descs, self.shapes):
+            d.ndim = len(s)
+            for a in range(min(len(s), 2)):
+                d.shape[a] = s[a]
+        self.cfg = DemoConfig(beta, chunk, topk, lr, weight_decay, num_workers, grad_dtype)
+        self.num_workers = num_workers
+        self.device = device
+        self._ctx = ctypes.c_void_p()
+        st = self.lib.demo_init(ctypes.byref(self._ctx), ctypes.byref(self.cfg), descs, len(self.shapes), device)
+        if st != 0:
+            self._ctx = ctypes.c_void_p()
+            raise DemoError(st, "demo_init")
+        self._ptr_cache = {}
+
+    # --- queries -------------------------------------------------------------------------------
+    @property
+    def payload_bytes(self) -> int:
+        return int(self.lib.demo_payload_bytes(self._ctx))
+
+    def payload_layout(self, tensor: int):
+        first, n_chunks, k_eff = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int32()
+        st = self.lib.demo_payload_layout(self._ctx, tensor, ctypes.byref(first), ctypes.byref(n_chunks),
+                                          ctypes.byref(k_eff))
+        if st != 0:
+            raise DemoError(st, "demo_payload_layout")
+        return first.value, n_chunks.value, k_eff.value
+
+    @property
+    def launch_count(self) -> int:
+        return int(self.lib.demo_launch_count(self._ctx))
+
+    # --- marshalling helpers -------------------------------------------------------------------
+    def _array(self, key, tensors):
+        """Pointer array for a list of tensors, cached per list identity and data pointers."""
+        ptrs = tuple(_tensor_ptrs(tensors))
+        hit = self._ptr_cache.get(key)
+        if hit is None or hit[0] != ptrs:
+            hit = (ptrs, _ptr_array(ptrs))
+            self._ptr_cache[key] = hit
+        return hit[1]
+
+    @staticmethod
+    def _stream(stream) -> ctypes.c_void_p:
+        if stream is None:
+            import torch
+
+            stream = torch.cuda.current_stream()
+        return ctypes.c_void_p(int(getattr(stream, "cuda_stream", stream)))
+
+    # --- the ABI calls -------------------------------------------------------------------------
+    def compress(self, worker: int, grads, momentum, payload_out, stream=None) -> None:
+        st = self.lib.demo_compress(self._ctx, worker, self._array(("g", worker), grads),
+                                    self._array(("m", worker), momentum), ctypes.c_void_p(payload_out.data_ptr()),
+                                    self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_compress")
+
+    def decode_apply(self, payloads, params, stream=None) -> None:
+        st = self.lib.demo_decode_apply(self._ctx, self._array("p", payloads), len(payloads),
+                                        self._array("x", params), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_decode_apply")
+
+    def step_host(self, host_grads, dev_grads, momentum, payloads, params, host_payloads_out=None, stream=None) -> None:
+        """host_grads / dev_grads / momentum: lists over workers of lists of tensors."""
+        flat = lambda ll: [t for l in ll for t in l]  # noqa: E731
+        out = ctypes.c_void_p(host_payloads_out.data_ptr()) if host_payloads_out is not None else ctypes.c_void_p()
+        st = self.lib.demo_step_host(self._ctx, self._array("hg", flat(host_grads)), self._array("dg", flat(dev_grads)),
+                                     self._array("mm", flat(momentum)), self._array("p", payloads),
+                                     self._array("x", params), out, self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_step_host")
+
+    def set_lr(self, lr: float) -> None:
+        st = self.lib.demo_set_lr(self._ctx, lr)
+        if st != 0:
+            raise DemoError(st, "demo_set_lr")
+
+    def set_path(self, path: int) -> None:
+        st = self.lib.demo_set_path(self._ctx, path)
+        if st != 0:
+            raise DemoError(st, "demo_set_path")
+
+    def device_status(self, stream=None) -> int:
+        return int(self.lib.demo_device_status(self._ctx, self._stream(stream)))
+
+    def close(self) -> None:
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            self.lib.demo_free(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,79 @@
+// Internal declarations shared by the host library and the kernel translation units.
+// Nothing here is part of the public ABI (see include/demo.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+// One payload record: flat index inside the chunk + fp32 coefficient (8 bytes, little-endian).
+struct DemoRecord {
+    int32_t idx;
+    float val;
+};
+
+// One tensor of a work list.  A work list holds either all 2-D tensors or all 1-D tensors; chunk
+// ids run over the list, row-major over each tensor's chunk grid (blocking operator, appendix
+// B.1.2 of the paper).
+struct DemoTensorEntry {
+    long long chunk_begin;  // id of this tensor's first chunk inside the list
+    long long rec_begin;    // index of this tensor's first record inside a payload
+    int tensor;             // position in the caller's pointer arrays
+    int n1;                 // row length in elements (2-D: shape[1]; 1-D: shape[0])
+    int c1;                 // chunks per row of the chunk grid
+    int k_eff;              // min(k, M)
+};
+
+struct DemoCompressArgs {
+    const DemoTensorEntry *entries;  // device
+    int n_entries;
+    long long n_chunks;
+    const void *const *g_ptrs;  // device array indexed by DemoTensorEntry::tensor
+    float *const *m_ptrs;       // device array
+    DemoRecord *payload;        // device, whole payload of this worker
+    const float *C;             // device, s x s orthonormal DCT-II, C[u*s + n]
+    float beta;
+    int grad_bf16;  // 1: gradients are bf16, 0: fp32
+    int *status;    // device status word (sticky)
+};
+
+struct DemoDecodeArgs {
+    const DemoTensorEntry *entries;
+    int n_entries;
+    long long n_chunks;
+    const DemoRecord *const *payloads;  // device array [W]
+    int W;
+    float *const *x_ptrs;  // device array
+    const float *C;
+    float lr;
+    float wd;
+    int *status;
+};
+
+// Launchers (defined in the kernel translation units).  `s` is the chunk size, `two_d` selects
+// s x s tiles (1) or length-s segments (0).  Return the CUDA error of the launch.
+cudaError_t demo_launch_compress_generic(int s, int two_d, const DemoCompressArgs &a, int sm_count,
+                                         cudaStream_t stream);
+cudaError_t demo_launch_decode_generic(int s, int two_d, const DemoDecodeArgs &a, int sm_count,
+                                       cudaStream_t stream);
+// Fast-DCT kernels for 2-D tensors; `supported` tells whether chunk size s has one.
+bool demo_fast_supported(int s);
+cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
+cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream);
+
+// Locate the tensor that owns chunk id c: the last entry with chunk_begin <= c.
+__device__ __forceinline__ int demo_find_entry(const DemoTensorEntry *entries, int n, long long c)
+{
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (entries[mid].chunk_begin <= c)
+            lo = mid;
+        else
+            hi = mid - 1;
+    }
+    return lo;
+}
+
+// Status values written by kernels (match demo_status in include/demo.h).
+#define DEMO_DEV_TIMEOUT 7
+#define DEMO_DEV_PAYLOAD 8

@@ -1,0 +1,448 @@
+// Host side of the C ABI declared in include/demo.h: context, planner (chunk tables of the blocking
+// operator, payload offsets, DCT basis), pointer-table caching and kernel dispatch.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/demo.h"
+#include "demo_internal.h"
+
+struct demo_ctx {
+    demo_config cfg;
+    int device = 0;
+    int sm_count = 0;
+    int n_tensors = 0;
+    int path = DEMO_PATH_AUTO;
+    long long launches = 0;
+    std::vector<demo_tensor_desc> descs;
+    std::vector<long long> first_record, n_chunks, n_elems;
+    std::vector<int> k_eff;
+    long long total_records = 0;
+
+    // work lists
+    int n2d = 0, n1d = 0;
+    long long chunks2d = 0, chunks1d = 0;
+    DemoTensorEntry *d_entries2d = nullptr, *d_entries1d = nullptr;
+
+    float *d_C = nullptr;
+    int *d_status = nullptr;
+
+    // device pointer tables and their host mirrors (uploaded only when the caller's pointers change)
+    const void **d_g = nullptr;      // [W][T]
+    float **d_m = nullptr;           // [W][T]
+    float **d_x = nullptr;           // [T]
+    const DemoRecord **d_p = nullptr;  // [W]
+    std::vector<const void *> h_g;
+    std::vector<float *> h_m, h_x;
+    std::vector<const DemoRecord *> h_p;
+    std::vector<char> g_valid, m_valid;  // per worker
+    bool x_valid = false, p_valid = false;
+};
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+// Upload `n` pointers to dev[0..n) if they differ from the mirror.  The mirror is pageable host
+// memory: cudaMemcpyAsync stages it before returning, so it may be overwritten by the next call.
+template <typename T>
+cudaError_t sync_table(T *dev, T *mirror, const T *now, int n, bool *valid, cudaStream_t stream)
+{
+    if (*valid && std::memcmp(mirror, now, sizeof(T) * (size_t)n) == 0) return cudaSuccess;
+    std::memcpy(mirror, now, sizeof(T) * (size_t)n);
+    cudaError_t err = cudaMemcpyAsync(dev, mirror, sizeof(T) * (size_t)n, cudaMemcpyHostToDevice, stream);
+    *valid = (err == cudaSuccess);
+    return err;
+}
+
+void release(demo_ctx *c)
+{
+    if (!c) return;
+    cudaFree(c->d_entries2d);
+    cudaFree(c->d_entries1d);
+    cudaFree(c->d_C);
+    cudaFree(c->d_status);
+    cudaFree((void *)c->d_g);
+    cudaFree((void *)c->d_m);
+    cudaFree((void *)c->d_x);
+    cudaFree((void *)c->d_p);
+    delete c;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *demo_status_string(demo_status status)
+{
+    switch (status) {
+        case DEMO_OK: return "ok";
+        case DEMO_ERR_INVALID_ARG: return "invalid argument";
+        case DEMO_ERR_SHAPE: return "tensor shape is not 1-D/2-D with dimensions divisible by the chunk size";
+        case DEMO_ERR_K: return "k out of range (1 <= k <= s*s)";
+        case DEMO_ERR_UNSUPPORTED: return "unsupported chunk size, dtype or tensor count";
+        case DEMO_ERR_ALLOC: return "allocation failed";
+        case DEMO_ERR_CUDA: return "CUDA runtime error";
+        case DEMO_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case DEMO_ERR_PAYLOAD: return "payload record index outside its chunk";
+        default: return "unknown status";
+    }
+}
+
+demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_desc *tensors, int32_t n_tensors,
+                      int32_t cuda_device)
+{
+    if (out) *out = nullptr;
+    if (!out || !cfg || !tensors || n_tensors < 1 || cuda_device < 0) return DEMO_ERR_INVALID_ARG;
+    if (cfg->num_workers < 1 || cfg->num_workers > 4096) return DEMO_ERR_INVALID_ARG;
+    if (!std::isfinite(cfg->beta) || !std::isfinite(cfg->lr) || !std::isfinite(cfg->weight_decay))
+        return DEMO_ERR_INVALID_ARG;
+    const int s = cfg->chunk;
+    if (!(s == 8 || s == 16 || s == 32 || s == 64 || s == 128)) return DEMO_ERR_UNSUPPORTED;
+    if (cfg->grad_dtype != DEMO_F32 && cfg->grad_dtype != DEMO_BF16) return DEMO_ERR_UNSUPPORTED;
+    if (n_tensors > (1 << 20)) return DEMO_ERR_UNSUPPORTED;
+    if (cfg->topk < 1 || (long long)cfg->topk > (long long)s * s) return DEMO_ERR_K;
+    for (int t = 0; t < n_tensors; ++t) {
+        const demo_tensor_desc &d = tensors[t];
+        if (d.ndim != 1 && d.ndim != 2) return DEMO_ERR_SHAPE;
+        for (int a = 0; a < d.ndim; ++a)
+            if (d.shape[a] < s || d.shape[a] % s != 0 || d.shape[a] > (1LL << 31) - 1) return DEMO_ERR_SHAPE;
+    }
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cuda_device >= n_dev) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    DeviceGuard guard(cuda_device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+
+    demo_ctx *c = new (std::nothrow) demo_ctx();
+    if (!c) return DEMO_ERR_ALLOC;
+    c->cfg = *cfg;
+    c->device = cuda_device;
+    c->n_tensors = n_tensors;
+    if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cuda_device) != cudaSuccess) {
+        release(c);
+        return DEMO_ERR_CUDA;
+    }
+
+    // planner: payload offsets and the two work lists (2-D tiles, 1-D segments)
+    std::vector<DemoTensorEntry> e2d, e1d;
+    try {
+        c->descs.assign(tensors, tensors + n_tensors);
+        c->first_record.resize(n_tensors);
+        c->n_chunks.resize(n_tensors);
+        c->n_elems.resize(n_tensors);
+        c->k_eff.resize(n_tensors);
+        long long rec = 0;
+        for (int t = 0; t < n_tensors; ++t) {
+            const demo_tensor_desc &d = tensors[t];
+            const bool two = d.ndim == 2;
+            const long long n1 = two ? d.shape[1] : d.shape[0];
+            const long long c0 = two ? d.shape[0] / s : 1, c1 = n1 / s;
+            const long long M = two ? (long long)s * s : s;
+            DemoTensorEntry e;
+            e.tensor = t;
+            e.n1 = (int)n1;
+            e.c1 = (int)c1;
+            e.k_eff = (int)(cfg->topk < M ? cfg->topk : M);
+            e.rec_begin = rec;
+            e.chunk_begin = two ? c->chunks2d : c->chunks1d;
+            (two ? c->chunks2d : c->chunks1d) += c0 * c1;
+            (two ? e2d : e1d).push_back(e);
+            c->first_record[t] = rec;
+            c->n_chunks[t] = c0 * c1;
+            c->n_elems[t] = two ? d.shape[0] * d.shape[1] : d.shape[0];
+            c->k_eff[t] = e.k_eff;
+            rec += c0 * c1 * e.k_eff;
+        }
+        c->total_records = rec;
+        const size_t W = (size_t)cfg->num_workers, T = (size_t)n_tensors;
+        c->h_g.assign(W * T, nullptr);
+        c->h_m.assign(W * T, nullptr);
+        c->h_x.assign(T, nullptr);
+        c->h_p.assign(W, nullptr);
+        c->g_valid.assign(W, 0);
+        c->m_valid.assign(W, 0);
+    } catch (const std::bad_alloc &) {
+        release(c);
+        return DEMO_ERR_ALLOC;
+    }
+    c->n2d = (int)e2d.size();
+    c->n1d = (int)e1d.size();
+
+    // orthonormal DCT-II basis, built in fp64 and rounded once to fp32:
+    // C[u][n] = a_u cos(pi (2n+1) u / (2s)), a_0 = sqrt(1/s), a_u = sqrt(2/s)
+    std::vector<float> C((size_t)s * s);
+    {
+        const double pi = 3.141592653589793238462643383279502884;
+        for (int u = 0; u < s; ++u)
+            for (int n = 0; n < s; ++n) {
+                const double a = (u == 0) ? std::sqrt(1.0 / s) : std::sqrt(2.0 / s);
+                C[(size_t)u * s + n] = (float)(a * std::cos(pi * (2.0 * n + 1.0) * u / (2.0 * s)));
+            }
+    }
+
+    const size_t W = (size_t)cfg->num_workers, T = (size_t)n_tensors;
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->d_C, C.size() * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+    if (ok && c->n2d) ok = cudaMalloc(&c->d_entries2d, e2d.size() * sizeof(DemoTensorEntry)) == cudaSuccess;
+    if (ok && c->n1d) ok = cudaMalloc(&c->d_entries1d, e1d.size() * sizeof(DemoTensorEntry)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_g, W * T * sizeof(void *)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_m, W * T * sizeof(void *)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_x, T * sizeof(void *)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_p, W * sizeof(void *)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        release(c);
+        return DEMO_ERR_ALLOC;
+    }
+    ok = ok && cudaMemcpy(c->d_C, C.data(), C.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+    if (ok && c->n2d)
+        ok = cudaMemcpy(c->d_entries2d, e2d.data(), e2d.size() * sizeof(DemoTensorEntry), cudaMemcpyHostToDevice) ==
+             cudaSuccess;
+    if (ok && c->n1d)
+        ok = cudaMemcpy(c->d_entries1d, e1d.data(), e1d.size() * sizeof(DemoTensorEntry), cudaMemcpyHostToDevice) ==
+             cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        release(c);
+        return DEMO_ERR_CUDA;
+    }
+    *out = c;
+    return DEMO_OK;
+}
+
+size_t demo_payload_bytes(const demo_ctx *ctx) { return ctx ? (size_t)ctx->total_records * sizeof(DemoRecord) : 0; }
+
+demo_status demo_payload_layout(const demo_ctx *ctx, int32_t tensor, int64_t *first_record, int64_t *n_chunks,
+                                int32_t *k_eff)
+{
+    if (!ctx || tensor < 0 || tensor >= ctx->n_tensors) return DEMO_ERR_INVALID_ARG;
+    if (first_record) *first_record = ctx->first_record[tensor];
+    if (n_chunks) *n_chunks = ctx->n_chunks[tensor];
+    if (k_eff) *k_eff = ctx->k_eff[tensor];
+    return DEMO_OK;
+}
+
+demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grads, float *const *momentum,
+                          void *payload_out, void *cuda_stream)
+{
+    if (!ctx || !grads || !momentum || !payload_out) return DEMO_ERR_INVALID_ARG;
+    if (worker < 0 || worker >= ctx->cfg.num_workers) return DEMO_ERR_INVALID_ARG;
+    if (!aligned16(payload_out)) return DEMO_ERR_INVALID_ARG;
+    const int T = ctx->n_tensors;
+    for (int t = 0; t < T; ++t)
+        if (!grads[t] || !momentum[t] || !aligned16(grads[t]) || !aligned16(momentum[t])) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    const size_t row = (size_t)worker * (size_t)T;
+    bool gv = ctx->g_valid[worker] != 0, mv = ctx->m_valid[worker] != 0;
+    cudaError_t err = sync_table<const void *>(ctx->d_g + row, ctx->h_g.data() + row, grads, T, &gv, stream);
+    ctx->g_valid[worker] = gv;
+    if (err == cudaSuccess) {
+        err = sync_table<float *>(ctx->d_m + row, ctx->h_m.data() + row, const_cast<float *const *>(momentum), T, &mv,
+                                  stream);
+        ctx->m_valid[worker] = mv;
+    }
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+
+    DemoCompressArgs a;
+    a.g_ptrs = ctx->d_g + row;
+    a.m_ptrs = ctx->d_m + row;
+    a.payload = static_cast<DemoRecord *>(payload_out);
+    a.C = ctx->d_C;
+    a.beta = ctx->cfg.beta;
+    a.grad_bf16 = ctx->cfg.grad_dtype == DEMO_BF16;
+    a.status = ctx->d_status;
+    const int s = ctx->cfg.chunk;
+    if (ctx->n2d) {
+        a.entries = ctx->d_entries2d;
+        a.n_entries = ctx->n2d;
+        a.n_chunks = ctx->chunks2d;
+        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s))
+            err = demo_launch_compress_fast(s, a, ctx->sm_count, stream);
+        else
+            err = demo_launch_compress_generic(s, 1, a, ctx->sm_count, stream);
+        ctx->launches += 1;
+    }
+    if (err == cudaSuccess && ctx->n1d) {
+        a.entries = ctx->d_entries1d;
+        a.n_entries = ctx->n1d;
+        a.n_chunks = ctx->chunks1d;
+        err = demo_launch_compress_generic(s, 0, a, ctx->sm_count, stream);
+        ctx->launches += 1;
+    }
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    return DEMO_OK;
+}
+
+demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads, float *const *params,
+                              void *cuda_stream)
+{
+    if (!ctx || !payloads || !params) return DEMO_ERR_INVALID_ARG;
+    if (n_payloads != ctx->cfg.num_workers) return DEMO_ERR_INVALID_ARG;
+    const int T = ctx->n_tensors, W = n_payloads;
+    for (int w = 0; w < W; ++w)
+        if (!payloads[w] || !aligned16(payloads[w])) return DEMO_ERR_INVALID_ARG;
+    for (int t = 0; t < T; ++t)
+        if (!params[t] || !aligned16(params[t])) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    cudaError_t err = sync_table<const DemoRecord *>(ctx->d_p, ctx->h_p.data(),
+                                                     reinterpret_cast<const DemoRecord *const *>(payloads), W,
+                                                     &ctx->p_valid, stream);
+    if (err == cudaSuccess)
+        err = sync_table<float *>(ctx->d_x, ctx->h_x.data(), const_cast<float *const *>(params), T, &ctx->x_valid,
+                                  stream);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+
+    DemoDecodeArgs a;
+    a.payloads = ctx->d_p;
+    a.W = W;
+    a.x_ptrs = ctx->d_x;
+    a.C = ctx->d_C;
+    a.lr = ctx->cfg.lr;
+    a.wd = ctx->cfg.weight_decay;
+    a.status = ctx->d_status;
+    const int s = ctx->cfg.chunk;
+    if (ctx->n2d) {
+        a.entries = ctx->d_entries2d;
+        a.n_entries = ctx->n2d;
+        a.n_chunks = ctx->chunks2d;
+        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s))
+            err = demo_launch_decode_fast(s, a, ctx->sm_count, stream);
+        else
+            err = demo_launch_decode_generic(s, 1, a, ctx->sm_count, stream);
+        ctx->launches += 1;
+    }
+    if (err == cudaSuccess && ctx->n1d) {
+        a.entries = ctx->d_entries1d;
+        a.n_entries = ctx->n1d;
+        a.n_chunks = ctx->chunks1d;
+        err = demo_launch_decode_generic(s, 0, a, ctx->sm_count, stream);
+        ctx->launches += 1;
+    }
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    return DEMO_OK;
+}
+
+demo_status demo_step_host(demo_ctx *ctx, const void *const *host_grads, void *const *dev_grads,
+                           float *const *momentum, void *const *payloads, float *const *params,
+                           void *host_payloads_out, void *cuda_stream)
+{
+    if (!ctx || !host_grads || !dev_grads || !momentum || !payloads || !params) return DEMO_ERR_INVALID_ARG;
+    const int T = ctx->n_tensors, W = ctx->cfg.num_workers;
+    const size_t gsize = ctx->cfg.grad_dtype == DEMO_BF16 ? 2 : 4;
+    for (size_t i = 0; i < (size_t)W * T; ++i)
+        if (!host_grads[i] || !dev_grads[i]) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (int w = 0; w < W; ++w) {
+        const size_t row = (size_t)w * T;
+        for (int t = 0; t < T; ++t) {
+            if (cudaMemcpyAsync(dev_grads[row + t], host_grads[row + t], (size_t)ctx->n_elems[t] * gsize,
+                                cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return DEMO_ERR_CUDA;
+            }
+        }
+        demo_status st = demo_compress(ctx, w, const_cast<const void *const *>(dev_grads + row), momentum + row,
+                                       payloads[w], cuda_stream);
+        if (st != DEMO_OK) return st;
+    }
+    demo_status st = demo_decode_apply(ctx, const_cast<const void *const *>(payloads), W, params, cuda_stream);
+    if (st != DEMO_OK) return st;
+    if (host_payloads_out) {
+        const size_t pb = demo_payload_bytes(ctx);
+        for (int w = 0; w < W; ++w)
+            if (cudaMemcpyAsync(static_cast<char *>(host_payloads_out) + (size_t)w * pb, payloads[w], pb,
+                                cudaMemcpyDeviceToHost, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return DEMO_ERR_CUDA;
+            }
+    }
+    return DEMO_OK;
+}
+
+demo_status demo_set_lr(demo_ctx *ctx, float lr)
+{
+    if (!ctx || !std::isfinite(lr)) return DEMO_ERR_INVALID_ARG;
+    ctx->cfg.lr = lr;
+    return DEMO_OK;
+}
+
+demo_status demo_set_path(demo_ctx *ctx, int32_t path)
+{
+    if (!ctx || (path != DEMO_PATH_AUTO && path != DEMO_PATH_GENERIC)) return DEMO_ERR_INVALID_ARG;
+    ctx->path = path;
+    return DEMO_OK;
+}
+
+int64_t demo_launch_count(const demo_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+demo_status demo_device_status(demo_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    if (word != 0 && (cudaMemsetAsync(ctx->d_status, 0, sizeof(int), stream) != cudaSuccess ||
+                      cudaStreamSynchronize(stream) != cudaSuccess)) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    if (word == DEMO_DEV_TIMEOUT) return DEMO_ERR_TIMEOUT;
+    if (word == DEMO_DEV_PAYLOAD) return DEMO_ERR_PAYLOAD;
+    return word == 0 ? DEMO_OK : DEMO_ERR_CUDA;
+}
+
+void demo_free(demo_ctx *ctx)
+{
+    if (!ctx) return;
+    DeviceGuard guard(ctx->device);
+    release(ctx);
+}
+
+}  // extern "C"

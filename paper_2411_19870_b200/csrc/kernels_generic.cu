@@ -1,0 +1,362 @@
+// Generic kernels of the DeMo optimizer transform: any chunk size s in {8,16,32,64,128}, 2-D tiles
+// and 1-D segments, any k <= M.  One CTA works on one chunk at a time; the chunk stays in shared
+// memory from the momentum update to the residual write-back, so HBM is touched once per operand.
+// The chunk DCT here is the dense contraction with the precomputed basis (the paper's own cost
+// model, Section 2.1 "Complexity Analysis"); the register-resident fast-DCT kernels for the common
+// sizes live in kernels_fast.cu.  These kernels are the path for 1-D tensors, for s in {8,16,128}
+// and the cross-check of the fast path.
+#include <cuda_bf16.h>
+
+#include "demo_internal.h"
+
+namespace {
+
+constexpr int GEN_THREADS = 256;
+
+// out[r][c] = sum_t L[r*lsr + t*lst] * R[t*rst + c*rsc]   (r < NR, c < NC, t < NT; out row-major)
+template <int NR, int NC, int NT>
+__device__ __forceinline__ void mm(float *__restrict__ out, const float *__restrict__ L, int lsr, int lst,
+                                   const float *__restrict__ R, int rst, int rsc)
+{
+    constexpr int TR = (NR >= 4) ? 4 : 1;
+    constexpr int TC = 4;
+    constexpr int tiles_c = NC / TC;
+    constexpr int n_tiles = (NR / TR) * tiles_c;
+    for (int tile = threadIdx.x; tile < n_tiles; tile += GEN_THREADS) {
+        const int r0 = (tile / tiles_c) * TR, c0 = (tile % tiles_c) * TC;
+        float acc[TR][TC];
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+#pragma unroll
+            for (int j = 0; j < TC; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+        for (int t = 0; t < NT; ++t) {
+            float l[TR], rr[TC];
+#pragma unroll
+            for (int i = 0; i < TR; ++i) l[i] = L[(r0 + i) * lsr + t * lst];
+#pragma unroll
+            for (int j = 0; j < TC; ++j) rr[j] = R[t * rst + (c0 + j) * rsc];
+#pragma unroll
+            for (int i = 0; i < TR; ++i)
+#pragma unroll
+                for (int j = 0; j < TC; ++j) acc[i][j] = fmaf(l[i], rr[j], acc[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+#pragma unroll
+            for (int j = 0; j < TC; ++j) out[(r0 + i) * NC + c0 + j] = acc[i][j];
+    }
+}
+
+// Forward chunk DCT: 2-D  Q = C B C^T,  1-D  q = C b.  Result in `q_out`, `tmp` is scratch.
+template <int S, int ROWS>
+__device__ __forceinline__ void forward_dct(const float *Bt, float *tmp, float *q_out, const float *C)
+{
+    if (ROWS > 1) {
+        mm<ROWS, S, S>(tmp, Bt, S, 1, C, 1, S);  // tmp[i][v] = sum_j B[i][j] C[v][j]
+        __syncthreads();
+        mm<S, S, S>(q_out, C, S, 1, tmp, S, 1);  // Q[u][v] = sum_i C[u][i] tmp[i][v]
+    } else {
+        mm<ROWS, S, S>(q_out, Bt, S, 1, C, 1, S);
+    }
+    __syncthreads();
+}
+
+// Inverse chunk DCT: 2-D  R = C^T Q C,  1-D  r = C^T q.  Result in `r_out`, `tmp` is scratch.
+template <int S, int ROWS>
+__device__ __forceinline__ void inverse_dct(const float *Qt, float *tmp, float *r_out, const float *C)
+{
+    if (ROWS > 1) {
+        mm<ROWS, S, S>(tmp, Qt, S, 1, C, S, 1);   // tmp[u][j] = sum_v Q[u][v] C[v][j]
+        __syncthreads();
+        mm<S, S, S>(r_out, C, 1, S, tmp, S, 1);   // R[i][j] = sum_u C[u][i] tmp[u][j]
+    } else {
+        mm<ROWS, S, S>(r_out, Qt, S, 1, C, S, 1);
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+// Exclusive prefix sum of one unsigned per thread over the 256-thread CTA.
+__device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned *warp_tot /*[8]*/)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        unsigned n = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= d) inc += n;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    unsigned base = 0;
+    for (int w = 0; w < warp; ++w) base += warp_tot[w];
+    __syncthreads();
+    return base + inc - v;
+}
+
+// Exact k-th largest magnitude of Q[0..M) by radix select on the fp32 magnitude bits (which order
+// like the magnitudes).  Returns the key of the k-th largest in *thr and, in *need_eq, how many
+// elements EQUAL to it belong to the top-k (those with the lowest indices are taken).
+template <int M>
+__device__ __forceinline__ void radix_select(const float *Q, int k_eff, unsigned *hist, unsigned *s_state,
+                                             unsigned *thr, unsigned *need_eq)
+{
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        s_state[0] = 0u;              // prefix of the key found so far
+        s_state[1] = (unsigned)k_eff; // rank still to resolve inside the prefix class
+    }
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const unsigned mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
+        hist[tid] = 0u;
+        __syncthreads();
+        const unsigned prefix = s_state[0];
+        for (int i = tid; i < M; i += GEN_THREADS) {
+            const unsigned key = mag_key(Q[i]);
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (tid < 32) {
+            // lane l owns bins 255-8l ... 248-8l (descending magnitude)
+            const unsigned rem = s_state[1];
+            unsigned local = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) local += hist[255 - 8 * tid - j];
+            unsigned inc = local;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                unsigned n = __shfl_up_sync(0xffffffffu, inc, d);
+                if (tid >= d) inc += n;
+            }
+            const unsigned before = inc - local;
+            if (before < rem && rem <= inc) {  // exactly one lane
+                unsigned cum = before;
+                int b = 255 - 8 * tid;
+                for (int j = 0; j < 8; ++j, --b) {
+                    const unsigned h = hist[b];
+                    if (cum + h >= rem) break;
+                    cum += h;
+                }
+                s_state[1] = rem - cum;
+                s_state[0] = prefix | ((unsigned)b << shift);
+            }
+        }
+        __syncthreads();
+    }
+    *thr = s_state[0];
+    *need_eq = s_state[1];
+    __syncthreads();
+}
+
+template <int S, int ROWS>
+__global__ void __launch_bounds__(GEN_THREADS) compress_generic_kernel(DemoCompressArgs a)
+{
+    constexpr int M = ROWS * S;
+    extern __shared__ float smem[];
+    float *Bt = smem;
+    float *X1 = Bt + M;
+    float *X2 = X1 + M;
+    unsigned *hist = reinterpret_cast<unsigned *>(X2 + M);  // [256]
+    unsigned *warp_tot = hist + 256;                        // [8]
+    unsigned *s_state = warp_tot + 8;                       // [2]
+    const int tid = threadIdx.x;
+
+    for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
+        const DemoTensorEntry te = a.entries[demo_find_entry(a.entries, a.n_entries, c)];
+        const long long lc = c - te.chunk_begin;
+        const long long k0 = lc / te.c1;
+        const int k1 = (int)(lc - k0 * te.c1);
+        const size_t base = (size_t)k0 * ROWS * (size_t)te.n1 + (size_t)k1 * S;
+        float *__restrict__ m = a.m_ptrs[te.tensor];
+        const void *g = a.g_ptrs[te.tensor];
+        const int k_eff = te.k_eff;
+
+        // momentum update  B = beta*m + g  on the chunk (Algorithm 1, worker side)
+        for (int i = tid; i < M; i += GEN_THREADS) {
+            const int r = i / S, j = i - r * S;
+            const size_t off = base + (size_t)r * te.n1 + j;
+            const float gv = a.grad_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(g)[off])
+                                         : reinterpret_cast<const float *>(g)[off];
+            Bt[i] = fmaf(a.beta, m[off], gv);
+        }
+        __syncthreads();
+
+        float *Q = (ROWS > 1) ? X2 : X1;   // coefficients
+        float *O = (ROWS > 1) ? X1 : X2;   // the other buffer
+        forward_dct<S, ROWS>(Bt, X1, Q, a.C);
+
+        // top-k: threshold by radix select, then index-ordered compaction into the payload
+        unsigned thr, need_eq;
+        radix_select<M>(Q, k_eff, hist, s_state, &thr, &need_eq);
+        constexpr int PER = (M + GEN_THREADS - 1) / GEN_THREADS;
+        const int start = tid * PER;
+        unsigned gt = 0, eq = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int i = start + j;
+            if (i < M) {
+                const unsigned key = mag_key(Q[i]);
+                gt += key > thr;
+                eq += key == thr;
+            }
+        }
+        const unsigned before = block_exclusive_scan(gt | (eq << 16), warp_tot);
+        unsigned gb = before & 0xffffu, eb = before >> 16;
+        DemoRecord *rec = a.payload + te.rec_begin + lc * (long long)k_eff;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int i = start + j;
+            if (i < M) {
+                const float v = Q[i];
+                const unsigned key = mag_key(v);
+                bool sel = false;
+                unsigned pos = 0;
+                if (key > thr) {
+                    pos = gb + min(eb, need_eq);
+                    ++gb;
+                    sel = true;
+                } else if (key == thr) {
+                    if (eb < need_eq) {
+                        pos = gb + eb;
+                        sel = true;
+                    }
+                    ++eb;
+                }
+                if (sel) {
+                    DemoRecord r;
+                    r.idx = i;
+                    r.val = v;
+                    rec[pos] = r;
+                }
+                O[i] = sel ? v : 0.f;
+            }
+        }
+        __syncthreads();
+
+        // momentum subtraction  m <- B - IDCT(kept coefficients)
+        float *R = (ROWS > 1) ? O : Q;
+        inverse_dct<S, ROWS>(O, Q, R, a.C);
+        for (int i = tid; i < M; i += GEN_THREADS) {
+            const int r = i / S, j = i - r * S;
+            m[base + (size_t)r * te.n1 + j] = Bt[i] - R[i];
+        }
+        __syncthreads();
+    }
+}
+
+template <int S, int ROWS>
+__global__ void __launch_bounds__(GEN_THREADS) decode_generic_kernel(DemoDecodeArgs a)
+{
+    constexpr int M = ROWS * S;
+    extern __shared__ float smem[];
+    float *St = smem;
+    float *X1 = St + M;
+    const int tid = threadIdx.x;
+
+    for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
+        const DemoTensorEntry te = a.entries[demo_find_entry(a.entries, a.n_entries, c)];
+        const long long lc = c - te.chunk_begin;
+        const long long k0 = lc / te.c1;
+        const int k1 = (int)(lc - k0 * te.c1);
+        const size_t base = (size_t)k0 * ROWS * (size_t)te.n1 + (size_t)k1 * S;
+        float *__restrict__ x = a.x_ptrs[te.tensor];
+        const int k_eff = te.k_eff;
+        const long long rec_off = te.rec_begin + lc * (long long)k_eff;
+
+        for (int i = tid; i < M; i += GEN_THREADS) St[i] = 0.f;
+        __syncthreads();
+        // aggregate: S = sum over workers, in worker order (Decompress&Aggregate); indices are
+        // unique inside one worker's chunk, so a barrier per worker fixes the summation order
+        for (int w = 0; w < a.W; ++w) {
+            const DemoRecord *rec = a.payloads[w] + rec_off;
+            for (int i = tid; i < k_eff; i += GEN_THREADS) {
+                const DemoRecord r = rec[i];
+                if ((unsigned)r.idx < (unsigned)M)
+                    St[r.idx] += r.val;
+                else
+                    atomicMax(a.status, DEMO_DEV_PAYLOAD);
+            }
+            __syncthreads();
+        }
+        float *R = (ROWS > 1) ? St : X1;
+        inverse_dct<S, ROWS>(St, X1, R, a.C);
+        // x <- x - lr * (sign(R) + wd * x), sign(0) = 0
+        for (int i = tid; i < M; i += GEN_THREADS) {
+            const int r = i / S, j = i - r * S;
+            const size_t off = base + (size_t)r * te.n1 + j;
+            const float rv = R[i];
+            const float sg = (float)((rv > 0.f) - (rv < 0.f));
+            const float xv = x[off];
+            x[off] = fmaf(-a.lr, fmaf(a.wd, xv, sg), xv);
+        }
+        __syncthreads();
+    }
+}
+
+template <typename K>
+cudaError_t launch_persistent(K kernel, size_t smem, long long n_chunks, int sm_count, cudaStream_t stream,
+                              const void *args_struct_ptr)
+{
+    if (n_chunks <= 0) return cudaSuccess;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    int per_sm = 0;
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, GEN_THREADS, smem);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    long long grid = (long long)sm_count * per_sm;
+    if (grid > n_chunks) grid = n_chunks;
+    void *params[] = {const_cast<void *>(args_struct_ptr)};
+    return cudaLaunchKernel((const void *)kernel, dim3((unsigned)grid), dim3(GEN_THREADS), params, smem, stream);
+}
+
+template <int S>
+cudaError_t compress_dispatch(int two_d, const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
+{
+    const size_t extra = (256 + 8 + 2) * sizeof(unsigned);
+    if (two_d)
+        return launch_persistent(compress_generic_kernel<S, S>, 3 * S * S * sizeof(float) + extra, a.n_chunks,
+                                 sm_count, stream, &a);
+    return launch_persistent(compress_generic_kernel<S, 1>, 3 * S * sizeof(float) + extra, a.n_chunks, sm_count,
+                             stream, &a);
+}
+
+template <int S>
+cudaError_t decode_dispatch(int two_d, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
+{
+    if (two_d)
+        return launch_persistent(decode_generic_kernel<S, S>, 2 * S * S * sizeof(float), a.n_chunks, sm_count,
+                                 stream, &a);
+    return launch_persistent(decode_generic_kernel<S, 1>, 2 * S * sizeof(float), a.n_chunks, sm_count, stream, &a);
+}
+
+}  // namespace
+
+cudaError_t demo_launch_compress_generic(int s, int two_d, const DemoCompressArgs &a, int sm_count,
+                                         cudaStream_t stream)
+{
+    switch (s) {
+        case 8: return compress_dispatch<8>(two_d, a, sm_count, stream);
+        case 16: return compress_dispatch<16>(two_d, a, sm_count, stream);
+        case 32: return compress_dispatch<32>(two_d, a, sm_count, stream);
+        case 64: return compress_dispatch<64>(two_d, a, sm_count, stream);
+        case 128: return compress_dispatch<128>(two_d, a, sm_count, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+cudaError_t demo_launch_decode_generic(int s, int two_d, const DemoDecodeArgs &a, int sm_count,
+                                       cudaStream_t stream)
+{
+    switch (s) {
+        case 8: return decode_dispatch<8>(two_d, a, sm_count, stream);
+        case 16: return decode_dispatch<16>(two_d, a, sm_count, stream);
+        case 32: return decode_dispatch<32>(two_d, a, sm_count, stream);
+        case 64: return decode_dispatch<64>(two_d, a, sm_count, stream);
+        case 128: return decode_dispatch<128>(two_d, a, sm_count, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}

@@ -1,0 +1,223 @@
+"""Comparison harness: CUDA path (through the C ABI) against the fp64 CPU oracle, chunk by chunk.
+
+Rules (written here once, used by every GPU parity test):
+  * values / residual momentum / parameters:  |gpu - ref| <= 1e-5*|ref| + 1e-7*max(1, ||ref_chunk||_inf)
+  * top-k index sets are compared bit for bit wherever the oracle's k-th and (k+1)-th magnitudes
+    differ by more than 1e-5 relative (and the k-th is above the noise floor 1e-6*||Q||_inf);
+    elsewhere the GPU's set must be a VALID top-k (selected magnitudes >= a_k(1-1e-5) - floor,
+    unselected <= a_k(1+1e-5) + floor, ascending, unique, in range) and the oracle continues from
+    the GPU's index set ("forced-index" residual);
+  * decode is checked by feeding the GPU-written payload bytes to the oracle decode; the sign may
+    differ only where |R| < 1e-6*max(1, ||R_chunk||_inf).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import demo_oracle as orc
+
+RTOL = 1e-5
+ATOL = 1e-7
+GAP_RTOL = 1e-5
+FLOOR_REL = 1e-6
+SIGN_EXEMPT = 1e-6
+
+
+def sample_chunk_ids(n_chunks: int, max_n: int, seed: int) -> np.ndarray:
+    if n_chunks <= max_n:
+        return np.arange(n_chunks, dtype=np.int64)
+    rng = np.random.default_rng(seed)
+    mid = rng.choice(np.arange(1, n_chunks - 1), size=max_n - 2, replace=False)
+    return np.sort(np.concatenate([[0, n_chunks - 1], mid])).astype(np.int64)
+
+
+def gather_tiles(t: torch.Tensor, s: int, chunk_ids: np.ndarray) -> np.ndarray:
+    """Tiles of the listed chunks (row-major chunk ids) as float64 [n, M]."""
+    ids = torch.as_tensor(chunk_ids, device=t.device)
+    if t.dim() == 2:
+        c0, c1 = t.shape[0] // s, t.shape[1] // s
+        v = t.view(c0, s, c1, s)
+        tiles = v[ids // c1, :, ids % c1, :]  # [n, s, s]
+    else:
+        tiles = t.view(-1, s)[ids]
+    return tiles.reshape(len(chunk_ids), -1).to(torch.float64).cpu().numpy()
+
+
+def gather_records(payload: torch.Tensor, first_record: int, k_eff: int, chunk_ids: np.ndarray) -> np.ndarray:
+    """Records of the listed chunks of one tensor from a uint8 payload buffer -> [n, k_eff] records."""
+    rec = payload.view(torch.int32).view(-1, 2)
+    ids = torch.as_tensor(chunk_ids, device=payload.device)
+    rows = first_record + ids[:, None] * k_eff + torch.arange(k_eff, device=payload.device)[None, :]
+    got = rec[rows.reshape(-1)].cpu().numpy().reshape(len(chunk_ids), k_eff, 2)
+    out = np.zeros((len(chunk_ids), k_eff), dtype=orc.RECORD_DTYPE)
+    out["idx"] = got[:, :, 0]
+    out["val"] = got[:, :, 1].copy().view(np.float32)
+    return out
+
+
+def _tol(ref: np.ndarray) -> np.ndarray:
+    scale = np.maximum(1.0, np.max(np.abs(ref), axis=-1, keepdims=True))
+    return RTOL * np.abs(ref) + ATOL * scale
+
+
+class Report(dict):
+    def add(self, key, n=1):
+        self[key] = self.get(key, 0) + int(n)
+
+
+def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, report: Report, what=""):
+    """All arguments are per-chunk arrays of the same n chunks (float64 / records)."""
+    M = rows * s
+    k_eff = min(k, M)
+    n = g.shape[0]
+    ref = orc.compress_chunks(g, m_before, s, rows, k, beta)
+    Q = ref["Q"]
+    qinf = np.max(np.abs(Q), axis=1)
+    floor = FLOOR_REL * qinf
+    a_k, a_k1 = ref["gap"][:, 0], ref["gap"][:, 1]
+    pinned = (k_eff == M) | (((a_k - a_k1) > GAP_RTOL * a_k) & (a_k > floor))
+    idx_gpu = rec_gpu["idx"].astype(np.int64)
+    val_gpu = rec_gpu["val"].astype(np.float64)
+
+    # structural checks on every chunk: in range, strictly ascending (hence unique)
+    assert idx_gpu.min() >= 0 and idx_gpu.max() < M, what + ": record index out of range"
+    if k_eff > 1:
+        assert np.all(np.diff(idx_gpu, axis=1) > 0), what + ": record indices not strictly ascending"
+
+    # pinned chunks: bit-exact index sets
+    same = np.all(idx_gpu == ref["idx"], axis=1)
+    bad = pinned & ~same
+    assert not bad.any(), "%s: top-k index set differs on %d pinned chunk(s), first %d" % (
+        what, bad.sum(), int(np.argmax(bad)))
+    report.add("chunks", n)
+    report.add("pinned", pinned.sum())
+    report.add("unpinned", (~pinned).sum())
+    report.add("unpinned_same_set", (~pinned & same).sum())
+
+    # unpinned chunks with a different set: the GPU's set must be a valid top-k of the oracle's Q
+    diff = np.nonzero(~same)[0]
+    for c in diff:
+        mag = np.abs(Q[c])
+        sel = np.zeros(M, bool)
+        sel[idx_gpu[c]] = True
+        lo = a_k[c] * (1 - GAP_RTOL) - floor[c]
+        hi = a_k[c] * (1 + GAP_RTOL) + floor[c]
+        assert mag[sel].min() >= lo, what + ": chunk %d selected a coefficient below the threshold band" % c
+        if k_eff < M:
+            assert mag[~sel].max() <= hi, what + ": chunk %d missed a coefficient above the threshold band" % c
+
+    # values at the GPU's own indices
+    qref = np.take_along_axis(Q, idx_gpu, axis=1)
+    scale = np.maximum(1.0, qinf)[:, None]
+    err = np.abs(val_gpu - qref)
+    okv = err <= RTOL * np.abs(qref) + ATOL * scale
+    assert okv.all(), "%s: %d coefficient value(s) outside tolerance, max err %.3e (chunk %d)" % (
+        what, (~okv).sum(), err.max(), int(np.argmax(err.max(axis=1))))
+    report["max_val_err"] = max(report.get("max_val_err", 0.0), float(err.max()))
+    report["max_val_err_unscaled_atol_viol"] = report.get("max_val_err_unscaled_atol_viol", 0) + int(
+        (err > RTOL * np.abs(qref) + ATOL).sum())
+
+    # residual momentum: oracle continued from the GPU's index set where the sets differ
+    m_ref = ref["m_new"]
+    if len(diff):
+        forced = orc.compress_chunks(g[diff], m_before[diff], s, rows, k, beta, forced_idx=idx_gpu[diff].astype(np.int32))
+        m_ref = m_ref.copy()
+        m_ref[diff] = forced["m_new"]
+    # the abs tolerance is scaled by the chunk's pre-subtraction magnitude (the fp32 rounding of
+    # beta*m+g and of the reconstruction both scale with it)
+    binf = np.maximum(1.0, np.maximum(np.max(np.abs(beta * m_before + g), axis=1), np.max(np.abs(m_ref), axis=1)))[:, None]
+    errm = np.abs(m_after - m_ref)
+    okm = errm <= RTOL * np.abs(m_ref) + ATOL * binf
+    assert okm.all(), "%s: %d residual-momentum value(s) outside tolerance, max err %.3e (chunk %d)" % (
+        what, (~okm).sum(), errm.max(), int(np.argmax(errm.max(axis=1))))
+    report["max_m_err"] = max(report.get("max_m_err", 0.0), float(errm.max()))
+    return ref
+
+
+def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Report, what=""):
+    """recs_gpu [W, n, k_eff] GPU-written records; x_* float64 [n, M]."""
+    ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd)
+    R = ref["R"]
+    rinf = np.maximum(1.0, np.max(np.abs(R), axis=1, keepdims=True))
+    exempt = np.abs(R) < SIGN_EXEMPT * rinf
+    x_ref = ref["x_new"]
+    tol = RTOL * np.abs(x_ref) + ATOL * np.maximum(1.0, np.max(np.abs(x_ref), axis=1, keepdims=True))
+    ok = np.abs(x_after - x_ref) <= tol
+    # where the reconstructed momentum is within rounding of zero any of the three signs is legal
+    if (~ok & exempt).any():
+        alt = np.zeros_like(ok)
+        for sg in (-1.0, 0.0, 1.0):
+            alt |= np.abs(x_after - (x_before - lr * (sg + wd * x_before))) <= tol
+        ok = ok | (exempt & alt)
+    assert ok.all(), "%s: %d parameter(s) outside tolerance (sign or value), first chunk %d" % (
+        what, (~ok).sum(), int(np.argmax((~ok).any(axis=1))))
+    report.add("decode_chunks", x_before.shape[0])
+    report.add("sign_exempt", exempt.sum())
+    # sign bit-exactness outside the exemption, recovered from the update itself
+    sg_gpu = np.rint((x_before * (1.0 - lr * wd) - x_after) / lr)
+    mism = (sg_gpu != np.sign(R)) & ~exempt
+    assert not mism.any(), what + ": sign mismatch outside the exemption band"
+    return ref
+
+
+class Runner:
+    """Drives a workload through the C ABI and checks sampled (or all) chunks every step."""
+
+    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0):
+        import paper_2411_19870_b200 as demo
+        from paper_2411_19870_b200 import inputs
+
+        self.wl, self.device = wl, torch.device(device)
+        self.demo = demo
+        gd = demo.DEMO_BF16 if wl.grad_dtype == torch.bfloat16 else demo.DEMO_F32
+        self.tr = demo.DemoTransform(wl.shapes, chunk=wl.chunk, topk=wl.topk, beta=wl.beta, lr=wl.lr,
+                                     weight_decay=wl.weight_decay, num_workers=wl.num_workers, grad_dtype=gd,
+                                     device=self.device.index or 0)
+        if path is not None:
+            self.tr.set_path(path)
+        self.params = inputs.make_params(wl, self.device)
+        self.mom = [inputs.make_momentum(wl, self.device) for _ in range(wl.num_workers)]
+        self.streams = [inputs.GradStream(wl, w, self.device) for w in range(wl.num_workers)]
+        self.payloads = [torch.zeros(self.tr.payload_bytes, dtype=torch.uint8, device=self.device)
+                         for _ in range(wl.num_workers)]
+        self.layout = [self.tr.payload_layout(t) for t in range(len(wl.shapes))]
+        self.ids = [sample_chunk_ids(self.layout[t][1], max_chunks, seed + t) for t in range(len(wl.shapes))]
+        self.report = Report()
+        # fp32 copies of the scalars, as the library sees them
+        self.beta = float(np.float32(wl.beta))
+        self.lr = float(np.float32(wl.lr))
+        self.wd = float(np.float32(wl.weight_decay))
+
+    def step(self, check=True, grads=None):
+        wl, s = self.wl, self.wl.chunk
+        T = len(wl.shapes)
+        for w in range(wl.num_workers):
+            g = grads[w] if grads is not None else self.streams[w].next()
+            if check:
+                before = [gather_tiles(self.mom[w][t], s, self.ids[t]) for t in range(T)]
+            self.tr.compress(w, g, self.mom[w], self.payloads[w])
+            if check:
+                for t in range(T):
+                    rows = s if len(wl.shapes[t]) == 2 else 1
+                    first, _, k_eff = self.layout[t]
+                    check_compress_chunks(
+                        gather_tiles(g[t], s, self.ids[t]), before[t], gather_tiles(self.mom[w][t], s, self.ids[t]),
+                        gather_records(self.payloads[w], first, k_eff, self.ids[t]), s, rows, wl.topk, self.beta,
+                        self.report, what="compress w%d t%d" % (w, t))
+        if check:
+            xb = [gather_tiles(self.params[t], s, self.ids[t]) for t in range(T)]
+        self.tr.decode_apply(self.payloads, self.params)
+        if check:
+            for t in range(T):
+                rows = s if len(wl.shapes[t]) == 2 else 1
+                first, _, k_eff = self.layout[t]
+                recs = np.stack([gather_records(self.payloads[w], first, k_eff, self.ids[t])
+                                 for w in range(wl.num_workers)])
+                check_decode_chunks(recs, xb[t], gather_tiles(self.params[t], s, self.ids[t]), s, rows, self.lr,
+                                    self.wd, self.report, what="decode t%d" % t)
+        st = self.tr.device_status()
+        assert st == 0, "device status %d (%s)" % (st, self.demo.demo_status_string(st))
+
+    def close(self):
+        self.tr.close()
