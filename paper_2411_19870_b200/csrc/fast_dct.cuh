@@ -1,0 +1,186 @@
+// Register-resident fast DCT-II / DCT-III of compile-time length N (power of two), fully unrolled,
+// every twiddle an immediate.  Used for the chunk DCT of the paper (Section 2.1: the projection
+// matrices are the fixed orthonormal DCT basis), where it replaces the dense s x s contraction:
+// about 9 flop per element and pass instead of 2s.
+//
+// Factorisation (all steps are butterflies or plane rotations, so rounding errors do not grow
+// beyond O(log N) ulps of the data scale -- no division by small cosines, no running recurrences):
+//   DCT-II_N :  u[n] = x[n] + x[N-1-n],  v[n] = x[n] - x[N-1-n]            (n < N/2)
+//               X[2j] = DCT-II_{N/2}(u)[j],   X[2j+1] = DCT-IV_{N/2}(v)[j]
+//   DCT-IV_N :  with th_n = (2n+1) pi / (4N), H = N/2, for n < H
+//               a[n] =          v[n] cos th_n + v[N-1-n] sin th_n
+//               b[n] = (-1)^n (-v[n] sin th_n + v[N-1-n] cos th_n)
+//               A = DCT-II_H(a),  Bt = DCT-II_H(b)
+//               V[0] = A[0],  V[2p-1] = A[p] - Bt[H-p],  V[2p] = A[p] + Bt[H-p]  (0 < p < H),
+//               V[N-1] = -Bt[0]
+//   DCT-III_N (transpose of DCT-II_N; DCT-IV is symmetric so it is its own transpose):
+//               e = DCT-III_{N/2}(X[even]),  o = DCT-IV_{N/2}(X[odd]),
+//               x[n] = e[n] + o[n],  x[N-1-n] = e[n] - o[n]
+// Transforms here are un-normalised except for one scale SC applied to every output whose index
+// is not 0 (folded into the rotation constants, so it is free); the caller scales the DC term.
+// With SC = sqrt(2/N) and DC * sqrt(1/N) this is the orthonormal DCT-II (and its inverse).
+#pragma once
+
+#include <type_traits>
+
+#if defined(__CUDACC__)
+#define FDCT_HD __host__ __device__ __forceinline__
+#else
+#define FDCT_HD inline
+#endif
+
+namespace fdct {
+
+constexpr double kPi = 3.141592653589793238462643383279502884;
+
+constexpr double c_sqrt(double x)
+{
+    double r = x > 1.0 ? x : 1.0;
+    for (int i = 0; i < 200; ++i) r = 0.5 * (r + x / r);
+    return r;
+}
+// Taylor series; |x| <= pi/2 in every use below, where 16 terms reach double precision.
+constexpr double c_sin(double x)
+{
+    double term = x, sum = x;
+    for (int i = 1; i < 18; ++i) {
+        term *= -x * x / ((2.0 * i) * (2.0 * i + 1.0));
+        sum += term;
+    }
+    return sum;
+}
+constexpr double c_cos(double x)
+{
+    double term = 1.0, sum = 1.0;
+    for (int i = 1; i < 18; ++i) {
+        term *= -x * x / ((2.0 * i - 1.0) * (2.0 * i));
+        sum += term;
+    }
+    return sum;
+}
+
+struct ScaleOne {
+    static constexpr double value = 1.0;
+};
+template <int N0>
+struct ScaleOrtho {  // sqrt(2/N0)
+    static constexpr double value = c_sqrt(2.0 / N0);
+};
+template <int N0>
+constexpr float dc_scale() { return (float)c_sqrt(1.0 / N0); }
+
+template <int I, int N, class F>
+FDCT_HD void static_for(F &&f)
+{
+    if constexpr (I < N) {
+        f(std::integral_constant<int, I>{});
+        static_for<I + 1, N>(f);
+    }
+}
+
+template <int N, class SC>
+FDCT_HD void dct4(const float (&v)[N], float (&V)[N]);
+
+// out[k] = w_k * sum_n x[n] cos(pi (2n+1) k / (2N)),  w_0 = 1, w_k = SC
+template <int N, class SC>
+FDCT_HD void dct2(const float (&x)[N], float (&X)[N])
+{
+    if constexpr (N == 1) {
+        X[0] = x[0];
+    } else {
+        constexpr int H = N / 2;
+        float u[H], v[H], E[H], O[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            u[n] = x[n] + x[N - 1 - n];
+            v[n] = x[n] - x[N - 1 - n];
+        });
+        dct2<H, SC>(u, E);
+        dct4<H, SC>(v, O);
+        static_for<0, H>([&](auto i) {
+            constexpr int j = decltype(i)::value;
+            X[2 * j] = E[j];
+            X[2 * j + 1] = O[j];
+        });
+    }
+}
+
+// V[j] = SC * sum_n v[n] cos(pi (2n+1)(2j+1) / (4N))
+template <int N, class SC>
+FDCT_HD void dct4(const float (&v)[N], float (&V)[N])
+{
+    if constexpr (N == 1) {
+        constexpr float c = (float)(SC::value * c_cos(kPi / 4.0));
+        V[0] = v[0] * c;
+    } else {
+        constexpr int H = N / 2;
+        float a[H], b[H], A[H], Bt[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            constexpr double th = (2.0 * n + 1.0) * kPi / (4.0 * N);
+            constexpr double sg = (n % 2 == 0) ? 1.0 : -1.0;
+            constexpr float c = (float)(SC::value * c_cos(th));
+            constexpr float s = (float)(SC::value * c_sin(th));
+            constexpr float cb = (float)(SC::value * sg * c_cos(th));
+            constexpr float sb = (float)(SC::value * sg * c_sin(th));
+            const float lo = v[n], hi = v[N - 1 - n];
+            a[n] = fmaf(hi, s, lo * c);
+            b[n] = fmaf(hi, cb, -(lo * sb));
+        });
+        dct2<H, ScaleOne>(a, A);
+        dct2<H, ScaleOne>(b, Bt);
+        V[0] = A[0];
+        V[N - 1] = -Bt[0];
+        static_for<1, H>([&](auto i) {
+            constexpr int p = decltype(i)::value;
+            V[2 * p - 1] = A[p] - Bt[H - p];
+            V[2 * p] = A[p] + Bt[H - p];
+        });
+    }
+}
+
+// x[n] = sum_k w_k X[k] cos(pi (2n+1) k / (2N)),  w_0 = 1, w_k = SC   (transpose of dct2)
+template <int N, class SC>
+FDCT_HD void dct3(const float (&X)[N], float (&x)[N])
+{
+    if constexpr (N == 1) {
+        x[0] = X[0];
+    } else {
+        constexpr int H = N / 2;
+        float Xe[H], Xo[H], e[H], o[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int j = decltype(i)::value;
+            Xe[j] = X[2 * j];
+            Xo[j] = X[2 * j + 1];
+        });
+        dct3<H, SC>(Xe, e);
+        dct4<H, SC>(Xo, o);
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            x[n] = e[n] + o[n];
+            x[N - 1 - n] = e[n] - o[n];
+        });
+    }
+}
+
+// Orthonormal DCT-II of x (in place): X[k] = a_k sum_n x[n] cos(pi (2n+1) k / (2N)).
+template <int N>
+FDCT_HD void dct2_ortho(float (&x)[N])
+{
+    float X[N];
+    dct2<N, ScaleOrtho<N>>(x, X);
+    X[0] *= dc_scale<N>();
+    static_for<0, N>([&](auto i) { x[decltype(i)::value] = X[decltype(i)::value]; });
+}
+
+// Inverse of dct2_ortho (orthonormal DCT-III), in place.
+template <int N>
+FDCT_HD void dct3_ortho(float (&X)[N])
+{
+    float x[N];
+    X[0] *= dc_scale<N>();
+    dct3<N, ScaleOrtho<N>>(X, x);
+    static_for<0, N>([&](auto i) { X[decltype(i)::value] = x[decltype(i)::value]; });
+}
+
+}  // namespace fdct
