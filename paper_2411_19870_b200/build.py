@@ -50,7 +50,7 @@ def build_library(force: bool = False, verbose: bool = False, ptxas_info: bool =
         objs.append(obj)
         stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time)
         if stale:
-            cmd = [nvcc] + NVCC_FLAGS + ["-I", INCLUDE, "-c", src, "-o", obj]
+            cmd = [nvcc] + NVCC_FLAGS + os.environ.get("DEMO_NVCC_EXTRA", "").split() + ["-I", INCLUDE, "-c", src, "-o", obj]
             if ptxas_info:
                 cmd += ["-Xptxas", "-v"]
             jobs.append(cmd)

@@ -34,6 +34,10 @@ struct DemoCompressArgs {
     float beta;
     int grad_bf16;  // 1: gradients are bf16, 0: fp32
     int *status;    // device status word (sticky)
+    // Optional TMA tensor maps (128-byte CUtensorMap objects in device memory, indexed like the
+    // pointer arrays; box = one s x s tile).  NULL: tiles are staged row by row with 1-D bulk copies.
+    const void *tmap_m;
+    const void *tmap_g;
 };
 
 struct DemoDecodeArgs {
@@ -47,6 +51,7 @@ struct DemoDecodeArgs {
     float lr;
     float wd;
     int *status;
+    const void *tmap_x;  // optional tensor maps of the parameter tensors (see DemoCompressArgs)
 };
 
 // Launchers (defined in the kernel translation units).  `s` is the chunk size, `two_d` selects

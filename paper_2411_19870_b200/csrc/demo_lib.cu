@@ -1,5 +1,8 @@
 // Host side of the C ABI declared in include/demo.h: context, planner (chunk tables of the blocking
 // operator, payload offsets, DCT basis), pointer-table caching and kernel dispatch.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include <cmath>
 #include <cstring>
 #include <new>
@@ -38,6 +41,13 @@ struct demo_ctx {
     std::vector<const DemoRecord *> h_p;
     std::vector<char> g_valid, m_valid;  // per worker
     bool x_valid = false, p_valid = false;
+
+    // TMA tensor maps for the fast kernels (2-D tensors; box = one s x s tile), rebuilt whenever
+    // the caller's pointers change.  NULL when the driver entry point is unavailable.
+    PFN_cuTensorMapEncodeTiled encode = nullptr;
+    CUtensorMap *d_tm_g = nullptr, *d_tm_m = nullptr;  // [W][T]
+    CUtensorMap *d_tm_x = nullptr;                     // [T]
+    std::vector<CUtensorMap> h_tm;                     // staging, [T]
 };
 
 namespace {
@@ -61,13 +71,41 @@ struct DeviceGuard {
 // Upload `n` pointers to dev[0..n) if they differ from the mirror.  The mirror is pageable host
 // memory: cudaMemcpyAsync stages it before returning, so it may be overwritten by the next call.
 template <typename T>
-cudaError_t sync_table(T *dev, T *mirror, const T *now, int n, bool *valid, cudaStream_t stream)
+cudaError_t sync_table(T *dev, T *mirror, const T *now, int n, bool *valid, cudaStream_t stream,
+                       bool *changed = nullptr)
 {
+    if (changed) *changed = false;
     if (*valid && std::memcmp(mirror, now, sizeof(T) * (size_t)n) == 0) return cudaSuccess;
+    if (changed) *changed = true;
     std::memcpy(mirror, now, sizeof(T) * (size_t)n);
     cudaError_t err = cudaMemcpyAsync(dev, mirror, sizeof(T) * (size_t)n, cudaMemcpyHostToDevice, stream);
     *valid = (err == cudaSuccess);
     return err;
+}
+
+// Encode one tensor map per 2-D tensor (box = s x s tile of `elem`-byte elements) for the given base
+// pointers and upload them to dev[0..T).  Returns false if the driver rejects a descriptor.
+template <typename P>
+bool upload_tensor_maps(demo_ctx *c, CUtensorMap *dev, const P *ptrs, bool bf16, cudaStream_t stream)
+{
+    const int T = c->n_tensors, s = c->cfg.chunk;
+    std::memset(c->h_tm.data(), 0, sizeof(CUtensorMap) * (size_t)T);
+    for (int t = 0; t < T; ++t) {
+        const demo_tensor_desc &d = c->descs[t];
+        if (d.ndim != 2) continue;
+        const cuuint64_t elem = bf16 ? 2 : 4;
+        const cuuint64_t gdim[2] = {(cuuint64_t)d.shape[1], (cuuint64_t)d.shape[0]};
+        const cuuint64_t gstride[1] = {(cuuint64_t)d.shape[1] * elem};
+        const cuuint32_t box[2] = {(cuuint32_t)s, (cuuint32_t)s};
+        const cuuint32_t estr[2] = {1, 1};
+        const CUresult r = c->encode(&c->h_tm[t], bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                     2, const_cast<void *>(static_cast<const void *>(ptrs[t])), gdim, gstride, box, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return false;
+    }
+    return cudaMemcpyAsync(dev, c->h_tm.data(), sizeof(CUtensorMap) * (size_t)T, cudaMemcpyHostToDevice, stream) ==
+           cudaSuccess;
 }
 
 void release(demo_ctx *c)
@@ -81,6 +119,9 @@ void release(demo_ctx *c)
     cudaFree((void *)c->d_m);
     cudaFree((void *)c->d_x);
     cudaFree((void *)c->d_p);
+    cudaFree(c->d_tm_g);
+    cudaFree(c->d_tm_m);
+    cudaFree(c->d_tm_x);
     delete c;
 }
 
@@ -209,6 +250,25 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
     ok = ok && cudaMalloc((void **)&c->d_m, W * T * sizeof(void *)) == cudaSuccess;
     ok = ok && cudaMalloc((void **)&c->d_x, T * sizeof(void *)) == cudaSuccess;
     ok = ok && cudaMalloc((void **)&c->d_p, W * sizeof(void *)) == cudaSuccess;
+    if (ok && c->n2d && demo_fast_supported(s)) {
+        // TMA descriptors need the driver's encoder; without it the fast kernels stage row by row
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess && fn) {
+            c->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+            try {
+                c->h_tm.resize(T);
+            } catch (const std::bad_alloc &) {
+                ok = false;
+            }
+            ok = ok && cudaMalloc(&c->d_tm_g, W * T * sizeof(CUtensorMap)) == cudaSuccess;
+            ok = ok && cudaMalloc(&c->d_tm_m, W * T * sizeof(CUtensorMap)) == cudaSuccess;
+            ok = ok && cudaMalloc(&c->d_tm_x, T * sizeof(CUtensorMap)) == cudaSuccess;
+        } else {
+            cudaGetLastError();
+        }
+    }
     if (!ok) {
         cudaGetLastError();
         release(c);
@@ -258,12 +318,21 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
 
     const size_t row = (size_t)worker * (size_t)T;
     bool gv = ctx->g_valid[worker] != 0, mv = ctx->m_valid[worker] != 0;
-    cudaError_t err = sync_table<const void *>(ctx->d_g + row, ctx->h_g.data() + row, grads, T, &gv, stream);
+    bool g_changed = false, m_changed = false;
+    cudaError_t err =
+        sync_table<const void *>(ctx->d_g + row, ctx->h_g.data() + row, grads, T, &gv, stream, &g_changed);
     ctx->g_valid[worker] = gv;
     if (err == cudaSuccess) {
         err = sync_table<float *>(ctx->d_m + row, ctx->h_m.data() + row, const_cast<float *const *>(momentum), T, &mv,
-                                  stream);
+                                  stream, &m_changed);
         ctx->m_valid[worker] = mv;
+    }
+    if (err == cudaSuccess && ctx->encode) {
+        const bool bf16 = ctx->cfg.grad_dtype == DEMO_BF16;
+        if (g_changed && !upload_tensor_maps(ctx, ctx->d_tm_g + row, grads, bf16, stream)) err = cudaErrorInvalidValue;
+        if (err == cudaSuccess && m_changed && !upload_tensor_maps(ctx, ctx->d_tm_m + row, momentum, false, stream))
+            err = cudaErrorInvalidValue;
+        if (err != cudaSuccess) ctx->g_valid[worker] = ctx->m_valid[worker] = 0;
     }
     if (err != cudaSuccess) {
         cudaGetLastError();
@@ -278,6 +347,8 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
     a.beta = ctx->cfg.beta;
     a.grad_bf16 = ctx->cfg.grad_dtype == DEMO_BF16;
     a.status = ctx->d_status;
+    a.tmap_m = ctx->encode ? ctx->d_tm_m + row : nullptr;
+    a.tmap_g = ctx->encode ? ctx->d_tm_g + row : nullptr;
     const int s = ctx->cfg.chunk;
     if (ctx->n2d) {
         a.entries = ctx->d_entries2d;
@@ -320,9 +391,14 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     cudaError_t err = sync_table<const DemoRecord *>(ctx->d_p, ctx->h_p.data(),
                                                      reinterpret_cast<const DemoRecord *const *>(payloads), W,
                                                      &ctx->p_valid, stream);
+    bool x_changed = false;
     if (err == cudaSuccess)
         err = sync_table<float *>(ctx->d_x, ctx->h_x.data(), const_cast<float *const *>(params), T, &ctx->x_valid,
-                                  stream);
+                                  stream, &x_changed);
+    if (err == cudaSuccess && ctx->encode && x_changed && !upload_tensor_maps(ctx, ctx->d_tm_x, params, false, stream)) {
+        err = cudaErrorInvalidValue;
+        ctx->x_valid = false;
+    }
     if (err != cudaSuccess) {
         cudaGetLastError();
         return DEMO_ERR_CUDA;
@@ -336,6 +412,7 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     a.lr = ctx->cfg.lr;
     a.wd = ctx->cfg.weight_decay;
     a.status = ctx->d_status;
+    a.tmap_x = ctx->encode ? ctx->d_tm_x : nullptr;
     const int s = ctx->cfg.chunk;
     if (ctx->n2d) {
         a.entries = ctx->d_entries2d;

@@ -67,8 +67,31 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, unsigned
                  : "memory");
 }
 
+// 2-D tiled TMA load of one box (coordinates in elements: x along the row, y the row index).
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(tmap), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+// Pull one box into L2 ahead of its use.
+__device__ __forceinline__ void tma_prefetch_2d(const void *tmap, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
+}
+constexpr int TMAP_BYTES = 128;  // sizeof(CUtensorMap)
+
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+// max of three (one instruction on sm_100)
+__device__ __forceinline__ float max3f(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float max3abs(float a, float b, float c) { return max3f(fabsf(a), fabsf(b), fabsf(c)); }
 __device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
 template <int S>
@@ -167,29 +190,35 @@ __device__ __forceinline__ unsigned warp_inclusive_scan(unsigned v, int lane)
     return v;
 }
 
-template <int S, typename GT>
-__global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
+#ifndef DEMO_FAST_MIN_BLOCKS
+#define DEMO_FAST_MIN_BLOCKS 8
+#endif
+
+template <int S, typename GT, bool TMAP>
+__global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(DemoCompressArgs a)
 {
     using C = Cfg<S>;
     constexpr int XS = C::XS, NW = C::NW, LOG2S = C::LOG2S;
     constexpr unsigned TILE_BYTES = S * S * sizeof(float) + S * S * sizeof(GT);
+    constexpr int CAPW = CAP / NW;        // candidate capacity of one warp's list
+    constexpr int CAPWP = CAPW + 4;       // list stride (padding for 128-bit key loads)
+    constexpr int ITER = CAPW / 32;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float *Bt = reinterpret_cast<float *>(smem_raw);             // [S*S]   m tile, then B
     float *X = Bt + S * S;                                       // [S*XS]  g staging / transpose / Q / T
-    float *costab = X + S * XS;                                  // [4*S]   cos(pi t / (2S))
-    float *tmax = costab + 4 * S;                                // [S]
+    float *tmax = X + S * XS;                                    // [S]
     int *cand_idx = reinterpret_cast<int *>(tmax + S);           // [CAP]
-    float *cand_val = reinterpret_cast<float *>(cand_idx + CAP); // [CAP]
+    float *cand_val = reinterpret_cast<float *>(cand_idx + CAP + 8); // [CAP + 8]
+    unsigned *cand_key = reinterpret_cast<unsigned *>(cand_val + CAP + 8);  // [CAP + 8]
     unsigned *hist = reinterpret_cast<unsigned *>(cand_idx);     // [256] aliases the candidate arrays
-    DemoRecord *recs = reinterpret_cast<DemoRecord *>(cand_val + CAP);  // [64]
-    unsigned *misc = reinterpret_cast<unsigned *>(recs + 64);    // [16]
+    int4 *recs4 = reinterpret_cast<int4 *>(cand_key + CAP + 8);  // [64] kept records, pre-decoded
+    unsigned *misc = reinterpret_cast<unsigned *>(recs4 + 64);   // [16]
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(misc + 16);
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const uint32_t bar = smem_u32(bar_mem);
 
-    for (int i = t; i < 4 * S; i += S) costab[i] = cospif((float)i / (float)(2 * S));
     if (t == 0) {
         mbar_init(bar, 1);
         fence_proxy_async();  // make the initialised barrier visible to the async proxy
@@ -203,7 +232,13 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
     int cached_tensor = -1;
     unsigned phase = 0;
 
-    auto issue_loads = [&](long long c) {
+    // Locate the tile of chunk c (advances the tensor cursor; chunk ids only grow): row t of the tile
+    // for the row-by-row path, tensor map and box coordinates for the TMA path.
+    const float *m_src = nullptr;
+    const GT *g_src = nullptr;
+    const char *tm_m = nullptr, *tm_g = nullptr;
+    int ld_x = 0, ld_y = 0;
+    auto locate = [&](long long c) {
         cur.seek(a.entries, a.n_entries, c);
         if (cur.te.tensor != cached_tensor) {
             cached_tensor = cur.te.tensor;
@@ -213,15 +248,37 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
         const long long lc = c - cur.te.chunk_begin;
         const long long k0 = lc / cur.te.c1;
         const int k1 = (int)(lc - k0 * cur.te.c1);
-        const size_t off = ((size_t)k0 * S + t) * (size_t)cur.te.n1 + (size_t)k1 * S;  // row t of the tile
-        if (t == 0) mbar_expect_tx(bar, TILE_BYTES);
-        fence_proxy_async();
-        bulk_g2s(smem_u32(Bt + t * S), m_ptr + off, S * sizeof(float), bar);
-        bulk_g2s(smem_u32(reinterpret_cast<GT *>(X) + t * S), g_ptr + off, S * sizeof(GT), bar);
+        if (TMAP) {
+            tm_m = static_cast<const char *>(a.tmap_m) + (size_t)cached_tensor * TMAP_BYTES;
+            tm_g = static_cast<const char *>(a.tmap_g) + (size_t)cached_tensor * TMAP_BYTES;
+            ld_x = k1 * S;
+            ld_y = (int)k0 * S;
+        } else {
+            const size_t off = ((size_t)k0 * S + t) * (size_t)cur.te.n1 + (size_t)k1 * S;
+            m_src = m_ptr + off;
+            g_src = g_ptr + off;
+        }
+    };
+    // Called right after a CTA-wide barrier that follows a fence.proxy.async of every thread.
+    auto issue_loads = [&]() {
+        if (TMAP) {
+            if (t == 0) {
+                mbar_expect_tx(bar, TILE_BYTES);
+                tma_load_2d(smem_u32(Bt), tm_m, ld_x, ld_y, bar);
+                tma_load_2d(smem_u32(X), tm_g, ld_x, ld_y, bar);
+            }
+        } else {
+            if (t == 0) mbar_expect_tx(bar, TILE_BYTES);
+            bulk_g2s(smem_u32(Bt + t * S), m_src, S * sizeof(float), bar);
+            bulk_g2s(smem_u32(reinterpret_cast<GT *>(X) + t * S), g_src, S * sizeof(GT), bar);
+        }
     };
 
     long long c = blockIdx.x;
-    if (c < a.n_chunks) issue_loads(c);
+    if (c < a.n_chunks) {
+        locate(c);
+        issue_loads();
+    }
 
     for (; c < a.n_chunks; c += gridDim.x) {
         // the cursor points at chunk c (issue_loads(c) ran last)
@@ -240,6 +297,15 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
             if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
             mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
             return;
+        }
+        // start pulling the next chunk's rows into L2 while this chunk is processed
+        const long long nc = c + gridDim.x;
+        if (nc < a.n_chunks) {
+            locate(nc);
+            if (TMAP && t == 0) {
+                tma_prefetch_2d(tm_m, ld_x, ld_y);
+                tma_prefetch_2d(tm_g, ld_x, ld_y);
+            }
         }
 
         // ---- momentum update on column t, first DCT pass down the column -------------------------
@@ -274,68 +340,64 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
 
         // ---- top-k ------------------------------------------------------------------------------
         bool use_fallback = (k_eff > S);
-        unsigned n_c = 0, off = 0;
-        unsigned long long mask = 0ull;
+        unsigned n_cw = 0, off = 0;
+        unsigned mlo = 0u, mhi = 0u;
         if (!use_fallback) {
+            // per-thread maximum magnitude: independent chains of 16 with 3-input max
             float tm = 0.f;
 #pragma unroll
-            for (int v = 0; v < S; ++v) tm = fmaxf(tm, fabsf(q[v]));
-            // bitonic sort (descending) of the 32 per-thread maxima of this warp
-            float sv = tm;
+            for (int ch = 0; ch < S / 16; ++ch) {
+                const int b0 = 16 * ch;
+                float c = max3abs(q[b0], q[b0 + 1], q[b0 + 2]);
 #pragma unroll
-            for (int k2 = 2; k2 <= 32; k2 <<= 1) {
+                for (int j = 3; j + 1 < 16; j += 2) c = max3f(c, fabsf(q[b0 + j]), fabsf(q[b0 + j + 1]));
+                tm = max3f(tm, c, fabsf(q[b0 + 15]));
+            }
+            // L = the k_eff-th largest of the S per-thread maxima = the smallest maximum that has
+            // fewer than k_eff strictly larger ones.  Every warp ranks all S maxima (its own and the
+            // partner warp's) so that no second exchange is needed.
+            const unsigned tkey = __float_as_uint(tm);
+            unsigned *tk = reinterpret_cast<unsigned *>(tmax);
+            tk[t] = tkey;
+            __syncthreads();
+            unsigned lmin;
+            {
+                const unsigned okey = (NW > 1) ? tk[t ^ 32] : tkey;
+                unsigned gtc = 0, gto = 0;
+                const uint4 *t4 = reinterpret_cast<const uint4 *>(tk);
 #pragma unroll
-                for (int j = k2 >> 1; j > 0; j >>= 1) {
-                    const float other = __shfl_xor_sync(0xffffffffu, sv, j);
-                    const bool keep_max = ((lane & j) == 0) == ((lane & k2) == 0);
-                    sv = keep_max ? fmaxf(sv, other) : fminf(sv, other);
+                for (int j4 = 0; j4 < S / 4; ++j4) {
+                    const uint4 o = t4[j4];
+                    gtc += (o.x > tkey) + (o.y > tkey) + (o.z > tkey) + (o.w > tkey);
+                    if (NW > 1) gto += (o.x > okey) + (o.y > okey) + (o.z > okey) + (o.w > okey);
                 }
+                unsigned cnd = (gtc < (unsigned)k_eff) ? tkey : 0xffffffffu;
+                if (NW > 1) cnd = min(cnd, (gto < (unsigned)k_eff) ? okey : 0xffffffffu);
+                lmin = __reduce_min_sync(0xffffffffu, cnd);
             }
-            float L;
-            if (NW == 1) {
-                L = __shfl_sync(0xffffffffu, sv, k_eff - 1);
-            } else {
-                tmax[t] = sv;
-                __syncthreads();
-                // rank of this element in the union of the two descending lists (strict order:
-                // equal values of warp 0 come first)
-                const float *other = tmax + (warp ^ 1) * 32;
-                int lo = 0, hi = 32;
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    const float o = other[mid];
-                    const bool before = (warp == 0) ? (o > sv) : (o >= sv);
-                    if (before)
-                        lo = mid + 1;
-                    else
-                        hi = mid;
-                }
-                if (lane + lo == k_eff - 1) reinterpret_cast<float *>(misc)[8] = sv;
-                __syncthreads();
-                L = reinterpret_cast<float *>(misc)[8];
-            }
-            // candidates: coefficients with magnitude >= L (at least k_eff of them exist)
-            unsigned mlo = 0u, mhi = 0u;
+            const float L = __uint_as_float(lmin);
+            // candidates: coefficients with magnitude >= L (at least k_eff of them exist).
+            // |q| >= L  <=>  |q| > Lm with Lm the float just below L; the sign bit of Lm - |q| is
+            // shifted into a bit mask (independent chains of 16).
+            const float Lm = (L > 0.f) ? __uint_as_float(lmin - 1u) : -1.f;
+            unsigned mc[S / 16];
 #pragma unroll
-            for (int v = 0; v < S; ++v) {
-                const bool p = fabsf(q[v]) >= L;
-                if (v < 32)
-                    mlo |= p ? (1u << v) : 0u;
-                else
-                    mhi |= p ? (1u << (v - 32)) : 0u;
+            for (int ch = 0; ch < S / 16; ++ch) {
+                unsigned mm = 0u;
+#pragma unroll
+                for (int j = 15; j >= 0; --j)
+                    mm = __funnelshift_l(__float_as_uint(Lm - fabsf(q[16 * ch + j])), mm, 1);
+                mc[ch] = mm;
             }
-            mask = ((unsigned long long)mhi << 32) | mlo;
+            mlo = mc[0] | (mc[1] << 16);
+            if (S == 64) mhi = mc[S / 16 - 2] | (mc[S / 16 - 1] << 16);
+            // each warp compacts its candidates into its own list (rows of warp 0 precede rows of
+            // warp 1, so the concatenation is in ascending index order)
             const unsigned cnt = __popc(mlo) + __popc(mhi);
             const unsigned inc = warp_inclusive_scan(cnt, lane);
-            if (lane == 31) misc[warp] = inc;
-            __syncthreads();
             off = inc - cnt;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                if (w < warp) off += misc[w];
-                n_c += misc[w];
-            }
-            use_fallback = (n_c > CAP);
+            n_cw = __shfl_sync(0xffffffffu, inc, 31);
+            if (lane == 0) misc[warp] = n_cw;
         }
         // stash the coefficients of row t (own row: no hazard with other threads)
         {
@@ -343,53 +405,104 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
 #pragma unroll
             for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(q[4 * v4], q[4 * v4 + 1], q[4 * v4 + 2], q[4 * v4 + 3]);
         }
-
         if (!use_fallback) {
-            unsigned o = off;
-            while (mask) {
-                const int v = __ffsll((long long)mask) - 1;
-                mask &= mask - 1ull;
-                cand_idx[o] = t * S + v;
-                cand_val[o] = X[t * XS + v];
-                ++o;
+            const unsigned lbase = warp * CAPWP;
+            if (n_cw <= CAPW) {
+                unsigned o = lbase + off;
+                unsigned long long mask = ((unsigned long long)mhi << 32) | mlo;
+                while (mask) {
+                    const int v = __ffsll((long long)mask) - 1;
+                    mask &= mask - 1ull;
+                    const float val = X[t * XS + v];
+                    cand_idx[o] = t * S + v;
+                    cand_val[o] = val;
+                    cand_key[o] = mag_key(val);
+                    ++o;
+                }
+                if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
             }
             __syncthreads();
-            // exact rank among the candidates: larger magnitude first, then lower index (the list
-            // is in ascending index order, so the list position stands for the index)
-            constexpr int ITER = CAP / S;
-            bool sel[ITER];
-            unsigned pre[ITER];
+            unsigned n_w[NW];
 #pragma unroll
-            for (int it = 0; it < ITER; ++it) {
-                const unsigned ci = it * S + t;
-                sel[it] = false;
-                if (ci < n_c) {
-                    const unsigned key = mag_key(cand_val[ci]);
-                    unsigned rank = 0;
-                    for (unsigned c2 = 0; c2 < n_c; ++c2) {
-                        const unsigned k2 = mag_key(cand_val[c2]);
-                        rank += (k2 > key) || (k2 == key && c2 < ci);
+            for (int w = 0; w < NW; ++w) {
+                n_w[w] = misc[w];
+                use_fallback = use_fallback || (n_w[w] > CAPW);
+            }
+            if (!use_fallback) {
+                // rank among all candidates by magnitude only.  If exactly k_eff candidates have
+                // fewer than k_eff larger ones, no tie straddles the threshold and that set is the
+                // answer; otherwise the count is redone with the index tie-break.
+                bool sel[ITER];
+                unsigned pre[ITER];
+#pragma unroll
+                for (int it = 0; it < ITER; ++it) {
+                    const unsigned li = it * 32 + lane;  // position in this warp's list
+                    sel[it] = false;
+                    if (it * 32 < (int)n_cw) {  // warp-uniform
+                        const unsigned key = (li < n_cw) ? cand_key[lbase + li] : 0xffffffffu;
+                        unsigned rank = 0;
+#pragma unroll
+                        for (int w = 0; w < NW; ++w) {
+                            const uint4 *keys4 = reinterpret_cast<const uint4 *>(cand_key + w * CAPWP);
+                            const unsigned n4 = (n_w[w] + 3u) >> 2;
+                            for (unsigned c4 = 0; c4 < n4; ++c4) {
+                                const uint4 k4 = keys4[c4];
+                                rank += (k4.x > key) + (k4.y > key) + (k4.z > key) + (k4.w > key);
+                            }
+                        }
+                        sel[it] = (li < n_cw) && rank < (unsigned)k_eff;
                     }
-                    sel[it] = rank < (unsigned)k_eff;
+                    const unsigned bal = __ballot_sync(0xffffffffu, sel[it]);
+                    pre[it] = __popc(bal & ((1u << lane) - 1u));
+                    if (lane == 0) misc[4 + warp * ITER + it] = __popc(bal);
                 }
-                const unsigned bal = __ballot_sync(0xffffffffu, sel[it]);
-                pre[it] = __popc(bal & ((1u << lane) - 1u));
-                if (lane == 0) misc[4 + it * NW + warp] = __popc(bal);
-            }
-            __syncthreads();
+                __syncthreads();
+                unsigned total = 0;
 #pragma unroll
-            for (int it = 0; it < ITER; ++it) {
-                if (sel[it]) {
-                    unsigned pos = pre[it];
-                    for (int g = 0; g < it * NW + warp; ++g) pos += misc[4 + g];
-                    DemoRecord r;
-                    r.idx = cand_idx[it * S + t];
-                    r.val = cand_val[it * S + t];
-                    rec[pos] = r;
-                    recs[pos] = r;  // k_eff <= S <= 64 on this path
+                for (int g = 0; g < ITER * NW; ++g) total += misc[4 + g];
+                if (total != (unsigned)k_eff) {  // block-uniform: equal magnitudes straddle the threshold
+                    __syncthreads();
+#pragma unroll
+                    for (int it = 0; it < ITER; ++it) {
+                        const unsigned li = it * 32 + lane;
+                        sel[it] = false;
+                        if (li < n_cw) {
+                            const unsigned key = cand_key[lbase + li];
+                            unsigned rank = 0;
+#pragma unroll
+                            for (int w = 0; w < NW; ++w)
+                                for (unsigned c2 = 0; c2 < n_w[w]; ++c2) {
+                                    const unsigned k2 = cand_key[w * CAPWP + c2];
+                                    const bool earlier = (w < warp) || (w == warp && c2 < li);
+                                    rank += (k2 > key) || (k2 == key && earlier);
+                                }
+                            sel[it] = rank < (unsigned)k_eff;
+                        }
+                        const unsigned bal = __ballot_sync(0xffffffffu, sel[it]);
+                        pre[it] = __popc(bal & ((1u << lane) - 1u));
+                        if (lane == 0) misc[4 + warp * ITER + it] = __popc(bal);
+                    }
+                    __syncthreads();
+                }
+#pragma unroll
+                for (int it = 0; it < ITER; ++it) {
+                    if (sel[it]) {
+                        unsigned pos = pre[it];
+                        for (int g = 0; g < warp * ITER + it; ++g) pos += misc[4 + g];
+                        DemoRecord r;
+                        r.idx = cand_idx[lbase + it * 32 + lane];
+                        r.val = cand_val[lbase + it * 32 + lane];
+                        rec[pos] = r;
+                        const int v = r.idx & (S - 1);  // k_eff <= S <= 64 on this path
+                        const int uo = (r.idx >> LOG2S) * XS;
+                        recs4[pos] = make_int4(uo, v * S, __float_as_int(r.val), 0);
+                        if ((int)pos == k_eff - 1)
+                            for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(uo, 0, 0, 0);
+                    }
                 }
             }
-        } else {
+        }
+        if (use_fallback) {
             __syncthreads();  // coefficient tile complete in X
             unsigned thr, need_eq;
             radix_select_tile<S>(X, k_eff, hist, misc, &thr, &need_eq);
@@ -430,7 +543,11 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
                     r.idx = t * S + v;
                     r.val = val;
                     rec[pos] = r;
-                    if (k_eff <= 64) recs[pos] = r;
+                    if (k_eff <= 64) {
+                        recs4[pos] = make_int4(t * XS, v * S, __float_as_int(val), 0);
+                        if ((int)pos == k_eff - 1)
+                            for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(t * XS, 0, 0, 0);
+                    }
                 }
             }
         }
@@ -444,22 +561,44 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
         }
         __syncthreads();
         {
-            constexpr float sc = (float)fdct::ScaleOrtho<S>::value, dc = fdct::dc_scale<S>();
-            const int tw = 2 * t + 1;
+            // T[u][t] = sum over kept (u, v) of val * C[v][t]; the basis is read through L1 (all CTAs
+            // of the SM share the same 4*S*S bytes), coalesced across the warp
+            const float *Ct = a.C + t;
             float acc = 0.f;
             int cur_u = -1;
-            for (int r = 0; r < k_eff; ++r) {
-                const DemoRecord rc = (k_eff <= 64) ? recs[r] : rec[r];
-                const int u = rc.idx >> LOG2S, v = rc.idx & (S - 1);
-                if (u != cur_u) {
-                    if (cur_u >= 0) X[cur_u * XS + t] = acc;
-                    acc = 0.f;
-                    cur_u = u;
+            if (k_eff <= 64) {
+                // the list is padded to a multiple of eight with zero-valued records of the last row;
+                // eight records and their cosines are fetched ahead of the dependent accumulation
+                cur_u = recs4[0].x;
+                for (int r0 = 0; r0 < k_eff; r0 += 8) {
+                    int4 rc[8];
+                    float cv[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) rc[j] = recs4[r0 + j];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) cv[j] = __ldg(Ct + rc[j].y);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const bool chg = rc[j].x != cur_u;
+                        if (chg) X[cur_u + t] = acc;
+                        acc = chg ? 0.f : acc;
+                        cur_u = rc[j].x;
+                        acc = fmaf(__int_as_float(rc[j].z), cv[j], acc);
+                    }
                 }
-                const float sv = rc.val * (v == 0 ? dc : sc);
-                acc = fmaf(sv, costab[(tw * v) & (4 * S - 1)], acc);  // T[u][t] += val * C[v][t]
+            } else {
+                for (int r = 0; r < k_eff; ++r) {
+                    const DemoRecord rc = rec[r];
+                    const int u = (rc.idx >> LOG2S) * XS, v = rc.idx & (S - 1);
+                    if (u != cur_u) {
+                        if (cur_u >= 0) X[cur_u + t] = acc;
+                        acc = 0.f;
+                        cur_u = u;
+                    }
+                    acc = fmaf(rc.val, __ldg(Ct + v * S), acc);
+                }
             }
-            if (cur_u >= 0) X[cur_u * XS + t] = acc;
+            if (cur_u >= 0) X[cur_u + t] = acc;
         }
         // column t of T was written by this thread only: no barrier needed before reading it back
         {
@@ -470,13 +609,13 @@ __global__ void __launch_bounds__(S) compress_fast_kernel(DemoCompressArgs a)
 #pragma unroll
             for (int i = 0; i < S; ++i) m[base + (size_t)i * te.n1 + t] = Bt[i * S + t] - r[i];
         }
-        __syncthreads();  // Bt and X are free again
-        const long long nc = c + gridDim.x;
-        if (nc < a.n_chunks) issue_loads(nc);
+        fence_proxy_async();  // order this thread's shared-memory accesses before the async-proxy writes
+        __syncthreads();      // Bt and X are free again
+        if (nc < a.n_chunks) issue_loads();
     }
 }
 
-template <int S>
+template <int S, bool TMAP>
 __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
 {
     using C = Cfg<S>;
@@ -516,10 +655,18 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + lc * (long long)k_eff;
 
-        // stage the x tile while the aggregate is built
-        if (t == 0) mbar_expect_tx(bar, S * S * sizeof(float));
-        fence_proxy_async();
-        bulk_g2s(smem_u32(Xt + t * S), x + base + (size_t)t * te.n1, S * sizeof(float), bar);
+        // stage the x tile while the aggregate is built (the previous iteration ended with a
+        // fence.proxy.async of every thread and a barrier)
+        if (TMAP) {
+            if (t == 0) {
+                mbar_expect_tx(bar, S * S * sizeof(float));
+                tma_load_2d(smem_u32(Xt), static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES, k1 * S,
+                            (int)k0 * S, bar);
+            }
+        } else {
+            if (t == 0) mbar_expect_tx(bar, S * S * sizeof(float));
+            bulk_g2s(smem_u32(Xt + t * S), x + base + (size_t)t * te.n1, S * sizeof(float), bar);
+        }
 
         {
             float4 *row = reinterpret_cast<float4 *>(St + t * XS);
@@ -527,17 +674,28 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
             for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         __syncthreads();
-        // S = sum over workers in worker order; a barrier per worker fixes the order of additions
-        for (int w = 0; w < a.W; ++w) {
-            const DemoRecord *rec = a.payloads[w] + rec_off;
-            for (int i = t; i < k_eff; i += S) {
-                const DemoRecord r = rec[i];
-                if ((unsigned)r.idx < (unsigned)M)
-                    St[(r.idx >> C::LOG2S) * XS + (r.idx & (S - 1))] += r.val;
-                else
-                    atomicMax(a.status, DEMO_DEV_PAYLOAD);
+        // S = sum over workers in worker order; a barrier per worker fixes the order of additions.
+        // Records are fetched eight workers ahead so that one memory latency covers eight workers.
+        for (int kb = 0; kb < k_eff; kb += S) {
+            const bool mine = kb + t < k_eff;
+            for (int w0 = 0; w0 < a.W; w0 += 8) {
+                DemoRecord r[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (mine && w0 + j < a.W) r[j] = a.payloads[w0 + j][rec_off + kb + t];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (w0 + j < a.W) {
+                        if (mine) {
+                            if ((unsigned)r[j].idx < (unsigned)M)
+                                St[(r[j].idx >> C::LOG2S) * XS + (r[j].idx & (S - 1))] += r[j].val;
+                            else
+                                atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                        }
+                        __syncthreads();
+                    }
+                }
             }
-            __syncthreads();
         }
         // inverse along the row (thread t owns row t, in place)
         {
@@ -565,18 +723,23 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
         }
         // inverse down column t, sign, update
         {
+            const unsigned lr_bits = __float_as_uint(a.lr);
+            const float decay = 1.f - a.lr * a.wd;
             float r[S];
 #pragma unroll
             for (int u = 0; u < S; ++u) r[u] = St[u * XS + t];
             fdct::dct3_ortho<S>(r);
 #pragma unroll
             for (int i = 0; i < S; ++i) {
+                // x - lr (sign(R) + wd x) = x (1 - lr wd) - lr sign(R); -lr sign(R) is lr with its sign
+                // flipped where R > 0, and zero where R == 0
                 const float rv = r[i];
-                const float sg = (float)((rv > 0.f) - (rv < 0.f));
-                const float xv = Xt[i * S + t];
-                x[base + (size_t)i * te.n1 + t] = fmaf(-a.lr, fmaf(a.wd, xv, sg), xv);
+                float stepv = __uint_as_float(lr_bits ^ (~__float_as_uint(rv) & 0x80000000u));
+                stepv = (rv == 0.f) ? 0.f : stepv;
+                x[base + (size_t)i * te.n1 + t] = fmaf(Xt[i * S + t], decay, stepv);
             }
         }
+        fence_proxy_async();
         __syncthreads();  // Xt and St are free again
     }
 }
@@ -584,7 +747,7 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
 template <int S>
 constexpr size_t compress_smem()
 {
-    return (size_t)S * S * 4 + (size_t)S * Cfg<S>::XS * 4 + 4 * S * 4 + S * 4 + CAP * 8 + 64 * 8 + 16 * 4 + 16;
+    return (size_t)S * S * 4 + (size_t)S * Cfg<S>::XS * 4 + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
 }
 template <int S>
 constexpr size_t decode_smem()
@@ -615,22 +778,24 @@ bool demo_fast_supported(int s) { return s == 64 || s == 32; }
 
 cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
 {
-    if (s == 64) {
-        if (a.grad_bf16)
-            return launch(compress_fast_kernel<64, __nv_bfloat16>, 64, compress_smem<64>(), a.n_chunks, sm_count, stream, &a);
-        return launch(compress_fast_kernel<64, float>, 64, compress_smem<64>(), a.n_chunks, sm_count, stream, &a);
-    }
-    if (s == 32) {
-        if (a.grad_bf16)
-            return launch(compress_fast_kernel<32, __nv_bfloat16>, 32, compress_smem<32>(), a.n_chunks, sm_count, stream, &a);
-        return launch(compress_fast_kernel<32, float>, 32, compress_smem<32>(), a.n_chunks, sm_count, stream, &a);
-    }
+    const bool tm = a.tmap_m != nullptr && a.tmap_g != nullptr;
+#define DEMO_LAUNCH_COMPRESS(SS, GT)                                                                              \
+    (tm ? launch(compress_fast_kernel<SS, GT, true>, SS, compress_smem<SS>(), a.n_chunks, sm_count, stream, &a)    \
+        : launch(compress_fast_kernel<SS, GT, false>, SS, compress_smem<SS>(), a.n_chunks, sm_count, stream, &a))
+    if (s == 64) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(64, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(64, float);
+    if (s == 32) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(32, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(32, float);
+#undef DEMO_LAUNCH_COMPRESS
     return cudaErrorInvalidValue;
 }
 
 cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
 {
-    if (s == 64) return launch(decode_fast_kernel<64>, 64, decode_smem<64>(), a.n_chunks, sm_count, stream, &a);
-    if (s == 32) return launch(decode_fast_kernel<32>, 32, decode_smem<32>(), a.n_chunks, sm_count, stream, &a);
+    const bool tm = a.tmap_x != nullptr;
+    if (s == 64)
+        return tm ? launch(decode_fast_kernel<64, true>, 64, decode_smem<64>(), a.n_chunks, sm_count, stream, &a)
+                  : launch(decode_fast_kernel<64, false>, 64, decode_smem<64>(), a.n_chunks, sm_count, stream, &a);
+    if (s == 32)
+        return tm ? launch(decode_fast_kernel<32, true>, 32, decode_smem<32>(), a.n_chunks, sm_count, stream, &a)
+                  : launch(decode_fast_kernel<32, false>, 32, decode_smem<32>(), a.n_chunks, sm_count, stream, &a);
     return cudaErrorInvalidValue;
 }
