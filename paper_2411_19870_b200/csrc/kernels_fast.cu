@@ -190,6 +190,16 @@ __device__ __forceinline__ unsigned warp_inclusive_scan(unsigned v, int lane)
     return v;
 }
 
+// Bytes of the tile area of the compress kernel: the staged m and g tiles, or the padded transpose
+// tile that later aliases them, whichever is larger.
+template <int S, typename GT>
+constexpr size_t compress_region_bytes()
+{
+    constexpr size_t stage = (size_t)S * S * (sizeof(float) + sizeof(GT));
+    constexpr size_t xt = (size_t)S * Cfg<S>::XS * sizeof(float);
+    return stage > xt ? stage : xt;
+}
+
 #ifndef DEMO_FAST_MIN_BLOCKS
 #define DEMO_FAST_MIN_BLOCKS 8
 #endif
@@ -205,9 +215,13 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
     constexpr int ITER = CAPW / 32;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    float *Bt = reinterpret_cast<float *>(smem_raw);             // [S*S]   m tile, then B
-    float *X = Bt + S * S;                                       // [S*XS]  g staging / transpose / Q / T
-    float *tmax = X + S * XS;                                    // [S]
+    // The staging area of the m and g tiles is reused as the transpose / coefficient / row-stage
+    // tile X once column t has been consumed; B itself is not kept in shared memory: for the residual
+    // the two tiles are fetched a second time (an L2 hit, issued behind the inverse transform).
+    float *Ms = reinterpret_cast<float *>(smem_raw);             // [S*S]   m tile
+    GT *Gs = reinterpret_cast<GT *>(Ms + S * S);                 // [S*S]   g tile
+    float *X = Ms;                                               // [S*XS]  transpose / Q / T (aliases the tiles)
+    float *tmax = reinterpret_cast<float *>(smem_raw + compress_region_bytes<S, GT>());  // [S]
     int *cand_idx = reinterpret_cast<int *>(tmax + S);           // [CAP]
     float *cand_val = reinterpret_cast<float *>(cand_idx + CAP + 8); // [CAP + 8]
     unsigned *cand_key = reinterpret_cast<unsigned *>(cand_val + CAP + 8);  // [CAP + 8]
@@ -232,12 +246,14 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
     int cached_tensor = -1;
     unsigned phase = 0;
 
-    // Locate the tile of chunk c (advances the tensor cursor; chunk ids only grow): row t of the tile
-    // for the row-by-row path, tensor map and box coordinates for the TMA path.
-    const float *m_src = nullptr;
-    const GT *g_src = nullptr;
-    const char *tm_m = nullptr, *tm_g = nullptr;
-    int ld_x = 0, ld_y = 0;
+    // Locate the tile of chunk c (advances the tensor cursor; chunk ids only grow): tensor maps and box
+    // coordinates for the TMA path, row t of the tile for the row-by-row path.
+    struct TileRef {
+        const char *tm_m, *tm_g;
+        int x, y;
+        const float *m_src;
+        const GT *g_src;
+    };
     auto locate = [&](long long c) {
         cur.seek(a.entries, a.n_entries, c);
         if (cur.te.tensor != cached_tensor) {
@@ -248,36 +264,42 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
         const long long lc = c - cur.te.chunk_begin;
         const long long k0 = lc / cur.te.c1;
         const int k1 = (int)(lc - k0 * cur.te.c1);
+        TileRef r;
+        r.tm_m = r.tm_g = nullptr;
+        r.x = k1 * S;
+        r.y = (int)k0 * S;
+        r.m_src = nullptr;
+        r.g_src = nullptr;
         if (TMAP) {
-            tm_m = static_cast<const char *>(a.tmap_m) + (size_t)cached_tensor * TMAP_BYTES;
-            tm_g = static_cast<const char *>(a.tmap_g) + (size_t)cached_tensor * TMAP_BYTES;
-            ld_x = k1 * S;
-            ld_y = (int)k0 * S;
+            r.tm_m = static_cast<const char *>(a.tmap_m) + (size_t)cached_tensor * TMAP_BYTES;
+            r.tm_g = static_cast<const char *>(a.tmap_g) + (size_t)cached_tensor * TMAP_BYTES;
         } else {
             const size_t off = ((size_t)k0 * S + t) * (size_t)cur.te.n1 + (size_t)k1 * S;
-            m_src = m_ptr + off;
-            g_src = g_ptr + off;
+            r.m_src = m_ptr + off;
+            r.g_src = g_ptr + off;
         }
+        return r;
     };
     // Called right after a CTA-wide barrier that follows a fence.proxy.async of every thread.
-    auto issue_loads = [&]() {
+    auto issue_loads = [&](const TileRef &r) {
         if (TMAP) {
             if (t == 0) {
                 mbar_expect_tx(bar, TILE_BYTES);
-                tma_load_2d(smem_u32(Bt), tm_m, ld_x, ld_y, bar);
-                tma_load_2d(smem_u32(X), tm_g, ld_x, ld_y, bar);
+                tma_load_2d(smem_u32(Ms), r.tm_m, r.x, r.y, bar);
+                tma_load_2d(smem_u32(Gs), r.tm_g, r.x, r.y, bar);
             }
         } else {
             if (t == 0) mbar_expect_tx(bar, TILE_BYTES);
-            bulk_g2s(smem_u32(Bt + t * S), m_src, S * sizeof(float), bar);
-            bulk_g2s(smem_u32(reinterpret_cast<GT *>(X) + t * S), g_src, S * sizeof(GT), bar);
+            bulk_g2s(smem_u32(Ms + t * S), r.m_src, S * sizeof(float), bar);
+            bulk_g2s(smem_u32(Gs + t * S), r.g_src, S * sizeof(GT), bar);
         }
     };
 
     long long c = blockIdx.x;
+    TileRef tile_cur, tile_next;
     if (c < a.n_chunks) {
-        locate(c);
-        issue_loads();
+        tile_cur = locate(c);
+        issue_loads(tile_cur);
     }
 
     for (; c < a.n_chunks; c += gridDim.x) {
@@ -301,42 +323,42 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
         // start pulling the next chunk's rows into L2 while this chunk is processed
         const long long nc = c + gridDim.x;
         if (nc < a.n_chunks) {
-            locate(nc);
+            tile_next = locate(nc);
             if (TMAP && t == 0) {
-                tma_prefetch_2d(tm_m, ld_x, ld_y);
-                tma_prefetch_2d(tm_g, ld_x, ld_y);
+                tma_prefetch_2d(tile_next.tm_m, tile_next.x, tile_next.y);
+                tma_prefetch_2d(tile_next.tm_g, tile_next.x, tile_next.y);
             }
         }
 
-        // ---- momentum update on column t, first DCT pass down the column -------------------------
-        {
-            float x[S];
-            const GT *gs = reinterpret_cast<const GT *>(X);
-#pragma unroll
-            for (int i = 0; i < S; ++i) x[i] = fmaf(a.beta, Bt[i * S + t], to_f32(gs[i * S + t]));
-            __syncthreads();  // every thread has consumed the g staging area inside X
-#pragma unroll
-            for (int i = 0; i < S; ++i) Bt[i * S + t] = x[i];
-            fdct::dct2_ortho<S>(x);
-#pragma unroll
-            for (int u = 0; u < S; ++u) X[u * XS + t] = x[u];
-        }
-        __syncthreads();
-
-        // ---- second DCT pass along row t: q[v] = Q[t][v] -----------------------------------------
+        // ---- momentum update on column t, then the two DCT passes --------------------------------
+        // One copy of the unrolled transform serves both passes (the loop is kept rolled to halve the
+        // instruction footprint): pass 0 runs down column t of B = beta*m + g and writes the
+        // transpose tile, pass 1 runs along row t and leaves q[v] = Q[t][v] in registers.
         float q[S];
-        {
-            const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass == 0) {
 #pragma unroll
-            for (int v4 = 0; v4 < S / 4; ++v4) {
-                const float4 f = row[v4];
-                q[4 * v4 + 0] = f.x;
-                q[4 * v4 + 1] = f.y;
-                q[4 * v4 + 2] = f.z;
-                q[4 * v4 + 3] = f.w;
+                for (int i = 0; i < S; ++i) q[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
+                __syncthreads();  // every thread has consumed its column of the staged tiles (X aliases them)
+            } else {
+                const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
+#pragma unroll
+                for (int v4 = 0; v4 < S / 4; ++v4) {
+                    const float4 f = row[v4];
+                    q[4 * v4 + 0] = f.x;
+                    q[4 * v4 + 1] = f.y;
+                    q[4 * v4 + 2] = f.z;
+                    q[4 * v4 + 3] = f.w;
+                }
+            }
+            fdct::dct2_ortho<S>(q);
+            if (pass == 0) {
+#pragma unroll
+                for (int u = 0; u < S; ++u) X[u * XS + t] = q[u];
+                __syncthreads();
             }
         }
-        fdct::dct2_ortho<S>(q);
 
         // ---- top-k ------------------------------------------------------------------------------
         bool use_fallback = (k_eff > S);
@@ -605,13 +627,29 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             float r[S];
 #pragma unroll
             for (int u = 0; u < S; ++u) r[u] = X[u * XS + t];
+            // X is dead: fetch the m and g tiles again (they were read moments ago, so this is an L2
+            // hit) while the inverse transform runs, and rebuild B = beta*m + g for the residual
+            fence_proxy_async();
+            __syncthreads();
+            issue_loads(tile_cur);
             fdct::dct3_ortho<S>(r);
+            const bool again = mbar_wait_bounded(bar, phase);
+            phase ^= 1u;
+            if (!__syncthreads_and(again)) {
+                if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
+                mbar_wait_bounded(bar, phase ^ 1u);
+                return;
+            }
 #pragma unroll
-            for (int i = 0; i < S; ++i) m[base + (size_t)i * te.n1 + t] = Bt[i * S + t] - r[i];
+            for (int i = 0; i < S; ++i)
+                m[base + (size_t)i * te.n1 + t] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t])) - r[i];
         }
         fence_proxy_async();  // order this thread's shared-memory accesses before the async-proxy writes
-        __syncthreads();      // Bt and X are free again
-        if (nc < a.n_chunks) issue_loads();
+        __syncthreads();      // the staging area is free again
+        if (nc < a.n_chunks) {
+            tile_cur = tile_next;
+            issue_loads(tile_cur);
+        }
     }
 }
 
@@ -744,10 +782,10 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
     }
 }
 
-template <int S>
+template <int S, typename GT>
 constexpr size_t compress_smem()
 {
-    return (size_t)S * S * 4 + (size_t)S * Cfg<S>::XS * 4 + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
+    return compress_region_bytes<S, GT>() + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
 }
 template <int S>
 constexpr size_t decode_smem()
@@ -780,8 +818,8 @@ cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_c
 {
     const bool tm = a.tmap_m != nullptr && a.tmap_g != nullptr;
 #define DEMO_LAUNCH_COMPRESS(SS, GT)                                                                              \
-    (tm ? launch(compress_fast_kernel<SS, GT, true>, SS, compress_smem<SS>(), a.n_chunks, sm_count, stream, &a)    \
-        : launch(compress_fast_kernel<SS, GT, false>, SS, compress_smem<SS>(), a.n_chunks, sm_count, stream, &a))
+    (tm ? launch(compress_fast_kernel<SS, GT, true>, SS, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a)    \
+        : launch(compress_fast_kernel<SS, GT, false>, SS, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a))
     if (s == 64) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(64, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(64, float);
     if (s == 32) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(32, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(32, float);
 #undef DEMO_LAUNCH_COMPRESS
