@@ -94,12 +94,43 @@ __device__ __forceinline__ float max3f(float a, float b, float c)
 __device__ __forceinline__ float max3abs(float a, float b, float c) { return max3f(fabsf(a), fabsf(b), fabsf(c)); }
 __device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
+// A CTA hosts NCH independent "slots" of S threads, one chunk each.  Threads of a slot meet at the
+// slot's own named barrier (a warp-level barrier when the slot is a single warp); all slots meet once
+// per chunk at the CTA barrier, which keeps the warps of the CTA in the same region of the (large,
+// fully unrolled) code so that instruction fetches are shared instead of streamed once per warp.
+template <int S>
+struct SlotBarrier {
+    int id;  // named barrier 1..15
+    __device__ __forceinline__ void sync() const
+    {
+        if (S == 32)
+            __syncwarp();
+        else
+            asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(S) : "memory");
+    }
+    __device__ __forceinline__ bool sync_and(bool pred) const
+    {
+        if (S == 32) return __all_sync(0xffffffffu, pred);
+        unsigned r;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 q, %3, 0;\n\t"
+            "bar.red.and.pred p, %1, %2, q;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(r)
+            : "r"(id), "n"(S), "r"((unsigned)pred)
+            : "memory");
+        return r != 0;
+    }
+};
+
 template <int S>
 struct Cfg {
     static constexpr int XS = S + 4;  // row stride of the transpose tile: conflict-free scalar
                                       // column access and 128-bit row access
     static constexpr int NW = S / 32;
     static constexpr int LOG2S = (S == 64) ? 6 : 5;
+    static constexpr int NCH = 256 / S;  // slots per CTA
 };
 
 // Walks the tensor table as the CTA's chunk ids grow.
@@ -130,10 +161,9 @@ struct EntryCursor {
 // ------------------------------------------------------------------------------------------------
 template <int S>
 __device__ __forceinline__ void radix_select_tile(const float *X, int k_eff, unsigned *hist, unsigned *s_state,
-                                                  unsigned *thr, unsigned *need_eq)
+                                                  unsigned *thr, unsigned *need_eq, int t, SlotBarrier<S> sb)
 {
     constexpr int XS = Cfg<S>::XS;
-    const int t = threadIdx.x;
     if (t == 0) {
         s_state[0] = 0u;
         s_state[1] = (unsigned)k_eff;
@@ -142,13 +172,13 @@ __device__ __forceinline__ void radix_select_tile(const float *X, int k_eff, uns
         const int shift = 24 - 8 * pass;
         const unsigned mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
         for (int i = t; i < 256; i += S) hist[i] = 0u;
-        __syncthreads();
+        sb.sync();
         const unsigned prefix = s_state[0];
         for (int v = 0; v < S; ++v) {
             const unsigned key = mag_key(X[t * XS + v]);
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
-        __syncthreads();
+        sb.sync();
         if (t < 32) {
             const unsigned rem = s_state[1];
             unsigned local = 0;
@@ -173,7 +203,7 @@ __device__ __forceinline__ void radix_select_tile(const float *X, int k_eff, uns
                 s_state[0] = prefix | ((unsigned)b << shift);
             }
         }
-        __syncthreads();
+        sb.sync();
     }
     *thr = s_state[0];
     *need_eq = s_state[1];
@@ -200,12 +230,19 @@ constexpr size_t compress_region_bytes()
     return stage > xt ? stage : xt;
 }
 
+template <int S, typename GT>
+constexpr size_t compress_slot_bytes()
+{
+    constexpr size_t raw = compress_region_bytes<S, GT>() + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
+    return (raw + 127) / 128 * 128;
+}
+
 #ifndef DEMO_FAST_MIN_BLOCKS
-#define DEMO_FAST_MIN_BLOCKS 8
+#define DEMO_FAST_MIN_BLOCKS 2
 #endif
 
 template <int S, typename GT, bool TMAP>
-__global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(DemoCompressArgs a)
+__global__ void __launch_bounds__(256, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(DemoCompressArgs a)
 {
     using C = Cfg<S>;
     constexpr int XS = C::XS, NW = C::NW, LOG2S = C::LOG2S;
@@ -214,7 +251,10 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
     constexpr int CAPWP = CAPW + 4;       // list stride (padding for 128-bit key loads)
     constexpr int ITER = CAPW / 32;
 
-    extern __shared__ __align__(128) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_all[];
+    const int slot = threadIdx.x / S;
+    unsigned char *smem_raw = smem_all + (size_t)slot * compress_slot_bytes<S, GT>();
+    const SlotBarrier<S> sb{slot + 1};
     // The staging area of the m and g tiles is reused as the transpose / coefficient / row-stage
     // tile X once column t has been consumed; B itself is not kept in shared memory: for the residual
     // the two tiles are fetched a second time (an L2 hit, issued behind the inverse transform).
@@ -230,7 +270,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
     unsigned *misc = reinterpret_cast<unsigned *>(recs4 + 64);   // [16]
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(misc + 16);
 
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    const int t = threadIdx.x % S, lane = t & 31, warp = t >> 5;
     const uint32_t bar = smem_u32(bar_mem);
 
     if (t == 0) {
@@ -239,6 +279,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
     }
     __syncthreads();
     fence_proxy_async();
+    bool failed = false;  // slot-uniform: a bounded wait of this slot expired
 
     EntryCursor cur;
     float *m_ptr = nullptr;
@@ -295,14 +336,20 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
         }
     };
 
-    long long c = blockIdx.x;
+    // chunk ids: CTA b, slot s, round r  ->  (r * gridDim.x + b) * NCH + s
+    constexpr int NCH = C::NCH;
+    const long long stride = (long long)gridDim.x * NCH;
+    long long c = (long long)blockIdx.x * NCH + slot;
     TileRef tile_cur, tile_next;
     if (c < a.n_chunks) {
         tile_cur = locate(c);
         issue_loads(tile_cur);
     }
 
-    for (; c < a.n_chunks; c += gridDim.x) {
+    for (long long cb = (long long)blockIdx.x * NCH; cb < a.n_chunks; cb += stride, c += stride) {
+        // all slots of the CTA start a chunk together; a slot whose wait expired takes the CTA down
+        if (__syncthreads_or(failed)) return;
+        if (c >= a.n_chunks) continue;
         // the cursor points at chunk c (issue_loads(c) ran last)
         const DemoTensorEntry te = cur.te;
         const long long lc = c - te.chunk_begin;
@@ -315,13 +362,14 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
 
         const bool arrived = mbar_wait_bounded(bar, phase);
         phase ^= 1u;
-        if (!__syncthreads_and(arrived)) {
+        if (!sb.sync_and(arrived)) {
             if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
             mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
-            return;
+            failed = true;
+            continue;
         }
         // start pulling the next chunk's rows into L2 while this chunk is processed
-        const long long nc = c + gridDim.x;
+        const long long nc = c + stride;
         if (nc < a.n_chunks) {
             tile_next = locate(nc);
             if (TMAP && t == 0) {
@@ -340,7 +388,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             if (pass == 0) {
 #pragma unroll
                 for (int i = 0; i < S; ++i) q[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
-                __syncthreads();  // every thread has consumed its column of the staged tiles (X aliases them)
+                sb.sync();  // every thread has consumed its column of the staged tiles (X aliases them)
             } else {
                 const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
 #pragma unroll
@@ -356,7 +404,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             if (pass == 0) {
 #pragma unroll
                 for (int u = 0; u < S; ++u) X[u * XS + t] = q[u];
-                __syncthreads();
+                sb.sync();
             }
         }
 
@@ -381,7 +429,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             const unsigned tkey = __float_as_uint(tm);
             unsigned *tk = reinterpret_cast<unsigned *>(tmax);
             tk[t] = tkey;
-            __syncthreads();
+            sb.sync();
             unsigned lmin;
             {
                 const unsigned okey = (NW > 1) ? tk[t ^ 32] : tkey;
@@ -443,7 +491,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
                 }
                 if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
             }
-            __syncthreads();
+            sb.sync();
             unsigned n_w[NW];
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
@@ -478,12 +526,12 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
                     pre[it] = __popc(bal & ((1u << lane) - 1u));
                     if (lane == 0) misc[4 + warp * ITER + it] = __popc(bal);
                 }
-                __syncthreads();
+                sb.sync();
                 unsigned total = 0;
 #pragma unroll
                 for (int g = 0; g < ITER * NW; ++g) total += misc[4 + g];
                 if (total != (unsigned)k_eff) {  // block-uniform: equal magnitudes straddle the threshold
-                    __syncthreads();
+                    sb.sync();
 #pragma unroll
                     for (int it = 0; it < ITER; ++it) {
                         const unsigned li = it * 32 + lane;
@@ -504,7 +552,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
                         pre[it] = __popc(bal & ((1u << lane) - 1u));
                         if (lane == 0) misc[4 + warp * ITER + it] = __popc(bal);
                     }
-                    __syncthreads();
+                    sb.sync();
                 }
 #pragma unroll
                 for (int it = 0; it < ITER; ++it) {
@@ -525,9 +573,9 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             }
         }
         if (use_fallback) {
-            __syncthreads();  // coefficient tile complete in X
+            sb.sync();  // coefficient tile complete in X
             unsigned thr, need_eq;
-            radix_select_tile<S>(X, k_eff, hist, misc, &thr, &need_eq);
+            radix_select_tile<S>(X, k_eff, hist, misc, &thr, &need_eq, t, sb);
             unsigned gt = 0, eq = 0;
             for (int v = 0; v < S; ++v) {
                 const unsigned key = mag_key(X[t * XS + v]);
@@ -536,9 +584,9 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             }
             const unsigned packed = gt | (eq << 16);
             const unsigned inc = warp_inclusive_scan(packed, lane);
-            __syncthreads();  // radix_select_tile's last reads of misc are done
+            sb.sync();  // radix_select_tile's last reads of misc are done
             if (lane == 31) misc[warp] = inc;
-            __syncthreads();
+            sb.sync();
             unsigned before = inc - packed;
 #pragma unroll
             for (int w = 0; w < NW; ++w)
@@ -573,7 +621,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
                 }
             }
         }
-        __syncthreads();  // records complete (shared list and global payload); X is free
+        sb.sync();  // records complete (shared list and global payload); X is free
 
         // ---- residual: row stage of the inverse from the k_eff records, sparse ------------------
         {
@@ -581,7 +629,7 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
 #pragma unroll
             for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        __syncthreads();
+        sb.sync();
         {
             // T[u][t] = sum over kept (u, v) of val * C[v][t]; the basis is read through L1 (all CTAs
             // of the SM share the same 4*S*S bytes), coalesced across the warp
@@ -630,22 +678,23 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
             // X is dead: fetch the m and g tiles again (they were read moments ago, so this is an L2
             // hit) while the inverse transform runs, and rebuild B = beta*m + g for the residual
             fence_proxy_async();
-            __syncthreads();
+            sb.sync();
             issue_loads(tile_cur);
             fdct::dct3_ortho<S>(r);
             const bool again = mbar_wait_bounded(bar, phase);
             phase ^= 1u;
-            if (!__syncthreads_and(again)) {
+            if (!sb.sync_and(again)) {
                 if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
                 mbar_wait_bounded(bar, phase ^ 1u);
-                return;
+                failed = true;
+                continue;
             }
 #pragma unroll
             for (int i = 0; i < S; ++i)
                 m[base + (size_t)i * te.n1 + t] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t])) - r[i];
         }
         fence_proxy_async();  // order this thread's shared-memory accesses before the async-proxy writes
-        __syncthreads();      // the staging area is free again
+        sb.sync();      // the staging area is free again
         if (nc < a.n_chunks) {
             tile_cur = tile_next;
             issue_loads(tile_cur);
@@ -653,18 +702,29 @@ __global__ void __launch_bounds__(S, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(
     }
 }
 
+template <int S>
+constexpr size_t decode_slot_bytes()
+{
+    return ((size_t)S * Cfg<S>::XS * 4 + 16 + 127) / 128 * 128;
+}
+
 template <int S, bool TMAP>
-__global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
+__global__ void __launch_bounds__(256, 2) decode_fast_kernel(DemoDecodeArgs a)
 {
     using C = Cfg<S>;
-    constexpr int XS = C::XS;
+    constexpr int XS = C::XS, NCH = C::NCH;
     constexpr int M = S * S;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    float *Xt = reinterpret_cast<float *>(smem_raw);  // [S*S]  x tile
-    float *St = Xt + S * S;                           // [S*XS] aggregate, then row-stage output
+    extern __shared__ __align__(128) unsigned char smem_all[];
+    const int slot = threadIdx.x / S;
+    unsigned char *smem_raw = smem_all + (size_t)slot * decode_slot_bytes<S>();
+    const SlotBarrier<S> sb{slot + 1};
+    // One tile per slot: the aggregate S, then the row-stage output, and -- once column t has been
+    // read back into registers -- the staging area of the x tile, fetched behind the second transform.
+    float *St = reinterpret_cast<float *>(smem_raw);  // [S*XS]
+    float *Xt = St;                                   // [S*S] (aliases St)
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XS);
 
-    const int t = threadIdx.x;
+    const int t = threadIdx.x % S;
     const uint32_t bar = smem_u32(bar_mem);
     if (t == 0) {
         mbar_init(bar, 1);
@@ -677,8 +737,15 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
     float *x_ptr = nullptr;
     int cached_tensor = -1;
     unsigned phase = 0;
+    bool failed = false;
+    const unsigned lr_bits = __float_as_uint(a.lr);
+    const float decay = 1.f - a.lr * a.wd;
 
-    for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
+    const long long stride = (long long)gridDim.x * NCH;
+    long long c = (long long)blockIdx.x * NCH + slot;
+    for (long long cb = (long long)blockIdx.x * NCH; cb < a.n_chunks; cb += stride, c += stride) {
+        if (__syncthreads_or(failed)) return;  // all slots start a chunk together (shared instruction stream)
+        if (c >= a.n_chunks) continue;
         cur.seek(a.entries, a.n_entries, c);
         const DemoTensorEntry te = cur.te;
         if (te.tensor != cached_tensor) {
@@ -692,26 +759,15 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
         float *__restrict__ x = x_ptr;
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + lc * (long long)k_eff;
-
-        // stage the x tile while the aggregate is built (the previous iteration ended with a
-        // fence.proxy.async of every thread and a barrier)
-        if (TMAP) {
-            if (t == 0) {
-                mbar_expect_tx(bar, S * S * sizeof(float));
-                tma_load_2d(smem_u32(Xt), static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES, k1 * S,
-                            (int)k0 * S, bar);
-            }
-        } else {
-            if (t == 0) mbar_expect_tx(bar, S * S * sizeof(float));
-            bulk_g2s(smem_u32(Xt + t * S), x + base + (size_t)t * te.n1, S * sizeof(float), bar);
-        }
+        if (TMAP && t == 0)
+            tma_prefetch_2d(static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES, k1 * S, (int)k0 * S);
 
         {
             float4 *row = reinterpret_cast<float4 *>(St + t * XS);
 #pragma unroll
             for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        __syncthreads();
+        sb.sync();
         // S = sum over workers in worker order; a barrier per worker fixes the order of additions.
         // Records are fetched eight workers ahead so that one memory latency covers eight workers.
         for (int kb = 0; kb < k_eff; kb += S) {
@@ -730,84 +786,103 @@ __global__ void __launch_bounds__(S) decode_fast_kernel(DemoDecodeArgs a)
                             else
                                 atomicMax(a.status, DEMO_DEV_PAYLOAD);
                         }
-                        __syncthreads();
+                        sb.sync();
                     }
                 }
             }
         }
-        // inverse along the row (thread t owns row t, in place)
-        {
-            float r[S];
-            float4 *row = reinterpret_cast<float4 *>(St + t * XS);
+        // Two inverse passes through one copy of the unrolled transform (rolled loop): pass 0 along
+        // row t in place, pass 1 down column t; the x tile is fetched while pass 1 computes.
+        float r[S];
+        bool arrived = true;
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass == 0) {
+                const float4 *row = reinterpret_cast<const float4 *>(St + t * XS);
 #pragma unroll
-            for (int v4 = 0; v4 < S / 4; ++v4) {
-                const float4 f = row[v4];
-                r[4 * v4 + 0] = f.x;
-                r[4 * v4 + 1] = f.y;
-                r[4 * v4 + 2] = f.z;
-                r[4 * v4 + 3] = f.w;
+                for (int v4 = 0; v4 < S / 4; ++v4) {
+                    const float4 f = row[v4];
+                    r[4 * v4 + 0] = f.x;
+                    r[4 * v4 + 1] = f.y;
+                    r[4 * v4 + 2] = f.z;
+                    r[4 * v4 + 3] = f.w;
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < S; ++u) r[u] = St[u * XS + t];
+                fence_proxy_async();
+                sb.sync();  // the tile is dead: stage x into it
+                if (TMAP) {
+                    if (t == 0) {
+                        mbar_expect_tx(bar, S * S * sizeof(float));
+                        tma_load_2d(smem_u32(Xt), static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES,
+                                    k1 * S, (int)k0 * S, bar);
+                    }
+                } else {
+                    if (t == 0) mbar_expect_tx(bar, S * S * sizeof(float));
+                    bulk_g2s(smem_u32(Xt + t * S), x + base + (size_t)t * te.n1, S * sizeof(float), bar);
+                }
             }
             fdct::dct3_ortho<S>(r);
+            if (pass == 0) {
+                float4 *row = reinterpret_cast<float4 *>(St + t * XS);
 #pragma unroll
-            for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(r[4 * v4], r[4 * v4 + 1], r[4 * v4 + 2], r[4 * v4 + 3]);
+                for (int v4 = 0; v4 < S / 4; ++v4)
+                    row[v4] = make_float4(r[4 * v4], r[4 * v4 + 1], r[4 * v4 + 2], r[4 * v4 + 3]);
+                sb.sync();
+            } else {
+                arrived = mbar_wait_bounded(bar, phase);
+                phase ^= 1u;
+            }
         }
-        __syncthreads();
-        const bool arrived = mbar_wait_bounded(bar, phase);
-        phase ^= 1u;
-        if (!__syncthreads_and(arrived)) {
+        if (!sb.sync_and(arrived)) {
             if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
             mbar_wait_bounded(bar, phase ^ 1u);
-            return;
+            failed = true;
+            continue;
         }
-        // inverse down column t, sign, update
-        {
-            const unsigned lr_bits = __float_as_uint(a.lr);
-            const float decay = 1.f - a.lr * a.wd;
-            float r[S];
+        // sign and update:  x - lr (sign(R) + wd x) = x (1 - lr wd) - lr sign(R); -lr sign(R) is lr with
+        // its sign flipped where R > 0, and zero where R == 0
 #pragma unroll
-            for (int u = 0; u < S; ++u) r[u] = St[u * XS + t];
-            fdct::dct3_ortho<S>(r);
-#pragma unroll
-            for (int i = 0; i < S; ++i) {
-                // x - lr (sign(R) + wd x) = x (1 - lr wd) - lr sign(R); -lr sign(R) is lr with its sign
-                // flipped where R > 0, and zero where R == 0
-                const float rv = r[i];
-                float stepv = __uint_as_float(lr_bits ^ (~__float_as_uint(rv) & 0x80000000u));
-                stepv = (rv == 0.f) ? 0.f : stepv;
-                x[base + (size_t)i * te.n1 + t] = fmaf(Xt[i * S + t], decay, stepv);
-            }
+        for (int i = 0; i < S; ++i) {
+            const float rv = r[i];
+            float stepv = __uint_as_float(lr_bits ^ (~__float_as_uint(rv) & 0x80000000u));
+            stepv = (rv == 0.f) ? 0.f : stepv;
+            x[base + (size_t)i * te.n1 + t] = fmaf(Xt[i * S + t], decay, stepv);
         }
-        fence_proxy_async();
-        __syncthreads();  // Xt and St are free again
+        sb.sync();  // the tile is free again
     }
 }
 
 template <int S, typename GT>
 constexpr size_t compress_smem()
 {
-    return compress_region_bytes<S, GT>() + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
+    return compress_slot_bytes<S, GT>() * Cfg<S>::NCH;
 }
 template <int S>
 constexpr size_t decode_smem()
 {
-    return (size_t)S * S * 4 + (size_t)S * Cfg<S>::XS * 4 + 16;
+    return decode_slot_bytes<S>() * Cfg<S>::NCH;
 }
 
+// Persistent launch: CTAs of 256 threads (nch slots), as many as fit the device, each striding over
+// groups of nch chunks.
 template <typename K>
-cudaError_t launch(K kernel, int threads, size_t smem, long long n_chunks, int sm_count, cudaStream_t stream,
+cudaError_t launch(K kernel, int nch, size_t smem, long long n_chunks, int sm_count, cudaStream_t stream,
                    const void *args)
 {
     if (n_chunks <= 0) return cudaSuccess;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     int per_sm = 0;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, smem);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
+    const long long groups = (n_chunks + nch - 1) / nch;
     long long grid = (long long)sm_count * per_sm;
-    if (grid > n_chunks) grid = n_chunks;
+    if (grid > groups) grid = groups;
     void *params[] = {const_cast<void *>(args)};
-    return cudaLaunchKernel((const void *)kernel, dim3((unsigned)grid), dim3(threads), params, smem, stream);
+    return cudaLaunchKernel((const void *)kernel, dim3((unsigned)grid), dim3(256), params, smem, stream);
 }
 
 }  // namespace
@@ -818,8 +893,8 @@ cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_c
 {
     const bool tm = a.tmap_m != nullptr && a.tmap_g != nullptr;
 #define DEMO_LAUNCH_COMPRESS(SS, GT)                                                                              \
-    (tm ? launch(compress_fast_kernel<SS, GT, true>, SS, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a)    \
-        : launch(compress_fast_kernel<SS, GT, false>, SS, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a))
+    (tm ? launch(compress_fast_kernel<SS, GT, true>, Cfg<SS>::NCH, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a)    \
+        : launch(compress_fast_kernel<SS, GT, false>, Cfg<SS>::NCH, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a))
     if (s == 64) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(64, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(64, float);
     if (s == 32) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(32, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(32, float);
 #undef DEMO_LAUNCH_COMPRESS
@@ -830,10 +905,10 @@ cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count
 {
     const bool tm = a.tmap_x != nullptr;
     if (s == 64)
-        return tm ? launch(decode_fast_kernel<64, true>, 64, decode_smem<64>(), a.n_chunks, sm_count, stream, &a)
-                  : launch(decode_fast_kernel<64, false>, 64, decode_smem<64>(), a.n_chunks, sm_count, stream, &a);
+        return tm ? launch(decode_fast_kernel<64, true>, Cfg<64>::NCH, decode_smem<64>(), a.n_chunks, sm_count, stream, &a)
+                  : launch(decode_fast_kernel<64, false>, Cfg<64>::NCH, decode_smem<64>(), a.n_chunks, sm_count, stream, &a);
     if (s == 32)
-        return tm ? launch(decode_fast_kernel<32, true>, 32, decode_smem<32>(), a.n_chunks, sm_count, stream, &a)
-                  : launch(decode_fast_kernel<32, false>, 32, decode_smem<32>(), a.n_chunks, sm_count, stream, &a);
+        return tm ? launch(decode_fast_kernel<32, true>, Cfg<32>::NCH, decode_smem<32>(), a.n_chunks, sm_count, stream, &a)
+                  : launch(decode_fast_kernel<32, false>, Cfg<32>::NCH, decode_smem<32>(), a.n_chunks, sm_count, stream, &a);
     return cudaErrorInvalidValue;
 }
