@@ -130,7 +130,6 @@ struct Cfg {
                                       // column access and 128-bit row access
     static constexpr int NW = S / 32;
     static constexpr int LOG2S = (S == 64) ? 6 : 5;
-    static constexpr int NCH = 256 / S;  // slots per CTA
 };
 
 // Walks the tensor table as the CTA's chunk ids grow.
@@ -237,12 +236,8 @@ constexpr size_t compress_slot_bytes()
     return (raw + 127) / 128 * 128;
 }
 
-#ifndef DEMO_FAST_MIN_BLOCKS
-#define DEMO_FAST_MIN_BLOCKS 2
-#endif
-
-template <int S, typename GT, bool TMAP>
-__global__ void __launch_bounds__(256, DEMO_FAST_MIN_BLOCKS) compress_fast_kernel(DemoCompressArgs a)
+template <int S, typename GT, bool TMAP, int THREADS>
+__global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(DemoCompressArgs a)
 {
     using C = Cfg<S>;
     constexpr int XS = C::XS, NW = C::NW, LOG2S = C::LOG2S;
@@ -337,7 +332,7 @@ __global__ void __launch_bounds__(256, DEMO_FAST_MIN_BLOCKS) compress_fast_kerne
     };
 
     // chunk ids: CTA b, slot s, round r  ->  (r * gridDim.x + b) * NCH + s
-    constexpr int NCH = C::NCH;
+    constexpr int NCH = THREADS / S;
     const long long stride = (long long)gridDim.x * NCH;
     long long c = (long long)blockIdx.x * NCH + slot;
     TileRef tile_cur, tile_next;
@@ -708,11 +703,11 @@ constexpr size_t decode_slot_bytes()
     return ((size_t)S * Cfg<S>::XS * 4 + 16 + 127) / 128 * 128;
 }
 
-template <int S, bool TMAP>
-__global__ void __launch_bounds__(256, 2) decode_fast_kernel(DemoDecodeArgs a)
+template <int S, bool TMAP, int THREADS>
+__global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(DemoDecodeArgs a)
 {
     using C = Cfg<S>;
-    constexpr int XS = C::XS, NCH = C::NCH;
+    constexpr int XS = C::XS, NCH = THREADS / S;
     constexpr int M = S * S;
     extern __shared__ __align__(128) unsigned char smem_all[];
     const int slot = threadIdx.x / S;
@@ -854,35 +849,56 @@ __global__ void __launch_bounds__(256, 2) decode_fast_kernel(DemoDecodeArgs a)
     }
 }
 
+// CTA sizes: the compress kernel runs best with all eight slots of an SM in one CTA (one shared
+// instruction stream); fp32 gradients need a larger staging area, so fewer slots fit.  The decode
+// kernel, whose code is smaller, prefers several smaller CTAs.
 template <int S, typename GT>
-constexpr size_t compress_smem()
+constexpr int compress_threads()
 {
-    return compress_slot_bytes<S, GT>() * Cfg<S>::NCH;
+    return (S == 64) ? ((sizeof(GT) == 2) ? 512 : 256) : 256;
 }
-template <int S>
-constexpr size_t decode_smem()
-{
-    return decode_slot_bytes<S>() * Cfg<S>::NCH;
-}
+constexpr int DECODE_THREADS = 128;
 
-// Persistent launch: CTAs of 256 threads (nch slots), as many as fit the device, each striding over
-// groups of nch chunks.
+// Persistent launch: CTAs of `threads` threads (threads / S slots), as many as fit the device, each
+// striding over groups of chunks.
 template <typename K>
-cudaError_t launch(K kernel, int nch, size_t smem, long long n_chunks, int sm_count, cudaStream_t stream,
+cudaError_t launch(K kernel, int threads, int nch, size_t smem, long long n_chunks, int sm_count, cudaStream_t stream,
                    const void *args)
 {
     if (n_chunks <= 0) return cudaSuccess;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     int per_sm = 0;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, smem);
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     const long long groups = (n_chunks + nch - 1) / nch;
     long long grid = (long long)sm_count * per_sm;
     if (grid > groups) grid = groups;
     void *params[] = {const_cast<void *>(args)};
-    return cudaLaunchKernel((const void *)kernel, dim3((unsigned)grid), dim3(256), params, smem, stream);
+    return cudaLaunchKernel((const void *)kernel, dim3((unsigned)grid), dim3(threads), params, smem, stream);
+}
+
+template <int S, typename GT>
+cudaError_t launch_compress(const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
+{
+    constexpr int TH = compress_threads<S, GT>();
+    constexpr int NCH = TH / S;
+    const size_t smem = compress_slot_bytes<S, GT>() * NCH;
+    if (a.tmap_m != nullptr && a.tmap_g != nullptr)
+        return launch(compress_fast_kernel<S, GT, true, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
+    return launch(compress_fast_kernel<S, GT, false, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
+}
+
+template <int S>
+cudaError_t launch_decode(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
+{
+    constexpr int TH = DECODE_THREADS;
+    constexpr int NCH = TH / S;
+    const size_t smem = decode_slot_bytes<S>() * NCH;
+    if (a.tmap_x != nullptr)
+        return launch(decode_fast_kernel<S, true, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
+    return launch(decode_fast_kernel<S, false, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
 }
 
 }  // namespace
@@ -891,24 +907,18 @@ bool demo_fast_supported(int s) { return s == 64 || s == 32; }
 
 cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
 {
-    const bool tm = a.tmap_m != nullptr && a.tmap_g != nullptr;
-#define DEMO_LAUNCH_COMPRESS(SS, GT)                                                                              \
-    (tm ? launch(compress_fast_kernel<SS, GT, true>, Cfg<SS>::NCH, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a)    \
-        : launch(compress_fast_kernel<SS, GT, false>, Cfg<SS>::NCH, compress_smem<SS, GT>(), a.n_chunks, sm_count, stream, &a))
-    if (s == 64) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(64, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(64, float);
-    if (s == 32) return a.grad_bf16 ? DEMO_LAUNCH_COMPRESS(32, __nv_bfloat16) : DEMO_LAUNCH_COMPRESS(32, float);
-#undef DEMO_LAUNCH_COMPRESS
+    if (s == 64)
+        return a.grad_bf16 ? launch_compress<64, __nv_bfloat16>(a, sm_count, stream)
+                           : launch_compress<64, float>(a, sm_count, stream);
+    if (s == 32)
+        return a.grad_bf16 ? launch_compress<32, __nv_bfloat16>(a, sm_count, stream)
+                           : launch_compress<32, float>(a, sm_count, stream);
     return cudaErrorInvalidValue;
 }
 
 cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
 {
-    const bool tm = a.tmap_x != nullptr;
-    if (s == 64)
-        return tm ? launch(decode_fast_kernel<64, true>, Cfg<64>::NCH, decode_smem<64>(), a.n_chunks, sm_count, stream, &a)
-                  : launch(decode_fast_kernel<64, false>, Cfg<64>::NCH, decode_smem<64>(), a.n_chunks, sm_count, stream, &a);
-    if (s == 32)
-        return tm ? launch(decode_fast_kernel<32, true>, Cfg<32>::NCH, decode_smem<32>(), a.n_chunks, sm_count, stream, &a)
-                  : launch(decode_fast_kernel<32, false>, Cfg<32>::NCH, decode_smem<32>(), a.n_chunks, sm_count, stream, &a);
+    if (s == 64) return launch_decode<64>(a, sm_count, stream);
+    if (s == 32) return launch_decode<32>(a, sm_count, stream);
     return cudaErrorInvalidValue;
 }
