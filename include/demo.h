@@ -138,6 +138,46 @@ demo_status demo_step_host(demo_ctx *ctx, const void *const *host_grads, void *c
                            float *const *momentum, void *const *payloads, float *const *params,
                            void *host_payloads_out, void *cuda_stream);
 
+/*
+ * demo_decode_apply_static -- the same decode + update as demo_decode_apply, for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this is a deployment variant of the
+ * server-side step, not another algorithm.)
+ *
+ * Who needs it: code running where cudaMalloc is off limits -- inside a memory pool that owns the
+ * whole device, in a plug-in whose host forbids driver allocations after start-up, or on a stream
+ * that must never hit an implicit synchronisation from an allocator.  demo_init allocates the
+ * context's tables with cudaMalloc; this entry point needs no context and calls neither cudaMalloc,
+ * cudaFree nor any allocating library routine.  The small tables the kernels read (DCT basis, tensor
+ * table, the two pointer tables, a status word) live in one fixed array of DEMO_STATIC_SCRATCH_BYTES
+ * bytes of device memory that every GPU loading this library holds until the process exits.
+ *
+ * Arguments are those of demo_init (cfg, tensors, n_tensors, cuda_device) plus those of
+ * demo_decode_apply (payloads, n_payloads == cfg->num_workers, params, cuda_stream); cfg->beta and
+ * cfg->grad_dtype are ignored.  Payloads and parameters are caller-owned DEVICE buffers, 16-byte
+ * aligned; the pointer arrays are host memory read during the call.
+ *
+ * Limits (larger problems are rejected with DEMO_ERR_UNSUPPORTED before anything is enqueued):
+ * n_tensors <= DEMO_STATIC_MAX_TENSORS, n_payloads <= DEMO_STATIC_MAX_WORKERS,
+ * cfg->chunk <= DEMO_STATIC_MAX_CHUNK.
+ *
+ * Sharing: all calls in the process use the same array on a given device.  Each call rewrites the
+ * tables and zeroes the status word in stream order, so consecutive calls on ONE stream are safe;
+ * calls whose kernels may overlap on the GPU (different streams without ordering, several host
+ * threads) race on the tables and must be serialised by the caller.  Records whose index lies outside
+ * their chunk are skipped as in demo_decode_apply, but are not reported (there is no context to query).
+ *
+ * The first call on a device looks up the array's device address (a one-time set-up that should
+ * happen before any stream capture begins).  The 2-D and 1-D tensors run through the generic decode
+ * kernels.  Errors: INVALID_ARG, SHAPE, K, UNSUPPORTED, CUDA.
+ */
+#define DEMO_STATIC_MAX_TENSORS 256
+#define DEMO_STATIC_MAX_WORKERS 64
+#define DEMO_STATIC_MAX_CHUNK 64
+#define DEMO_STATIC_SCRATCH_BYTES (64 * 64 * 4 + 256 * 32 + 256 * 8 + 64 * 8 + 256)
+demo_status demo_decode_apply_static(const demo_config *cfg, const demo_tensor_desc *tensors, int32_t n_tensors,
+                                     const void *const *payloads, int32_t n_payloads, float *const *params,
+                                     int32_t cuda_device, void *cuda_stream);
+
 /* The learning rate is scheduled (eta_t in the update equation of Section 2.1): takes effect for
  * the next demo_decode_apply.  Errors: INVALID_ARG (null ctx, non-finite lr). */
 demo_status demo_set_lr(demo_ctx *ctx, float lr);

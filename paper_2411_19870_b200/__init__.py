@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     DemoTensorDesc,
     DemoTransform,
     RECORD_BYTES,
+    decode_apply_static,
     demo_status_string,
     load_library,
 )

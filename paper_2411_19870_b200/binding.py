@@ -20,7 +20,7 @@ RECORD_BYTES = 8
 
 EXPORTS = [
     "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
-    "demo_step_host", "demo_set_lr", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
 ]
 
@@ -70,6 +70,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_decode_apply.restype = i32
     lib.demo_step_host.argtypes = [vp, pvp, pvp, pvp, pvp, pvp, vp, vp]
     lib.demo_step_host.restype = i32
+    lib.demo_decode_apply_static.argtypes = [ctypes.POINTER(DemoConfig), ctypes.POINTER(DemoTensorDesc), i32, pvp, i32,
+                                             pvp, i32, vp]
+    lib.demo_decode_apply_static.restype = i32
     lib.demo_set_lr.argtypes = [vp, ctypes.c_float]
     lib.demo_set_lr.restype = i32
     lib.demo_set_path.argtypes = [vp, i32]
@@ -97,6 +100,25 @@ def _ptr_array(ptrs: Sequence[int]):
 
 def _tensor_ptrs(tensors) -> List[int]:
     return [int(t.data_ptr()) for t in tensors]
+
+
+def decode_apply_static(shapes, payloads, params, *, chunk: int, topk: int, lr: float, weight_decay: float,
+                        device: int = 0, stream=None) -> None:
+    """``demo_decode_apply_static``: decode + update without a context and without any allocation by
+    the library (its tables live in a fixed device array; see include/demo.h for the limits).
+    ``payloads`` / ``params`` are lists of device tensors."""
+    lib = load_library()
+    descs = (DemoTensorDesc * len(shapes))()
+    for d, s in zip(descs, shapes):
+        d.ndim = len(s)
+        for a in range(min(len(s), 2)):
+            d.shape[a] = int(s[a])
+    cfg = DemoConfig(0.0, chunk, topk, lr, weight_decay, len(payloads), DEMO_F32)
+    st = lib.demo_decode_apply_static(ctypes.byref(cfg), descs, len(shapes), _ptr_array(_tensor_ptrs(payloads)),
+                                      len(payloads), _ptr_array(_tensor_ptrs(params)), device,
+                                      DemoTransform._stream(stream))
+    if st != 0:
+        raise DemoError(st, "demo_decode_apply_static")
 
 
 class DemoTransform:

@@ -360,3 +360,188 @@ cudaError_t demo_launch_decode_generic(int s, int two_d, const DemoDecodeArgs &a
         default: return cudaErrorInvalidValue;
     }
 }
+
+// =================================================================================================
+// demo_decode_apply_static: the decode + update step for callers that must not allocate.
+//
+// The generic decode kernels above read four small tables from global memory besides the caller's
+// payloads and parameters: the DCT basis, the tensor table, the two pointer tables and a status
+// word.  A context built by demo_init gets them from cudaMalloc; this entry point keeps them in the
+// fixed array below instead, so it never allocates -- at the price of hard limits on the problem
+// size and of one array shared by every call in the process.
+// =================================================================================================
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/demo.h"
+
+namespace {
+
+constexpr int STATIC_MAX_TENSORS = DEMO_STATIC_MAX_TENSORS;
+constexpr int STATIC_MAX_WORKERS = DEMO_STATIC_MAX_WORKERS;
+constexpr int STATIC_MAX_CHUNK = DEMO_STATIC_MAX_CHUNK;
+
+// layout of the scratch array (byte offsets, all multiples of 256)
+constexpr size_t OFF_BASIS = 0;                                                                   // s*s floats
+constexpr size_t OFF_ENTRIES = OFF_BASIS + sizeof(float) * STATIC_MAX_CHUNK * STATIC_MAX_CHUNK;   // tensor table
+constexpr size_t OFF_XPTRS = OFF_ENTRIES + sizeof(DemoTensorEntry) * STATIC_MAX_TENSORS;          // float*[T]
+constexpr size_t OFF_PPTRS = OFF_XPTRS + sizeof(void *) * STATIC_MAX_TENSORS;                     // record*[W]
+constexpr size_t OFF_STATUS = OFF_PPTRS + sizeof(void *) * STATIC_MAX_WORKERS;                    // int
+constexpr size_t STATIC_SCRATCH_BYTES = OFF_STATUS + 256;
+
+static_assert(STATIC_SCRATCH_BYTES == DEMO_STATIC_SCRATCH_BYTES, "header and layout disagree");
+
+}  // namespace
+
+// Device-resident scratch.  In host code this name is only a handle for cudaGetSymbolAddress; the
+// device address is looked up once per device and passed to the kernels like any other pointer.
+static __device__ __align__(256) unsigned char demo_static_scratch[DEMO_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+unsigned char *g_static_base[STATIC_MAX_DEVICES];  // device address of the scratch, per device (0 = not set up)
+
+}  // namespace
+
+extern "C" demo_status demo_decode_apply_static(const demo_config *cfg, const demo_tensor_desc *tensors,
+                                                int32_t n_tensors, const void *const *payloads, int32_t n_payloads,
+                                                float *const *params, int32_t cuda_device, void *cuda_stream)
+{
+    if (!cfg || !tensors || !payloads || !params || n_tensors < 1 || cuda_device < 0) return DEMO_ERR_INVALID_ARG;
+    if (cuda_device >= STATIC_MAX_DEVICES) return DEMO_ERR_UNSUPPORTED;
+    if (n_payloads < 1 || n_payloads != cfg->num_workers) return DEMO_ERR_INVALID_ARG;
+    if (!std::isfinite(cfg->lr) || !std::isfinite(cfg->weight_decay)) return DEMO_ERR_INVALID_ARG;
+    const int s = cfg->chunk;
+    if (!(s == 8 || s == 16 || s == 32 || s == 64 || s == 128)) return DEMO_ERR_UNSUPPORTED;
+    // the fixed scratch bounds the problem: reject anything larger instead of overrunning it
+    if (s > STATIC_MAX_CHUNK || n_tensors > STATIC_MAX_TENSORS || n_payloads > STATIC_MAX_WORKERS)
+        return DEMO_ERR_UNSUPPORTED;
+    if (cfg->topk < 1 || (long long)cfg->topk > (long long)s * s) return DEMO_ERR_K;
+    for (int t = 0; t < n_tensors; ++t) {
+        const demo_tensor_desc &d = tensors[t];
+        if (d.ndim != 1 && d.ndim != 2) return DEMO_ERR_SHAPE;
+        for (int ax = 0; ax < d.ndim; ++ax)
+            if (d.shape[ax] < s || d.shape[ax] % s != 0 || d.shape[ax] > (1LL << 31) - 1) return DEMO_ERR_SHAPE;
+        if (!params[t] || (reinterpret_cast<uintptr_t>(params[t]) & 15u)) return DEMO_ERR_INVALID_ARG;
+    }
+    for (int w = 0; w < n_payloads; ++w)
+        if (!payloads[w] || (reinterpret_cast<uintptr_t>(payloads[w]) & 15u)) return DEMO_ERR_INVALID_ARG;
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    if (prev != cuda_device && cudaSetDevice(cuda_device) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    demo_status result = DEMO_OK;
+    do {
+        // one-time set-up per device, with that device current: translate the symbol into a device address
+        unsigned char *base = nullptr;
+        {
+            std::lock_guard<std::mutex> lock(g_static_mutex);
+            if (!g_static_base[cuda_device]) {
+                void *p = nullptr;
+                if (cudaGetSymbolAddress(&p, demo_static_scratch) != cudaSuccess || !p) {
+                    cudaGetLastError();
+                    result = DEMO_ERR_CUDA;
+                    break;
+                }
+                g_static_base[cuda_device] = static_cast<unsigned char *>(p);
+            }
+            base = g_static_base[cuda_device];
+        }
+        int sm_count = 0;
+        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, cuda_device) != cudaSuccess) {
+            result = DEMO_ERR_CUDA;
+            break;
+        }
+
+        // host-side images of the tables (fixed-size, on the stack / in static storage: no heap)
+        static thread_local float h_basis[STATIC_MAX_CHUNK * STATIC_MAX_CHUNK];
+        DemoTensorEntry h_entries[STATIC_MAX_TENSORS];  // 2-D tensors first, then 1-D tensors
+        int n2d = 0, n1d = 0;
+        long long chunks2d = 0, chunks1d = 0;
+        {
+            const double pi = 3.141592653589793238462643383279502884;
+            for (int u = 0; u < s; ++u)
+                for (int n = 0; n < s; ++n) {
+                    const double au = (u == 0) ? std::sqrt(1.0 / s) : std::sqrt(2.0 / s);
+                    h_basis[(size_t)u * s + n] = (float)(au * std::cos(pi * (2.0 * n + 1.0) * u / (2.0 * s)));
+                }
+            for (int t = 0; t < n_tensors; ++t) n2d += tensors[t].ndim == 2;
+            int i2 = 0, i1 = n2d;
+            long long rec = 0;
+            for (int t = 0; t < n_tensors; ++t) {
+                const demo_tensor_desc &d = tensors[t];
+                const bool two = d.ndim == 2;
+                const long long n1 = two ? d.shape[1] : d.shape[0];
+                const long long c0 = two ? d.shape[0] / s : 1, c1 = n1 / s;
+                const long long M = two ? (long long)s * s : s;
+                DemoTensorEntry e;
+                e.tensor = t;
+                e.n1 = (int)n1;
+                e.c1 = (int)c1;
+                e.k_eff = (int)(cfg->topk < M ? cfg->topk : M);
+                e.rec_begin = rec;
+                e.chunk_begin = two ? chunks2d : chunks1d;
+                (two ? chunks2d : chunks1d) += c0 * c1;
+                h_entries[two ? i2++ : i1++] = e;
+                rec += c0 * c1 * e.k_eff;
+            }
+            n1d = n_tensors - n2d;
+        }
+
+        bool ok = true;
+        ok = ok && cudaMemcpyAsync(base + OFF_BASIS, h_basis, sizeof(float) * (size_t)s * s, cudaMemcpyHostToDevice,
+                                   stream) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(base + OFF_ENTRIES, h_entries, sizeof(DemoTensorEntry) * (size_t)n_tensors,
+                                   cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(base + OFF_XPTRS, params, sizeof(void *) * (size_t)n_tensors, cudaMemcpyHostToDevice,
+                                   stream) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(base + OFF_PPTRS, payloads, sizeof(void *) * (size_t)n_payloads,
+                                   cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        // the array keeps the previous call's contents: the status word must start at zero
+        ok = ok && cudaMemsetAsync(base + OFF_STATUS, 0, sizeof(int), stream) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            result = DEMO_ERR_CUDA;
+            break;
+        }
+
+        DemoDecodeArgs a;
+        a.payloads = reinterpret_cast<const DemoRecord *const *>(base + OFF_PPTRS);
+        a.W = n_payloads;
+        a.x_ptrs = reinterpret_cast<float *const *>(base + OFF_XPTRS);
+        a.C = reinterpret_cast<const float *>(base + OFF_BASIS);
+        a.lr = cfg->lr;
+        a.wd = cfg->weight_decay;
+        a.status = reinterpret_cast<int *>(base + OFF_STATUS);
+        a.tmap_x = nullptr;
+        cudaError_t err = cudaSuccess;
+        if (n2d) {
+            a.entries = reinterpret_cast<const DemoTensorEntry *>(base + OFF_ENTRIES);
+            a.n_entries = n2d;
+            a.n_chunks = chunks2d;
+            err = demo_launch_decode_generic(s, 1, a, sm_count, stream);
+        }
+        if (err == cudaSuccess && n1d) {
+            a.entries = reinterpret_cast<const DemoTensorEntry *>(base + OFF_ENTRIES) + n2d;
+            a.n_entries = n1d;
+            a.n_chunks = chunks1d;
+            err = demo_launch_decode_generic(s, 0, a, sm_count, stream);
+        }
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            result = DEMO_ERR_CUDA;
+        }
+    } while (false);
+    if (prev >= 0 && prev != cuda_device) cudaSetDevice(prev);
+    return result;
+}
