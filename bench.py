@@ -224,16 +224,12 @@ def run_ours(args, rank, world):
     barrier()
     clocks = sampler.stop()
     launches = tr.launch_count - launches0
-    ms_total = t_start.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(t_start.elapsed_time(t_end), dist, dev)
     ms_step = ms_total / args.steps
     assert tr.device_status() == 0
 
     P = wl.n_params
-    value = world * P / (ms_step * 1e-3)
+    value = replica_throughput(P, world, ms_step)
     core_bytes, payload_bytes = algorithmic_bytes(wl, gbytes)
     peak, peak_src = _peaks()
     c_ms = [a.elapsed_time(b) for a, b in events["compress"]]
@@ -323,18 +319,25 @@ def run_e2e(torch, tr, wl, grads, mom, payloads, params, dev, world, dist, gbyte
         tr.step_host(host, grads, mom, payloads, params, out)
     e1.record()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return {"value": world * P / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+    ms = max_over_ranks(e0.elapsed_time(e1) / steps, dist, dev)
+    return {"value": replica_throughput(P, world, ms), "unit": UNIT, "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": W * P * gbytes, "d2h_bytes_per_step": W * tr.payload_bytes, "note": note}
 
 
-def aggregate_replicas(ms_per_rank, units_per_rank):
-    """Whole-job throughput of independent replicas: all units over the slowest rank's time."""
-    return sum(units_per_rank) / (max(ms_per_rank) * 1e-3)
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Device time of the slowest rank (identity when there is one process)."""
+    if dist is None:
+        return float(ms)
+    import torch
+
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(units_per_rank: float, world: int, ms: float) -> float:
+    """Whole-job throughput of `world` independent replicas: all units over the slowest rank's time."""
+    return world * units_per_rank / (ms * 1e-3)
 
 
 def main():
