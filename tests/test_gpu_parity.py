@@ -219,3 +219,50 @@ def test_step_host_matches_separate_calls():
     assert all(torch.equal(a, b) for a, b in zip(pay2, r.payloads))
     assert torch.equal(out.view(wl.num_workers, -1)[1], r.payloads[1].cpu())
     r.close()
+
+
+@pytest.mark.parametrize("k", [32, 128])
+def test_decode_fan_in_64_workers(k):
+    """Config 5's W=64 cell on the 4096 x 4096 matrix: one step from zero momentum (m = g), every
+    worker compressed into its own payload, decode of 64 payloads checked on sampled chunks."""
+    wl = inputs.stress(chunk=64, topk=k, num_workers=64, full_set=False)
+    r = parity.Runner(wl, max_chunks=64, seed=k)
+    r.step()
+    assert r.report["decode_chunks"] == 64
+    r.close()
+
+
+def _free_gb():
+    free, _ = torch.cuda.mem_get_info()
+    return free / 1e9
+
+
+def test_decoder_300m_full_size_sampled():
+    """Config 3 at full size (217 tensors, P = 454 M, W = 8) in the launch configuration the benchmark
+    times; 12 sampled chunks per tensor and worker (first, last, 10 random), all chunks of 1-D tensors
+    up to that count, plus the whole-tensor record invariants."""
+    wl = inputs.decoder_300m()
+    if _free_gb() < 30:
+        pytest.skip("not enough free device memory")
+    r = parity.Runner(wl, max_chunks=12)
+    r.step()
+    r.step()
+    rec = r.payloads[3].view(torch.int32).view(-1, 2)
+    assert rec.shape[0] == wl.records_per_worker()
+    first, n_chunks, k_eff = r.layout[len(wl.shapes) - 1]  # the embedding, the largest tensor
+    idx = rec[first:first + n_chunks * k_eff, 0].view(n_chunks, k_eff)
+    assert idx.min().item() >= 0 and idx.max().item() < 4096 and torch.all(idx[:, 1:] > idx[:, :-1])
+    r.close()
+
+
+def test_decoder_1b_full_size_sampled():
+    """Config 4 at full size (146 tensors, P = 1.28 G, W = 16): the benchmark's workload and launch
+    configuration, 6 sampled chunks per tensor and worker."""
+    wl = inputs.decoder_1b()
+    if _free_gb() < 110:
+        pytest.skip("not enough free device memory")
+    r = parity.Runner(wl, max_chunks=6)
+    r.step()
+    assert r.report["chunks"] == 16 * 146 * 6
+    r.close()
+    torch.cuda.empty_cache()
