@@ -163,6 +163,9 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
         if (d.ndim != 1 && d.ndim != 2) return DEMO_ERR_SHAPE;
         for (int a = 0; a < d.ndim; ++a)
             if (d.shape[a] < s || d.shape[a] % s != 0 || d.shape[a] > (1LL << 31) - 1) return DEMO_ERR_SHAPE;
+        // the kernels index the chunks of one tensor with 31 bits
+        const long long n_ch = (d.shape[0] / s) * (d.ndim == 2 ? d.shape[1] / s : 1);
+        if (n_ch > (1LL << 31) - 1) return DEMO_ERR_UNSUPPORTED;
     }
 
     int n_dev = 0;

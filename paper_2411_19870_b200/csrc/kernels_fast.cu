@@ -167,12 +167,14 @@ __device__ __forceinline__ void radix_select_tile(const float *X, int k_eff, uns
         s_state[0] = 0u;
         s_state[1] = (unsigned)k_eff;
     }
+#pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
         const int shift = 24 - 8 * pass;
         const unsigned mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
         for (int i = t; i < 256; i += S) hist[i] = 0u;
         sb.sync();
         const unsigned prefix = s_state[0];
+#pragma unroll 1
         for (int v = 0; v < S; ++v) {
             const unsigned key = mag_key(X[t * XS + v]);
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
@@ -297,9 +299,10 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             m_ptr = a.m_ptrs[cached_tensor];
             g_ptr = reinterpret_cast<const GT *>(a.g_ptrs[cached_tensor]);
         }
-        const long long lc = c - cur.te.chunk_begin;
-        const long long k0 = lc / cur.te.c1;
-        const int k1 = (int)(lc - k0 * cur.te.c1);
+        // chunks per tensor fit 31 bits (checked at init): 32-bit division
+        const unsigned lc = (unsigned)(c - cur.te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)cur.te.c1;
+        const int k1 = (int)(lc - k0 * (unsigned)cur.te.c1);
         TileRef r;
         r.tm_m = r.tm_g = nullptr;
         r.x = k1 * S;
@@ -342,14 +345,16 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
     }
 
     for (long long cb = (long long)blockIdx.x * NCH; cb < a.n_chunks; cb += stride, c += stride) {
-        // all slots of the CTA start a chunk together; a slot whose wait expired takes the CTA down
+        // all slots of the CTA start a chunk together; a slot whose wait expired takes the CTA down.
+        // (Running the two halves of the slots half a chunk apart, or smaller CTAs, was measured
+        // slower: the second instruction stream costs more than the overlap of phases gains.)
         if (__syncthreads_or(failed)) return;
         if (c >= a.n_chunks) continue;
         // the cursor points at chunk c (issue_loads(c) ran last)
         const DemoTensorEntry te = cur.te;
-        const long long lc = c - te.chunk_begin;
-        const long long k0 = lc / te.c1;
-        const int k1 = (int)(lc - k0 * te.c1);
+        const unsigned lc = (unsigned)(c - te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)te.c1;
+        const int k1 = (int)(lc - k0 * (unsigned)te.c1);
         const size_t base = (size_t)k0 * S * (size_t)te.n1 + (size_t)k1 * S;
         float *__restrict__ m = m_ptr;
         const int k_eff = te.k_eff;
@@ -528,7 +533,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                 if (total != (unsigned)k_eff) {  // block-uniform: equal magnitudes straddle the threshold
                     sb.sync();
 #pragma unroll
-                    for (int it = 0; it < ITER; ++it) {
+                    for (int it = 0; it < ITER; ++it) {  // (rare path: inner loops stay rolled)
                         const unsigned li = it * 32 + lane;
                         sel[it] = false;
                         if (li < n_cw) {
@@ -536,6 +541,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                             unsigned rank = 0;
 #pragma unroll
                             for (int w = 0; w < NW; ++w)
+#pragma unroll 1
                                 for (unsigned c2 = 0; c2 < n_w[w]; ++c2) {
                                     const unsigned k2 = cand_key[w * CAPWP + c2];
                                     const bool earlier = (w < warp) || (w == warp && c2 < li);
@@ -572,6 +578,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             unsigned thr, need_eq;
             radix_select_tile<S>(X, k_eff, hist, misc, &thr, &need_eq, t, sb);
             unsigned gt = 0, eq = 0;
+#pragma unroll 1
             for (int v = 0; v < S; ++v) {
                 const unsigned key = mag_key(X[t * XS + v]);
                 gt += key > thr;
@@ -587,6 +594,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             for (int w = 0; w < NW; ++w)
                 if (w < warp) before += misc[w];
             unsigned gb = before & 0xffffu, eb = before >> 16;
+#pragma unroll 1
             for (int v = 0; v < S; ++v) {
                 const float val = X[t * XS + v];
                 const unsigned key = mag_key(val);
@@ -747,9 +755,9 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
             cached_tensor = te.tensor;
             x_ptr = a.x_ptrs[cached_tensor];
         }
-        const long long lc = c - te.chunk_begin;
-        const long long k0 = lc / te.c1;
-        const int k1 = (int)(lc - k0 * te.c1);
+        const unsigned lc = (unsigned)(c - te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)te.c1;
+        const int k1 = (int)(lc - k0 * (unsigned)te.c1);
         const size_t base = (size_t)k0 * S * (size_t)te.n1 + (size_t)k1 * S;
         float *__restrict__ x = x_ptr;
         const int k_eff = te.k_eff;
