@@ -340,6 +340,57 @@ def replica_throughput(units_per_rank: float, world: int, ms: float) -> float:
     return world * units_per_rank / (ms * 1e-3)
 
 
+def run_grid(args):
+    """Ablation grid of the stress configuration (heavy-tailed gradients with tie-maker chunks):
+    chunk s x k x fan-in W, ms per optimizer step, one JSON line per cell.  The 4096 x 4096 matrix runs
+    every cell; `--grid-set` adds the 1B-class set for the cells that fit in memory (W <= 16)."""
+    import torch
+
+    import paper_2411_19870_b200 as demo
+    from paper_2411_19870_b200 import inputs
+
+    dev = torch.device("cuda", 0)
+    for full in ([False, True] if args.grid_set else [False]):
+        for s in (32, 64, 128):
+            for k in (1, 8, 32, 128):
+                for W in (1, 8, 64):
+                    if full and W > 16:
+                        continue  # 64 momentum sets of the 1B-class set do not fit in 180 GB
+                    wl = inputs.stress(chunk=s, topk=k, num_workers=W, full_set=full)
+                    tr = demo.DemoTransform(wl.shapes, chunk=s, topk=k, beta=wl.beta, lr=wl.lr,
+                                            weight_decay=wl.weight_decay, num_workers=W)
+                    params = inputs.make_params(wl, dev)
+                    mom = [inputs.make_momentum(wl, dev) for _ in range(W)]
+                    grads = [inputs.GradStream(wl, w, dev).next() for w in range(W)]
+                    payloads = [torch.empty(tr.payload_bytes, dtype=torch.uint8, device=dev) for _ in range(W)]
+
+                    def step():
+                        for w in range(W):
+                            tr.compress(w, grads[w], mom[w], payloads[w])
+                        tr.decode_apply(payloads, params)
+
+                    for _ in range(3):
+                        step()
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    n = 5
+                    e0.record()
+                    for _ in range(n):
+                        step()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    ms = e0.elapsed_time(e1) / n
+                    assert tr.device_status() == 0
+                    core, _ = algorithmic_bytes(wl, 2)
+                    print(json.dumps({"workload": wl.name, "n_params": wl.n_params, "chunk": s, "topk": k,
+                                      "num_workers": W, "ms_per_step": ms, "params_per_s": wl.n_params / (ms * 1e-3),
+                                      "algorithmic_GBps": core / (ms * 1e-3) / 1e9,
+                                      "kernels": "fast" if s in (32, 64) else "generic"}), flush=True)
+                    tr.close()
+                    del params, mom, grads, payloads
+                    torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -351,12 +402,17 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--grid", action="store_true", help="print the stress/ablation grid instead of the benchmark line")
+    ap.add_argument("--grid-set", action="store_true", help="with --grid: also run the 1B-class set")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = max(args.warmup, 1)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
+    if args.grid:
+        if rank == 0:
+            run_grid(args)
+    elif args.impl == "reference":
         run_reference(args, rank)
     else:
         run_ours(args, rank, world)
