@@ -357,7 +357,7 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
-        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s))
+        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s) && (s != 128 || ctx->encode))
             err = demo_launch_compress_fast(s, a, ctx->sm_count, stream);
         else
             err = demo_launch_compress_generic(s, 1, a, ctx->sm_count, stream);
@@ -421,7 +421,7 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
-        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s))
+        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s) && (s != 128 || ctx->encode))
             err = demo_launch_decode_fast(s, a, ctx->sm_count, stream);
         else
             err = demo_launch_decode_generic(s, 1, a, ctx->sm_count, stream);

@@ -19,81 +19,14 @@
 #include <cuda_bf16.h>
 
 #include "demo_internal.h"
+#include "fast_common.cuh"
 #include "fast_dct.cuh"
 
 namespace {
 
+using namespace fastk;
+
 constexpr int CAP = 128;                          // candidate capacity of the fast top-k
-constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;  // ~1 s
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within WAIT_LIMIT_CYCLES.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
-    }
-    return true;
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// 1-D bulk async copy global -> shared (16-byte aligned addresses, size a multiple of 16).
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, unsigned bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
-// 2-D tiled TMA load of one box (coordinates in elements: x along the row, y the row index).
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(tmap), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-// Pull one box into L2 ahead of its use.
-__device__ __forceinline__ void tma_prefetch_2d(const void *tmap, int x, int y)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
-}
-constexpr int TMAP_BYTES = 128;  // sizeof(CUtensorMap)
-
-__device__ __forceinline__ float to_f32(float v) { return v; }
-__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
-// max of three (one instruction on sm_100)
-__device__ __forceinline__ float max3f(float a, float b, float c)
-{
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float max3abs(float a, float b, float c) { return max3f(fabsf(a), fabsf(b), fabsf(c)); }
-__device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
-
 // A CTA hosts NCH independent "slots" of S threads, one chunk each.  Threads of a slot meet at the
 // slot's own named barrier (a warp-level barrier when the slot is a single warp); all slots meet once
 // per chunk at the CTA barrier, which keeps the warps of the CTA in the same region of the (large,
@@ -130,28 +63,6 @@ struct Cfg {
                                       // column access and 128-bit row access
     static constexpr int NW = S / 32;
     static constexpr int LOG2S = (S == 64) ? 6 : 5;
-};
-
-// Walks the tensor table as the CTA's chunk ids grow.
-struct EntryCursor {
-    int e = 0;
-    DemoTensorEntry te;
-    bool loaded = false;
-    __device__ __forceinline__ void seek(const DemoTensorEntry *entries, int n, long long c)
-    {
-        if (!loaded) {
-            e = demo_find_entry(entries, n, c);
-            te = entries[e];
-            loaded = true;
-            return;
-        }
-        bool moved = false;
-        while (e + 1 < n && entries[e + 1].chunk_begin <= c) {
-            ++e;
-            moved = true;
-        }
-        if (moved) te = entries[e];
-    }
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -208,17 +119,6 @@ __device__ __forceinline__ void radix_select_tile(const float *X, int k_eff, uns
     }
     *thr = s_state[0];
     *need_eq = s_state[1];
-}
-
-// Inclusive warp scan.
-__device__ __forceinline__ unsigned warp_inclusive_scan(unsigned v, int lane)
-{
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        unsigned n = __shfl_up_sync(0xffffffffu, v, d);
-        if (lane >= d) v += n;
-    }
-    return v;
 }
 
 // Bytes of the tile area of the compress kernel: the staged m and g tiles, or the padded transpose
@@ -911,10 +811,11 @@ cudaError_t launch_decode(const DemoDecodeArgs &a, int sm_count, cudaStream_t st
 
 }  // namespace
 
-bool demo_fast_supported(int s) { return s == 64 || s == 32; }
+bool demo_fast_supported(int s) { return s == 128 || s == 64 || s == 32; }
 
 cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
 {
+    if (s == 128) return demo_launch_compress_fast128(a, sm_count, stream);
     if (s == 64)
         return a.grad_bf16 ? launch_compress<64, __nv_bfloat16>(a, sm_count, stream)
                            : launch_compress<64, float>(a, sm_count, stream);
@@ -926,6 +827,7 @@ cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_c
 
 cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
 {
+    if (s == 128) return demo_launch_decode_fast128(a, sm_count, stream);
     if (s == 64) return launch_decode<64>(a, sm_count, stream);
     if (s == 32) return launch_decode<32>(a, sm_count, stream);
     return cudaErrorInvalidValue;

@@ -1,0 +1,475 @@
+// Fast kernels for 2-D tensors with chunk size 128: one 256-thread CTA per 128 x 128 chunk.
+//
+// A 128-point transform does not fit one thread's registers, so it is split by the first stage of the
+// same factorisation the 64-point code uses (fast_dct.cuh):
+//     DCT-II_128:  u[n] = x[n] + x[127-n],  v[n] = x[n] - x[127-n]   (n < 64)
+//                  X[2p] = DCT-II_64(u)[p],  X[2p+1] = DCT-IV_64(v)[p]
+// Thread (h, j) = (threadIdx.x / 128, threadIdx.x % 128) owns line j (a column in the first pass, a row
+// in the second) and computes its even (h = 0) or odd (h = 1) outputs; h is warp-uniform, so the two
+// transform bodies never diverge inside a warp.  The inverse runs the transposed graph:
+//     e = DCT-III_64(X[even]),  o = DCT-IV_64(X[odd]),  x[n] = e[n] + o[n],  x[127-n] = e[n] - o[n]
+// with e and o exchanged between the two threads of a line through shared memory.
+//
+// compress: TMA-staged m and g tiles -> B = beta*m + g -> column pass -> row pass -> coefficients in
+// shared memory -> exact radix select (4 x 8 bits on the magnitude) + index-ordered compaction ->
+// records; sparse row stage of the inverse from the records, fast column stage, m and g fetched again
+// (L2) for the residual m <- B - IDCT(kept).  decode: scatter-add of the W payloads in worker order,
+// two inverse passes, sign, update; the x tile is staged into the (then dead) coefficient tile.
+// Tiles need the TMA tensor maps; without them the host uses the generic kernels for s = 128.
+#include <cuda_bf16.h>
+
+#include "demo_internal.h"
+#include "fast_common.cuh"
+#include "fast_dct.cuh"
+
+namespace {
+
+using namespace fastk;
+
+constexpr int S = 128, H = 64, XS = S + 4, M = S * S, THREADS = 256;
+using SC = fdct::ScaleOrtho<S>;
+
+__device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned *warp_tot /*[8]*/)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned inc = warp_inclusive_scan(v, lane);
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    unsigned base = 0;
+    for (int w = 0; w < warp; ++w) base += warp_tot[w];
+    __syncthreads();
+    return base + inc - v;
+}
+
+// Forward half-transform of one line: in[n] = x[n] (+/-) x[127-n] already formed; out[p] is
+// coefficient 2p (h = 0) or 2p+1 (h = 1) of the orthonormal 128-point DCT-II.
+__device__ __forceinline__ void forward_half(int h, float (&in)[H], float (&out)[H])
+{
+    if (h == 0) {
+        fdct::dct2<H, SC>(in, out);
+        out[0] *= fdct::dc_scale<S>();
+    } else {
+        fdct::dct4<H, SC>(in, out);
+    }
+}
+// Inverse half-transform: in[p] = coefficient 2p (h = 0) or 2p+1 (h = 1); out = e (h = 0) or o (h = 1).
+__device__ __forceinline__ void inverse_half(int h, float (&in)[H], float (&out)[H])
+{
+    if (h == 0) {
+        in[0] *= fdct::dc_scale<S>();
+        fdct::dct3<H, SC>(in, out);
+    } else {
+        fdct::dct4<H, SC>(in, out);
+    }
+}
+
+template <typename GT>
+constexpr size_t compress128_tile_bytes()
+{
+    return (size_t)M * (sizeof(float) + sizeof(GT)) > (size_t)S * XS * 4 ? (size_t)M * (sizeof(float) + sizeof(GT))
+                                                                         : (size_t)S * XS * 4;
+}
+template <typename GT>
+constexpr size_t compress128_smem()
+{
+    return compress128_tile_bytes<GT>() + (256 + 8 + 4) * 4 + 128 * 16 + 16;
+}
+
+template <typename GT>
+__global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompressArgs a)
+{
+    constexpr unsigned TILE_BYTES = M * sizeof(float) + M * sizeof(GT);
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float *Ms = reinterpret_cast<float *>(smem_raw);  // [128*128] m tile
+    GT *Gs = reinterpret_cast<GT *>(Ms + M);          // [128*128] g tile
+    float *X = Ms;                                    // [128*132] transpose / coefficients / row stage (aliases the tiles)
+    unsigned *hist = reinterpret_cast<unsigned *>(smem_raw + compress128_tile_bytes<GT>());  // [256]
+    unsigned *warp_tot = hist + 256;                                                         // [8]
+    unsigned *s_state = warp_tot + 8;                                                        // [4]
+    int4 *recs4 = reinterpret_cast<int4 *>(s_state + 4);                                     // [128]
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(recs4 + 128);
+
+    const int tid = threadIdx.x, h = tid >> 7, j = tid & 127;
+    const uint32_t bar = smem_u32(bar_mem);
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        fence_proxy_async();
+    }
+    __syncthreads();
+    fence_proxy_async();
+
+    EntryCursor cur;
+    unsigned phase = 0;
+
+    auto issue_tiles = [&](const DemoTensorEntry &te, long long c) {
+        const unsigned lc = (unsigned)(c - te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)te.c1, k1 = lc - k0 * (unsigned)te.c1;
+        if (tid == 0) {
+            mbar_expect_tx(bar, TILE_BYTES);
+            tma_load_2d(smem_u32(Ms), static_cast<const char *>(a.tmap_m) + (size_t)te.tensor * TMAP_BYTES, k1 * S, k0 * S, bar);
+            tma_load_2d(smem_u32(Gs), static_cast<const char *>(a.tmap_g) + (size_t)te.tensor * TMAP_BYTES, k1 * S, k0 * S, bar);
+        }
+    };
+
+    long long c = blockIdx.x;
+    if (c < a.n_chunks) {
+        cur.seek(a.entries, a.n_entries, c);
+        issue_tiles(cur.te, c);
+    }
+    for (; c < a.n_chunks; c += gridDim.x) {
+        const DemoTensorEntry te = cur.te;  // the cursor points at chunk c
+        const unsigned lc = (unsigned)(c - te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)te.c1, k1 = lc - k0 * (unsigned)te.c1;
+        const size_t base = (size_t)k0 * S * (size_t)te.n1 + (size_t)k1 * S;
+        float *__restrict__ m = a.m_ptrs[te.tensor];
+        const int k_eff = te.k_eff;
+        DemoRecord *rec = a.payload + te.rec_begin + (long long)lc * k_eff;
+
+        bool arrived = mbar_wait_bounded(bar, phase);
+        phase ^= 1u;
+        if (!__syncthreads_and(arrived)) {
+            if (tid == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
+            mbar_wait_bounded(bar, phase ^ 1u);
+            return;
+        }
+
+        // ---- two forward passes through one rolled copy of the half-transforms ---------------------
+        float in[H], out[H];
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            if (pass == 0) {
+                // column j of B = beta*m + g, folded: in[n] = B[n][j] +/- B[127-n][j]
+#pragma unroll
+                for (int n = 0; n < H; ++n) {
+                    const float lo = fmaf(a.beta, Ms[n * S + j], to_f32(Gs[n * S + j]));
+                    const float hi = fmaf(a.beta, Ms[(S - 1 - n) * S + j], to_f32(Gs[(S - 1 - n) * S + j]));
+                    in[n] = h ? lo - hi : lo + hi;
+                }
+                __syncthreads();  // the staged tiles are consumed (X aliases them)
+            } else {
+                // row j of the column-transformed tile, folded
+                const float4 *row = reinterpret_cast<const float4 *>(X + j * XS);
+#pragma unroll
+                for (int n4 = 0; n4 < H / 4; ++n4) {
+                    const float4 lo = row[n4];
+                    const float4 hi = row[S / 4 - 1 - n4];  // elements 127-4n4-3 .. 127-4n4
+                    in[4 * n4 + 0] = h ? lo.x - hi.w : lo.x + hi.w;
+                    in[4 * n4 + 1] = h ? lo.y - hi.z : lo.y + hi.z;
+                    in[4 * n4 + 2] = h ? lo.z - hi.y : lo.z + hi.y;
+                    in[4 * n4 + 3] = h ? lo.w - hi.x : lo.w + hi.x;
+                }
+                __syncthreads();  // every thread has read its row before the coefficients overwrite the tile
+            }
+            forward_half(h, in, out);
+            if (pass == 0) {
+#pragma unroll
+                for (int p = 0; p < H; ++p) X[(2 * p + h) * XS + j] = out[p];  // Y[u][j]
+            } else {
+#pragma unroll
+                for (int p = 0; p < H; ++p) X[j * XS + 2 * p + h] = out[p];    // Q[j][v]
+            }
+            __syncthreads();
+        }
+
+        // ---- exact top-k: radix select on the magnitude bits, then index-ordered compaction --------
+        unsigned thr, need_eq;
+        {
+            if (tid == 0) {
+                s_state[0] = 0u;
+                s_state[1] = (unsigned)k_eff;
+            }
+            // thread tid scans the half row [tid/2][64*(tid&1) .. +64): flat indices 64*tid .. 64*tid+63
+            const float *mine = X + (tid >> 1) * XS + 64 * (tid & 1);
+#pragma unroll 1
+            for (int pass = 0; pass < 4; ++pass) {
+                const int shift = 24 - 8 * pass;
+                const unsigned mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
+                hist[tid] = 0u;
+                __syncthreads();
+                const unsigned prefix = s_state[0];
+#pragma unroll 4
+                for (int e = 0; e < 64; ++e) {
+                    const unsigned key = mag_key(mine[e]);
+                    if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+                }
+                __syncthreads();
+                if (tid < 32) {
+                    const unsigned rem = s_state[1];
+                    unsigned local = 0;
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) local += hist[255 - 8 * tid - b];
+                    const unsigned inc = warp_inclusive_scan(local, tid);
+                    const unsigned before = inc - local;
+                    if (before < rem && rem <= inc) {
+                        unsigned cum = before;
+                        int b = 255 - 8 * tid;
+                        for (int q = 0; q < 8; ++q, --b) {
+                            const unsigned hh = hist[b];
+                            if (cum + hh >= rem) break;
+                            cum += hh;
+                        }
+                        s_state[1] = rem - cum;
+                        s_state[0] = prefix | ((unsigned)b << shift);
+                    }
+                }
+                __syncthreads();
+            }
+            thr = s_state[0];
+            need_eq = s_state[1];
+            unsigned gt = 0, eq = 0;
+#pragma unroll 4
+            for (int e = 0; e < 64; ++e) {
+                const unsigned key = mag_key(mine[e]);
+                gt += key > thr;
+                eq += key == thr;
+            }
+            const unsigned before = block_exclusive_scan(gt | (eq << 16), warp_tot);
+            unsigned gb = before & 0xffffu, eb = before >> 16;
+#pragma unroll 1
+            for (int e = 0; e < 64; ++e) {
+                const float val = mine[e];
+                const unsigned key = mag_key(val);
+                bool sel = false;
+                unsigned pos = 0;
+                if (key > thr) {
+                    pos = gb + min(eb, need_eq);
+                    ++gb;
+                    sel = true;
+                } else if (key == thr) {
+                    if (eb < need_eq) {
+                        pos = gb + eb;
+                        sel = true;
+                    }
+                    ++eb;
+                }
+                if (sel) {
+                    const int idx = 64 * tid + e;
+                    DemoRecord r;
+                    r.idx = idx;
+                    r.val = val;
+                    rec[pos] = r;
+                    if (k_eff <= 128) recs4[pos] = make_int4((idx >> 7) * XS, (idx & 127) * S, __float_as_int(val), 0);
+                }
+            }
+        }
+        __syncthreads();  // records complete; the coefficient tile is dead
+
+        // ---- residual: sparse row stage T[u][j] = sum over kept (u, v) of val * C[v][j] ------------
+        for (int i = tid; i < S * XS / 4; i += THREADS) reinterpret_cast<float4 *>(X)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncthreads();
+        if (h == 0) {
+            const float *Cj = a.C + j;
+            float acc = 0.f;
+            int cur_u = -1;
+            for (int r = 0; r < k_eff; ++r) {
+                int uo, vo;
+                float val;
+                if (k_eff <= 128) {
+                    const int4 rc = recs4[r];
+                    uo = rc.x;
+                    vo = rc.y;
+                    val = __int_as_float(rc.z);
+                } else {
+                    const DemoRecord rc = rec[r];
+                    uo = (rc.idx >> 7) * XS;
+                    vo = (rc.idx & 127) * S;
+                    val = rc.val;
+                }
+                if (uo != cur_u) {
+                    if (cur_u >= 0) X[cur_u + j] = acc;
+                    acc = 0.f;
+                    cur_u = uo;
+                }
+                acc = fmaf(val, __ldg(Cj + vo), acc);
+            }
+            if (cur_u >= 0) X[cur_u + j] = acc;
+        }
+        __syncthreads();
+
+        // ---- column stage of the inverse (split), second fetch of the tiles, residual --------------
+#pragma unroll
+        for (int p = 0; p < H; ++p) in[p] = X[(2 * p + h) * XS + j];
+        fence_proxy_async();
+        __syncthreads();  // T is in registers: the tile area is free
+        inverse_half(h, in, out);
+        // exchange e and o through the tile area (the staged tiles would overlap it, so they are
+        // fetched again only after the exchange)
+        float *Ex = X;  // [2][64][128]
+#pragma unroll
+        for (int n = 0; n < H; ++n) Ex[(h * H + n) * S + j] = out[n];
+        __syncthreads();
+#pragma unroll
+        for (int n = 0; n < H; ++n) {
+            const float other = Ex[((h ^ 1) * H + n) * S + j];
+            out[n] = h ? other - out[n] : out[n] + other;  // h=0: x[n] = e+o;  h=1: x[127-n] = e-o
+        }
+        fence_proxy_async();
+        __syncthreads();
+        issue_tiles(te, c);
+        arrived = mbar_wait_bounded(bar, phase);
+        phase ^= 1u;
+        if (!__syncthreads_and(arrived)) {
+            if (tid == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
+            mbar_wait_bounded(bar, phase ^ 1u);
+            return;
+        }
+#pragma unroll
+        for (int n = 0; n < H; ++n) {
+            const int row = h ? (S - 1 - n) : n;
+            m[base + (size_t)row * te.n1 + j] = fmaf(a.beta, Ms[row * S + j], to_f32(Gs[row * S + j])) - out[n];
+        }
+        fence_proxy_async();
+        __syncthreads();
+        const long long nc = c + gridDim.x;
+        if (nc < a.n_chunks) {
+            cur.seek(a.entries, a.n_entries, nc);
+            issue_tiles(cur.te, nc);
+        }
+    }
+}
+
+constexpr size_t decode128_smem() { return (size_t)S * XS * 4 + 16; }
+
+__global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float *St = reinterpret_cast<float *>(smem_raw);  // [128*132] aggregate / intermediate; later the x tile [128*128]
+    float *Xt = St;
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XS);
+
+    const int tid = threadIdx.x, h = tid >> 7, j = tid & 127;
+    const uint32_t bar = smem_u32(bar_mem);
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        fence_proxy_async();
+    }
+    __syncthreads();
+    fence_proxy_async();
+
+    EntryCursor cur;
+    unsigned phase = 0;
+    const unsigned lr_bits = __float_as_uint(a.lr);
+    const float decay = 1.f - a.lr * a.wd;
+
+    for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
+        cur.seek(a.entries, a.n_entries, c);
+        const DemoTensorEntry te = cur.te;
+        const unsigned lc = (unsigned)(c - te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)te.c1, k1 = lc - k0 * (unsigned)te.c1;
+        const size_t base = (size_t)k0 * S * (size_t)te.n1 + (size_t)k1 * S;
+        float *__restrict__ x = a.x_ptrs[te.tensor];
+        const int k_eff = te.k_eff;
+        const long long rec_off = te.rec_begin + (long long)lc * k_eff;
+        const char *tm_x = static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES;
+        if (tid == 0) tma_prefetch_2d(tm_x, k1 * S, k0 * S);
+
+        for (int i = tid; i < S * XS / 4; i += THREADS) reinterpret_cast<float4 *>(St)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncthreads();
+        // S = sum over workers in worker order (a barrier per worker fixes the order of additions)
+        for (int kb = 0; kb < k_eff; kb += THREADS) {
+            const bool mine = kb + tid < k_eff;
+            for (int w0 = 0; w0 < a.W; w0 += 8) {
+                DemoRecord r[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (mine && w0 + q < a.W) r[q] = a.payloads[w0 + q][rec_off + kb + tid];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (w0 + q < a.W) {
+                        if (mine) {
+                            if ((unsigned)r[q].idx < (unsigned)M)
+                                St[(r[q].idx >> 7) * XS + (r[q].idx & 127)] += r[q].val;
+                            else
+                                atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                        }
+                        __syncthreads();
+                    }
+                }
+            }
+        }
+        // two inverse passes (rolled): pass 0 along row j, pass 1 down column j
+        float in[H], out[H];
+        bool arrived = true;
+#pragma unroll 1
+        for (int pass = 0; pass < 2; ++pass) {
+            const int line = pass == 0 ? j * XS : j;   // start of line j
+            const int step = pass == 0 ? 1 : XS;       // distance between consecutive elements of the line
+#pragma unroll
+            for (int p = 0; p < H; ++p) in[p] = St[line + (2 * p + h) * step];
+            fence_proxy_async();
+            __syncthreads();  // every coefficient of the tile has been read
+            inverse_half(h, in, out);
+            // exchange e / o inside the line: e at elements 0..63, o at 64..127
+#pragma unroll
+            for (int n = 0; n < H; ++n) St[line + (h * H + n) * step] = out[n];
+            __syncthreads();
+#pragma unroll
+            for (int n = 0; n < H; ++n) {
+                const float other = St[line + ((h ^ 1) * H + n) * step];
+                out[n] = h ? other - out[n] : out[n] + other;  // h=0: element n;  h=1: element 127-n
+            }
+            fence_proxy_async();
+            __syncthreads();  // both halves of every line have read their partner's values
+            if (pass == 0) {
+#pragma unroll
+                for (int n = 0; n < H; ++n) St[line + (h ? (S - 1 - n) : n) * step] = out[n];
+                __syncthreads();
+            } else {
+                if (tid == 0) {
+                    mbar_expect_tx(bar, M * sizeof(float));
+                    tma_load_2d(smem_u32(Xt), tm_x, k1 * S, k0 * S, bar);
+                }
+                arrived = mbar_wait_bounded(bar, phase);
+                phase ^= 1u;
+            }
+        }
+        if (!__syncthreads_and(arrived)) {
+            if (tid == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
+            mbar_wait_bounded(bar, phase ^ 1u);
+            return;
+        }
+#pragma unroll
+        for (int n = 0; n < H; ++n) {
+            const int row = h ? (S - 1 - n) : n;
+            const float rv = out[n];
+            float stepv = __uint_as_float(lr_bits ^ (~__float_as_uint(rv) & 0x80000000u));
+            stepv = (rv == 0.f) ? 0.f : stepv;
+            x[base + (size_t)row * te.n1 + j] = fmaf(Xt[row * S + j], decay, stepv);
+        }
+        fence_proxy_async();
+        __syncthreads();
+    }
+}
+
+template <typename K>
+cudaError_t launch128(K kernel, size_t smem, long long n_chunks, int sm_count, cudaStream_t stream, const void *args)
+{
+    if (n_chunks <= 0) return cudaSuccess;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    int per_sm = 0;
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, THREADS, smem);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    long long grid = (long long)sm_count * per_sm;
+    if (grid > n_chunks) grid = n_chunks;
+    void *params[] = {const_cast<void *>(args)};
+    return cudaLaunchKernel((const void *)kernel, dim3((unsigned)grid), dim3(THREADS), params, smem, stream);
+}
+
+}  // namespace
+
+cudaError_t demo_launch_compress_fast128(const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
+{
+    if (!a.tmap_m || !a.tmap_g) return cudaErrorNotSupported;
+    if (a.grad_bf16)
+        return launch128(compress_fast128_kernel<__nv_bfloat16>, compress128_smem<__nv_bfloat16>(), a.n_chunks, sm_count,
+                         stream, &a);
+    return launch128(compress_fast128_kernel<float>, compress128_smem<float>(), a.n_chunks, sm_count, stream, &a);
+}
+
+cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
+{
+    if (!a.tmap_x) return cudaErrorNotSupported;
+    return launch128(decode_fast128_kernel, decode128_smem(), a.n_chunks, sm_count, stream, &a);
+}

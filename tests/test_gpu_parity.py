@@ -41,6 +41,18 @@ def test_small_decoder_s64_k32(path):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("k", [32, 200])
+def test_small_decoder_s128(path, k):
+    """Chunk size 128 (the paper's second setting): split 128-point transforms on the fast path."""
+    wl = inputs.small_decoder(chunk=128, topk=k, num_workers=3)
+    r = parity.Runner(wl, max_chunks=40, path=path)
+    for _ in range(2):
+        r.step()
+    assert r.report["pinned"] > 0.95 * r.report["chunks"]
+    r.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_single_matrix_sampled(path):
     """Config 2 at full size (8192 x 8192, row-scaled bf16 grads), 2 steps, 300 sampled chunks."""
     wl = inputs.single_matrix()
@@ -50,7 +62,7 @@ def test_single_matrix_sampled(path):
     r.close()
 
 
-@pytest.mark.parametrize("s,k", [(8, 64), (32, 1024), (64, 4096), (64, 64)])
+@pytest.mark.parametrize("s,k", [(8, 64), (32, 1024), (64, 4096), (64, 64), (128, 16384)])
 def test_lossless_when_k_covers_the_chunk(s, k):
     """k = M: zero residual momentum and an update of exactly sign(sum_w m_w)."""
     shapes = [(2 * s, 3 * s), (4 * s,)]
@@ -84,7 +96,7 @@ def test_stress_matrix_ties(s, k):
 
 def test_all_zero_chunks_emit_lowest_indices():
     """Exactly tied magnitudes: the deterministic tie-break (lowest index) is bit-testable."""
-    for s, shapes in [(64, [(128, 128), (128,)]), (8, [(16, 16), (16,)]), (32, [(64, 64)])]:
+    for s, shapes in [(64, [(128, 128), (128,)]), (8, [(16, 16), (16,)]), (32, [(64, 64)]), (128, [(256, 128)])]:
         for path in PATHS:
             tr = demo.DemoTransform(shapes, chunk=s, topk=5, beta=0.9, lr=1e-3, weight_decay=0.0, num_workers=1,
                                     grad_dtype=demo.DEMO_F32)
