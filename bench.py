@@ -94,7 +94,7 @@ def algorithmic_bytes(wl, gbytes: int):
     return core, payload
 
 
-def cpu_baseline(wl, target_s: float = 12.0):
+def cpu_baseline(wl, target_s: float = 20.0):
     """Time the oracle, as it stands, on a bounded sample: n chunks of 2-D tiles through W compress
     passes and one decode.  Returns params/s on that sample."""
     import numpy as np
