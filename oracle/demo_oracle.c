@@ -18,7 +18,8 @@
  *   - momentum update is m <- beta*m + g (every algorithm listing), not the (1-beta) form
  *     of the Section 2.1 text equation;
  *   - aggregation is the plain sum over workers, in worker order (Decompress&Aggregate);
- *   - full momentum subtraction (alpha = 1; Algorithm 1 line "in-place residual");
+ *   - momentum subtraction m <- B - alpha * IDCT(kept) (Section 2.1, "Momentum Subtraction as Error
+ *     Feedback", alpha in (0, 1]); alpha = 1 is what every algorithm listing uses and the default;
  *   - exactly k_eff coefficients per chunk (||Q_hat||_0 = k, Section 2.1); ties at the
  *     k-th magnitude go to the lowest flat index;
  *   - sign(0) = 0 (the sign lemmas of the appendix treat sign(y) = 0 as a legal case);
@@ -182,14 +183,14 @@ void oracle_topk(int M, int k, const double *Q, int32_t *idx_out, double *a_k, d
  *   B     = beta*m + g                                   (momentum update)
  *   Q     = T(B; C)                                      (chunk DCT)
  *   Q_sp  = Top-k(Q)                                     (k_eff records, ascending index)
- *   m_new = B - T^-1(Q_sp; C^T)                          (momentum subtraction, alpha = 1)
+ *   m_new = B - alpha * T^-1(Q_sp; C^T)                  (momentum subtraction)
  * forced_idx (nullable): use this index set (k_eff ascending indices) instead of the
  * oracle's own top-k -- used by the comparison rule for chunks whose k-th / (k+1)-th
  * magnitudes are too close to pin the set.
  * Outputs (any may be NULL except m_new): Q_out[M], idx_out[k_eff], val_out[k_eff] (fp64
  * coefficient at each index), gap[2] = {a_k, a_k1} of the oracle's OWN order.
  * ------------------------------------------------------------------------------------- */
-void oracle_compress_chunk(int s, int rows, int k, double beta, const double *C, const double *g,
+void oracle_compress_chunk(int s, int rows, int k, double beta, double alpha, const double *C, const double *g,
                            const double *m, const int32_t *forced_idx, double *Q_out,
                            int32_t *idx_out, double *val_out, double *m_new, double *gap)
 {
@@ -212,7 +213,7 @@ void oracle_compress_chunk(int s, int rows, int k, double beta, const double *C,
     if (forced_idx) memcpy(idx, forced_idx, sizeof(int32_t) * (size_t)k_eff);
     for (int i = 0; i < k_eff; ++i) Qsp[idx[i]] = Q[idx[i]];
     oracle_inverse(s, rows, C, Qsp, R);
-    for (int i = 0; i < M; ++i) m_new[i] = B[i] - R[i];
+    for (int i = 0; i < M; ++i) m_new[i] = B[i] - alpha * R[i];
 
     if (Q_out) memcpy(Q_out, Q, sizeof(double) * (size_t)M);
     if (idx_out) memcpy(idx_out, idx, sizeof(int32_t) * (size_t)k_eff);
@@ -226,7 +227,7 @@ void oracle_compress_chunk(int s, int rows, int k, double beta, const double *C,
 }
 
 /* Batch of independent chunks given as tiles: g, m are [n][M]; outputs [n][...]. */
-void oracle_compress_chunks(int64_t n, int s, int rows, int k, double beta, const double *g,
+void oracle_compress_chunks(int64_t n, int s, int rows, int k, double beta, double alpha, const double *g,
                             const double *m, const int32_t *forced_idx, double *Q_out,
                             int32_t *idx_out, double *val_out, double *m_new, double *gap,
                             int n_threads)
@@ -240,7 +241,7 @@ void oracle_compress_chunks(int64_t n, int s, int rows, int k, double beta, cons
 #pragma omp parallel for schedule(dynamic, 1) num_threads(n_threads > 0 ? n_threads : omp_get_max_threads())
 #endif
     for (int64_t c = 0; c < n; ++c) {
-        oracle_compress_chunk(s, rows, k, beta, C, g + c * M, m + c * M,
+        oracle_compress_chunk(s, rows, k, beta, alpha, C, g + c * M, m + c * M,
                               forced_idx ? forced_idx + c * k_eff : NULL,
                               Q_out ? Q_out + c * M : NULL, idx_out ? idx_out + c * k_eff : NULL,
                               val_out ? val_out + c * k_eff : NULL, m_new + c * M,
@@ -257,7 +258,7 @@ void oracle_compress_chunks(int64_t n, int s, int rows, int k, double beta, cons
  * records: [n_chunks][k_eff] of {int32 idx, float val} -- val is the fp64 coefficient
  * rounded once to fp32.  val64 / gap / forced_idx as in the chunk routine (nullable).
  * ------------------------------------------------------------------------------------- */
-int oracle_compress_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, double beta, const double *g,
+int oracle_compress_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, double beta, double alpha, const double *g,
                            double *m, const int32_t *forced_idx, oracle_record *records, double *val64,
                            double *gap, int n_threads)
 {
@@ -283,7 +284,7 @@ int oracle_compress_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, doubl
         int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)k_eff);
         oracle_block_extract(g, n1, rows, s, k0, k1, gt);
         oracle_block_extract(m, n1, rows, s, k0, k1, mt);
-        oracle_compress_chunk(s, rows, k, beta, C, gt, mt, forced_idx ? forced_idx + c * k_eff : NULL, NULL,
+        oracle_compress_chunk(s, rows, k, beta, alpha, C, gt, mt, forced_idx ? forced_idx + c * k_eff : NULL, NULL,
                               idx, vals, mn, gap ? gap + c * 2 : NULL);
         oracle_block_insert(m, n1, rows, s, k0, k1, mn);
         for (int i = 0; i < k_eff; ++i) {

@@ -54,10 +54,10 @@ def _load():
             lib.oracle_inverse.restype = None
             lib.oracle_topk.argtypes = [i32, i32, c_dp, c_ip, c_dp, c_dp]
             lib.oracle_topk.restype = None
-            lib.oracle_compress_chunks.argtypes = [i64, i32, i32, i32, f64, c_dp, c_dp, c_ip, c_dp, c_ip,
+            lib.oracle_compress_chunks.argtypes = [i64, i32, i32, i32, f64, f64, c_dp, c_dp, c_ip, c_dp, c_ip,
                                                    c_dp, c_dp, c_dp, i32]
             lib.oracle_compress_chunks.restype = None
-            lib.oracle_compress_tensor.argtypes = [i32, i64, i64, i32, i32, f64, c_dp, c_dp, c_ip, vp, c_dp,
+            lib.oracle_compress_tensor.argtypes = [i32, i64, i64, i32, i32, f64, f64, c_dp, c_dp, c_ip, vp, c_dp,
                                                    c_dp, i32]
             lib.oracle_compress_tensor.restype = i32
             lib.oracle_decode_chunks.argtypes = [i64, i32, i32, i32, i32, vp, c_dp, f64, f64, c_dp, c_dp, i32]
@@ -136,7 +136,8 @@ def topk(Q: np.ndarray, k: int):
     return idx, a.value, b.value
 
 
-def compress_chunks(g, m, s: int, rows: int, k: int, beta: float, forced_idx=None, n_threads: int = 0):
+def compress_chunks(g, m, s: int, rows: int, k: int, beta: float, forced_idx=None, n_threads: int = 0,
+                    alpha: float = 1.0):
     """Independent chunks given as tiles [n, rows*s].
 
     Returns dict(Q [n,M], idx [n,k_eff] int32, val [n,k_eff] fp64, m_new [n,M], gap [n,2])."""
@@ -155,12 +156,12 @@ def compress_chunks(g, m, s: int, rows: int, k: int, beta: float, forced_idx=Non
     fi = None
     if forced_idx is not None:
         fi = np.ascontiguousarray(forced_idx, dtype=np.int32).reshape(n, k_eff)
-    _load().oracle_compress_chunks(n, s, rows, k, float(beta), _dp(g), _dp(m), _ip(fi) if fi is not None else None,
+    _load().oracle_compress_chunks(n, s, rows, k, float(beta), float(alpha), _dp(g), _dp(m), _ip(fi) if fi is not None else None,
                                    _dp(Q), _ip(idx), _dp(val), _dp(m_new), _dp(gap), n_threads)
     return dict(Q=Q, idx=idx, val=val, m_new=m_new, gap=gap)
 
 
-def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_threads: int = 0):
+def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_threads: int = 0, alpha: float = 1.0):
     """One tensor (1-D or 2-D), one worker.  Returns dict(m_new, records [n_chunks,k_eff], val64, gap)."""
     g = _f64(g)
     m_new = _f64(m).copy()
@@ -178,7 +179,7 @@ def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_thread
     fi = None
     if forced_idx is not None:
         fi = np.ascontiguousarray(forced_idx, dtype=np.int32).reshape(n_chunks, k_eff)
-    rc = _load().oracle_compress_tensor(ndim, n0, n1, s, k, float(beta), _dp(g), _dp(m_new),
+    rc = _load().oracle_compress_tensor(ndim, n0, n1, s, k, float(beta), float(alpha), _dp(g), _dp(m_new),
                                         _ip(fi) if fi is not None else None, rec.ctypes.data_as(ctypes.c_void_p),
                                         _dp(val64), _dp(gap), n_threads)
     if rc != 0:

@@ -390,3 +390,30 @@ def test_payload_volume_matches_paper_ratios():
     assert n_records == (n0 // s) * (n1 // s) * k
     assert (n0 * n1) // n_records == kv["tx_reduction"]  # coefficients sent: M / k
     assert (n0 * n1) // (W * n_records) == kv["rx_reduction"]  # received from 8 workers
+
+
+# --------------------------------------------------------------------------------------------
+# alpha-scaled momentum subtraction (Section 2.1 "Momentum Subtraction as Error Feedback")
+# --------------------------------------------------------------------------------------------
+def test_alpha_scaled_momentum_subtraction():
+    s, rows, k, beta = 8, 8, 6, 0.999
+    rng = np.random.default_rng(31)
+    g = rng.standard_normal((3, 64)) * 0.01
+    m = rng.standard_normal((3, 64)) * 0.1
+    B = beta * m + g
+    full = orc.compress_chunks(g, m, s, rows, k, beta)  # default alpha = 1
+    one = orc.compress_chunks(g, m, s, rows, k, beta, alpha=1.0)
+    assert np.array_equal(full["m_new"], one["m_new"])
+    zero = orc.compress_chunks(g, m, s, rows, k, beta, alpha=0.0)
+    assert np.array_equal(zero["m_new"], B)  # nothing removed
+    assert np.array_equal(zero["idx"], full["idx"]) and np.array_equal(zero["val"], full["val"])  # payload unaffected
+    a = 0.2
+    part = orc.compress_chunks(g, m, s, rows, k, beta, alpha=a)
+    # linear in alpha: B - alpha * IDCT(kept), with IDCT(kept) = B - m_new(alpha = 1)
+    assert np.max(np.abs(part["m_new"] - (B - a * (B - full["m_new"])))) < 1e-14
+    # the transmitted part is removed only partially: DCT of the residual keeps (1 - alpha) of the kept coefficients
+    for c in range(3):
+        Qres = orc.forward(part["m_new"][c].reshape(s, s)).reshape(-1)
+        assert np.max(np.abs(Qres[full["idx"][c]] - (1 - a) * full["val"][c])) < 1e-12
+    t = orc.compress_tensor(g.reshape(24, 8), m.reshape(24, 8), s, k, beta, alpha=a)
+    assert np.max(np.abs(t["m_new"].reshape(3, 64) - part["m_new"])) < 1e-14
