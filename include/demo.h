@@ -182,6 +182,12 @@ demo_status demo_decode_apply_static(const demo_config *cfg, const demo_tensor_d
  * the next demo_decode_apply.  Errors: INVALID_ARG (null ctx, non-finite lr). */
 demo_status demo_set_lr(demo_ctx *ctx, float lr);
 
+/* Momentum-subtraction coefficient of Section 2.1 ("Momentum Subtraction as Error Feedback"):
+ * demo_compress leaves m <- (beta*m + g) - alpha * IDCT(kept coefficients); the records always carry
+ * the full coefficients.  Default 1 (the algorithm listings); 0 <= alpha <= 1.  Takes effect for the
+ * next demo_compress.  Errors: INVALID_ARG. */
+demo_status demo_set_alpha(demo_ctx *ctx, float alpha);
+
 /* Select the kernel family (see demo_path).  Errors: INVALID_ARG. */
 demo_status demo_set_path(demo_ctx *ctx, int32_t path);
 

@@ -20,7 +20,7 @@ RECORD_BYTES = 8
 
 EXPORTS = [
     "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
-    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
 ]
 
@@ -75,6 +75,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_decode_apply_static.restype = i32
     lib.demo_set_lr.argtypes = [vp, ctypes.c_float]
     lib.demo_set_lr.restype = i32
+    lib.demo_set_alpha.argtypes = [vp, ctypes.c_float]
+    lib.demo_set_alpha.restype = i32
     lib.demo_set_path.argtypes = [vp, i32]
     lib.demo_set_path.restype = i32
     lib.demo_launch_count.argtypes = [vp]
@@ -206,6 +208,11 @@ class DemoTransform:
         st = self.lib.demo_set_lr(self._ctx, lr)
         if st != 0:
             raise DemoError(st, "demo_set_lr")
+
+    def set_alpha(self, alpha: float) -> None:
+        st = self.lib.demo_set_alpha(self._ctx, alpha)
+        if st != 0:
+            raise DemoError(st, "demo_set_alpha")
 
     def set_path(self, path: int) -> None:
         st = self.lib.demo_set_path(self._ctx, path)

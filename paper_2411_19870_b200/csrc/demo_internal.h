@@ -32,6 +32,7 @@ struct DemoCompressArgs {
     DemoRecord *payload;        // device, whole payload of this worker
     const float *C;             // device, s x s orthonormal DCT-II, C[u*s + n]
     float beta;
+    float alpha;    // momentum-subtraction coefficient: m <- B - alpha * IDCT(kept)
     int grad_bf16;  // 1: gradients are bf16, 0: fp32
     int *status;    // device status word (sticky)
     // Optional TMA tensor maps (128-byte CUtensorMap objects in device memory, indexed like the

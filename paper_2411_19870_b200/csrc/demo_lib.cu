@@ -17,6 +17,7 @@ struct demo_ctx {
     int sm_count = 0;
     int n_tensors = 0;
     int path = DEMO_PATH_AUTO;
+    float alpha = 1.0f;  // momentum-subtraction coefficient
     long long launches = 0;
     std::vector<demo_tensor_desc> descs;
     std::vector<long long> first_record, n_chunks, n_elems;
@@ -348,6 +349,7 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
     a.payload = static_cast<DemoRecord *>(payload_out);
     a.C = ctx->d_C;
     a.beta = ctx->cfg.beta;
+    a.alpha = ctx->alpha;
     a.grad_bf16 = ctx->cfg.grad_dtype == DEMO_BF16;
     a.status = ctx->d_status;
     a.tmap_m = ctx->encode ? ctx->d_tm_m + row : nullptr;
@@ -484,6 +486,13 @@ demo_status demo_set_lr(demo_ctx *ctx, float lr)
 {
     if (!ctx || !std::isfinite(lr)) return DEMO_ERR_INVALID_ARG;
     ctx->cfg.lr = lr;
+    return DEMO_OK;
+}
+
+demo_status demo_set_alpha(demo_ctx *ctx, float alpha)
+{
+    if (!ctx || !(alpha >= 0.0f && alpha <= 1.0f)) return DEMO_ERR_INVALID_ARG;
+    ctx->alpha = alpha;
     return DEMO_OK;
 }
 

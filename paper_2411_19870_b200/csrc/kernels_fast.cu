@@ -466,7 +466,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                         rec[pos] = r;
                         const int v = r.idx & (S - 1);  // k_eff <= S <= 64 on this path
                         const int uo = (r.idx >> LOG2S) * XS;
-                        recs4[pos] = make_int4(uo, v * S, __float_as_int(r.val), 0);
+                        recs4[pos] = make_int4(uo, v * S, __float_as_int(a.alpha * r.val), 0);
                         if ((int)pos == k_eff - 1)
                             for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(uo, 0, 0, 0);
                     }
@@ -517,7 +517,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                     r.val = val;
                     rec[pos] = r;
                     if (k_eff <= 64) {
-                        recs4[pos] = make_int4(t * XS, v * S, __float_as_int(val), 0);
+                        recs4[pos] = make_int4(t * XS, v * S, __float_as_int(a.alpha * val), 0);
                         if ((int)pos == k_eff - 1)
                             for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(t * XS, 0, 0, 0);
                     }
@@ -568,7 +568,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                         acc = 0.f;
                         cur_u = u;
                     }
-                    acc = fmaf(rc.val, __ldg(Ct + v * S), acc);
+                    acc = fmaf(a.alpha * rc.val, __ldg(Ct + v * S), acc);
                 }
             }
             if (cur_u >= 0) X[cur_u + t] = acc;

@@ -248,7 +248,8 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                     r.idx = idx;
                     r.val = val;
                     rec[pos] = r;
-                    if (k_eff <= 128) recs4[pos] = make_int4((idx >> 7) * XS, (idx & 127) * S, __float_as_int(val), 0);
+                    if (k_eff <= 128)
+                        recs4[pos] = make_int4((idx >> 7) * XS, (idx & 127) * S, __float_as_int(a.alpha * val), 0);
                 }
             }
         }
@@ -273,7 +274,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                     const DemoRecord rc = rec[r];
                     uo = (rc.idx >> 7) * XS;
                     vo = (rc.idx & 127) * S;
-                    val = rc.val;
+                    val = a.alpha * rc.val;
                 }
                 if (uo != cur_u) {
                     if (cur_u >= 0) X[cur_u + j] = acc;

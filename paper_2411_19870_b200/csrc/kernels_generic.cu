@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(GEN_THREADS) compress_generic_kernel(DemoCompr
                     r.val = v;
                     rec[pos] = r;
                 }
-                O[i] = sel ? v : 0.f;
+                O[i] = sel ? a.alpha * v : 0.f;  // the residual removes alpha times the kept part
             }
         }
         __syncthreads();

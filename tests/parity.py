@@ -66,12 +66,12 @@ class Report(dict):
         self[key] = self.get(key, 0) + int(n)
 
 
-def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, report: Report, what=""):
+def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, report: Report, what="", alpha=1.0):
     """All arguments are per-chunk arrays of the same n chunks (float64 / records)."""
     M = rows * s
     k_eff = min(k, M)
     n = g.shape[0]
-    ref = orc.compress_chunks(g, m_before, s, rows, k, beta)
+    ref = orc.compress_chunks(g, m_before, s, rows, k, beta, alpha=alpha)
     Q = ref["Q"]
     qinf = np.max(np.abs(Q), axis=1)
     floor = FLOOR_REL * qinf
@@ -121,7 +121,7 @@ def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, repor
     # residual momentum: oracle continued from the GPU's index set where the sets differ
     m_ref = ref["m_new"]
     if len(diff):
-        forced = orc.compress_chunks(g[diff], m_before[diff], s, rows, k, beta, forced_idx=idx_gpu[diff].astype(np.int32))
+        forced = orc.compress_chunks(g[diff], m_before[diff], s, rows, k, beta, forced_idx=idx_gpu[diff].astype(np.int32), alpha=alpha)
         m_ref = m_ref.copy()
         m_ref[diff] = forced["m_new"]
     # the abs tolerance is scaled by the chunk's pre-subtraction magnitude (the fp32 rounding of
@@ -164,7 +164,7 @@ def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Re
 class Runner:
     """Drives a workload through the C ABI and checks sampled (or all) chunks every step."""
 
-    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0):
+    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0, alpha=None):
         import paper_2411_19870_b200 as demo
         from paper_2411_19870_b200 import inputs
 
@@ -176,6 +176,10 @@ class Runner:
                                      device=self.device.index or 0)
         if path is not None:
             self.tr.set_path(path)
+        self.alpha = 1.0
+        if alpha is not None:
+            self.tr.set_alpha(alpha)
+            self.alpha = float(np.float32(alpha))
         self.params = inputs.make_params(wl, self.device)
         self.mom = [inputs.make_momentum(wl, self.device) for _ in range(wl.num_workers)]
         self.streams = [inputs.GradStream(wl, w, self.device) for w in range(wl.num_workers)]
@@ -204,7 +208,7 @@ class Runner:
                     check_compress_chunks(
                         gather_tiles(g[t], s, self.ids[t]), before[t], gather_tiles(self.mom[w][t], s, self.ids[t]),
                         gather_records(self.payloads[w], first, k_eff, self.ids[t]), s, rows, wl.topk, self.beta,
-                        self.report, what="compress w%d t%d" % (w, t))
+                        self.report, what="compress w%d t%d" % (w, t), alpha=self.alpha)
         if check:
             xb = [gather_tiles(self.params[t], s, self.ids[t]) for t in range(T)]
         self.tr.decode_apply(self.payloads, self.params)

@@ -278,3 +278,22 @@ def test_decoder_1b_full_size_sampled():
     assert r.report["chunks"] == 16 * 146 * 6
     r.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("s", [8, 64, 128])
+@pytest.mark.parametrize("alpha", [0.2, 0.0])
+def test_alpha_scaled_momentum_subtraction(s, alpha):
+    """Section 2.1's subtraction coefficient: the residual removes only alpha of the transmitted part."""
+    shapes = [(2 * s, 4 * s), (2 * s,)]
+    wl = inputs.Workload("alpha", shapes, chunk=s, topk=max(2, s // 2), num_workers=2, grad_kind="normal", grad_std=0.01)
+    for path in PATHS:
+        r = parity.Runner(wl, max_chunks=10**9, path=path, alpha=alpha)
+        r.step()
+        r.step()
+        r.close()
+    with pytest.raises(demo.DemoError):
+        r2 = parity.Runner(wl, max_chunks=4)
+        try:
+            r2.tr.set_alpha(1.5)
+        finally:
+            r2.close()
