@@ -17,7 +17,10 @@
  * notes too):
  *   - momentum update is m <- beta*m + g (every algorithm listing), not the (1-beta) form
  *     of the Section 2.1 text equation;
- *   - aggregation is the plain sum over workers, in worker order (Decompress&Aggregate);
+ *   - aggregation is the plain sum over workers, in worker order (Decompress&Aggregate) by default;
+ *     the mean over workers (Section 2.1, AvgAllGather) and the per-coordinate count-normalised
+ *     mean with 0/0 = 0 (appendix algorithm "Sparse Top-k Averaging") are selectable, as is the
+ *     identity in place of the sign for the transform phi of Section 2.1;
  *   - momentum subtraction m <- B - alpha * IDCT(kept) (Section 2.1, "Momentum Subtraction as Error
  *     Feedback", alpha in (0, 1]); alpha = 1 is what every algorithm listing uses and the default;
  *   - exactly k_eff coefficients per chunk (||Q_hat||_0 = k, Section 2.1); ties at the
@@ -305,23 +308,36 @@ int oracle_compress_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, doubl
 /* ---------------------------------------------------------------------------------------
  * One chunk of Decompress&Aggregate + the parameter update (Algorithm 1, server side):
  *   S = 0;  for w = 0..W-1 in order:  S[idx] += val  for that worker's k_eff records
+ *   agg = 0: S as is (sum);  agg = 1: S / W (mean, AvgAllGather);
+ *   agg = 2: S[i] / n[i] with n[i] the number of workers that sent coordinate i, 0/0 = 0
+ *            (appendix algorithm "Sparse Top-k Averaging")
  *   R = T^-1(S; C^T)
- *   sg = (R > 0) - (R < 0)                                  (sign(0) = 0)
+ *   phi = 0: sg = (R > 0) - (R < 0)  (Signum, sign(0) = 0);  phi = 1: sg = R  (SGD-style, Section 2.1)
  *   x_new = x - lr * (sg + wd * x)                          (decoupled weight decay)
  * recs[w] points at that worker's k_eff records for this chunk (fp32 values as stored).
  * R_out (nullable) receives the reconstructed momentum chunk.
  * ------------------------------------------------------------------------------------- */
-void oracle_decode_chunk(int s, int rows, int k_eff, int W, const double *C, const oracle_record *const *recs,
-                         const double *x, double lr, double wd, double *x_new, double *R_out)
+void oracle_decode_chunk(int s, int rows, int k_eff, int W, int agg, int phi, const double *C,
+                         const oracle_record *const *recs, const double *x, double lr, double wd, double *x_new,
+                         double *R_out)
 {
     const int M = rows * s;
     double *S = (double *)calloc((size_t)M, sizeof(double));
+    int *cnt = (int *)calloc((size_t)M, sizeof(int));
     double *R = (double *)malloc(sizeof(double) * (size_t)M);
     for (int w = 0; w < W; ++w)
-        for (int i = 0; i < k_eff; ++i) S[recs[w][i].idx] += (double)recs[w][i].val;
+        for (int i = 0; i < k_eff; ++i) {
+            S[recs[w][i].idx] += (double)recs[w][i].val;
+            cnt[recs[w][i].idx] += 1;
+        }
+    if (agg == 1)
+        for (int i = 0; i < M; ++i) S[i] /= (double)W;
+    if (agg == 2)
+        for (int i = 0; i < M; ++i) S[i] = cnt[i] ? S[i] / (double)cnt[i] : 0.0;
+    free(cnt);
     oracle_inverse(s, rows, C, S, R);
     for (int i = 0; i < M; ++i) {
-        double sg = (double)((R[i] > 0.0) - (R[i] < 0.0));
+        double sg = (phi == 1) ? R[i] : (double)((R[i] > 0.0) - (R[i] < 0.0));
         x_new[i] = x[i] - lr * (sg + wd * x[i]);
     }
     if (R_out) memcpy(R_out, R, sizeof(double) * (size_t)M);
@@ -330,7 +346,7 @@ void oracle_decode_chunk(int s, int rows, int k_eff, int W, const double *C, con
 }
 
 /* Batch of independent chunks: recs is [W][n][k_eff] contiguous; x, x_new, R_out are [n][M]. */
-void oracle_decode_chunks(int64_t n, int s, int rows, int k_eff, int W, const oracle_record *recs,
+void oracle_decode_chunks(int64_t n, int s, int rows, int k_eff, int W, int agg, int phi, const oracle_record *recs,
                           const double *x, double lr, double wd, double *x_new, double *R_out, int n_threads)
 {
     const int M = rows * s;
@@ -343,7 +359,7 @@ void oracle_decode_chunks(int64_t n, int s, int rows, int k_eff, int W, const or
     for (int64_t c = 0; c < n; ++c) {
         const oracle_record **rw = (const oracle_record **)malloc(sizeof(void *) * (size_t)W);
         for (int w = 0; w < W; ++w) rw[w] = recs + ((size_t)w * (size_t)n + (size_t)c) * (size_t)k_eff;
-        oracle_decode_chunk(s, rows, k_eff, W, C, rw, x + c * M, lr, wd, x_new + c * M,
+        oracle_decode_chunk(s, rows, k_eff, W, agg, phi, C, rw, x + c * M, lr, wd, x_new + c * M,
                             R_out ? R_out + c * M : NULL);
         free(rw);
     }
@@ -352,7 +368,7 @@ void oracle_decode_chunks(int64_t n, int s, int rows, int k_eff, int W, const or
 
 /* Whole tensor: payloads[w] points at worker w's [n_chunks][k_eff] records for THIS tensor.
  * x is updated in place; R_out (nullable) receives the reconstructed global momentum. */
-int oracle_decode_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, int W,
+int oracle_decode_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, int W, int agg, int phi,
                          const oracle_record *const *payloads, double *x, double lr, double wd, double *R_out,
                          int n_threads)
 {
@@ -377,7 +393,7 @@ int oracle_decode_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, int W,
         const oracle_record **rw = (const oracle_record **)malloc(sizeof(void *) * (size_t)W);
         for (int w = 0; w < W; ++w) rw[w] = payloads[w] + (size_t)c * (size_t)k_eff;
         oracle_block_extract(x, n1, rows, s, k0, k1, xt);
-        oracle_decode_chunk(s, rows, k_eff, W, C, rw, xt, lr, wd, xn, Rt);
+        oracle_decode_chunk(s, rows, k_eff, W, agg, phi, C, rw, xt, lr, wd, xn, Rt);
         oracle_block_insert(x, n1, rows, s, k0, k1, xn);
         if (R_out) oracle_block_insert(R_out, n1, rows, s, k0, k1, Rt);
         free(xt);

@@ -60,9 +60,9 @@ def _load():
             lib.oracle_compress_tensor.argtypes = [i32, i64, i64, i32, i32, f64, f64, c_dp, c_dp, c_ip, vp, c_dp,
                                                    c_dp, i32]
             lib.oracle_compress_tensor.restype = i32
-            lib.oracle_decode_chunks.argtypes = [i64, i32, i32, i32, i32, vp, c_dp, f64, f64, c_dp, c_dp, i32]
+            lib.oracle_decode_chunks.argtypes = [i64, i32, i32, i32, i32, i32, i32, vp, c_dp, f64, f64, c_dp, c_dp, i32]
             lib.oracle_decode_chunks.restype = None
-            lib.oracle_decode_tensor.argtypes = [i32, i64, i64, i32, i32, i32, ctypes.POINTER(vp), c_dp, f64,
+            lib.oracle_decode_tensor.argtypes = [i32, i64, i64, i32, i32, i32, i32, i32, ctypes.POINTER(vp), c_dp, f64,
                                                  f64, c_dp, i32]
             lib.oracle_decode_tensor.restype = i32
             lib.oracle_max_threads.argtypes = []
@@ -187,7 +187,11 @@ def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_thread
     return dict(m_new=m_new, records=rec, val64=val64, gap=gap)
 
 
-def decode_chunks(records, x, s: int, rows: int, lr: float, wd: float, n_threads: int = 0):
+AGG_SUM, AGG_MEAN, AGG_COUNT_MEAN = 0, 1, 2
+PHI_SIGN, PHI_IDENTITY = 0, 1
+
+
+def decode_chunks(records, x, s: int, rows: int, lr: float, wd: float, n_threads: int = 0, agg: int = 0, phi: int = 0):
     """records [W, n, k_eff] (RECORD_DTYPE), x [n, rows*s] -> dict(x_new [n,M], R [n,M])."""
     records = np.ascontiguousarray(records, dtype=RECORD_DTYPE)
     W, n, k_eff = records.shape
@@ -195,12 +199,12 @@ def decode_chunks(records, x, s: int, rows: int, lr: float, wd: float, n_threads
     x = _f64(x).reshape(n, M)
     x_new = np.empty_like(x)
     R = np.empty_like(x)
-    _load().oracle_decode_chunks(n, s, rows, k_eff, W, records.ctypes.data_as(ctypes.c_void_p), _dp(x), float(lr),
+    _load().oracle_decode_chunks(n, s, rows, k_eff, W, agg, phi, records.ctypes.data_as(ctypes.c_void_p), _dp(x), float(lr),
                                  float(wd), _dp(x_new), _dp(R), n_threads)
     return dict(x_new=x_new, R=R)
 
 
-def decode_tensor(payloads, x, s: int, k: int, lr: float, wd: float, n_threads: int = 0):
+def decode_tensor(payloads, x, s: int, k: int, lr: float, wd: float, n_threads: int = 0, agg: int = 0, phi: int = 0):
     """payloads: list over workers of [n_chunks, k_eff] record arrays for this tensor.
 
     Returns dict(x_new, R) with R the reconstructed global momentum of the tensor."""
@@ -211,7 +215,7 @@ def decode_tensor(payloads, x, s: int, k: int, lr: float, wd: float, n_threads: 
     keep = [np.ascontiguousarray(p, dtype=RECORD_DTYPE) for p in payloads]
     arr = (ctypes.c_void_p * W)(*[p.ctypes.data for p in keep])
     R = np.empty_like(x_new)
-    rc = _load().oracle_decode_tensor(ndim, n0, n1, s, k, W, arr, _dp(x_new), float(lr), float(wd), _dp(R),
+    rc = _load().oracle_decode_tensor(ndim, n0, n1, s, k, W, agg, phi, arr, _dp(x_new), float(lr), float(wd), _dp(R),
                                       n_threads)
     if rc != 0:
         raise ValueError("oracle_decode_tensor rejected the shape")

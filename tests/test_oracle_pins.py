@@ -417,3 +417,58 @@ def test_alpha_scaled_momentum_subtraction():
         assert np.max(np.abs(Qres[full["idx"][c]] - (1 - a) * full["val"][c])) < 1e-12
     t = orc.compress_tensor(g.reshape(24, 8), m.reshape(24, 8), s, k, beta, alpha=a)
     assert np.max(np.abs(t["m_new"].reshape(3, 64) - part["m_new"])) < 1e-14
+
+
+# --------------------------------------------------------------------------------------------
+# Aggregation variants and phi = identity (Section 2.1: AvgAllGather, phi; appendix algorithm
+# "Sparse Top-k Averaging": sum / per-coordinate count, 0/0 = 0)
+# --------------------------------------------------------------------------------------------
+def _recs(W, n, k, idx_lists, val_lists):
+    r = np.zeros((W, n, k), dtype=orc.RECORD_DTYPE)
+    for w in range(W):
+        r[w, 0]["idx"] = idx_lists[w]
+        r[w, 0]["val"] = np.asarray(val_lists[w], dtype=np.float32)
+    return r
+
+
+def test_aggregation_variants_hand_example():
+    s, rows, M = 4, 1, 4  # 1-D segments of 4: coefficients are easy to follow by hand
+    # three workers; coordinate 0 sent by all, 1 by two, 2 by one, 3 by none
+    recs = _recs(3, 1, 2, [[0, 1], [0, 1], [0, 2]], [[3.0, 1.0], [6.0, -2.0], [-3.0, 8.0]])
+    x = np.zeros((1, M))
+    want_sum = np.array([6.0, -1.0, 8.0, 0.0])
+    want_mean = want_sum / 3.0
+    want_cnt = np.array([6.0 / 3, -1.0 / 2, 8.0 / 1, 0.0])  # 0/0 = 0 at coordinate 3
+    for agg, want in [(orc.AGG_SUM, want_sum), (orc.AGG_MEAN, want_mean), (orc.AGG_COUNT_MEAN, want_cnt)]:
+        out = orc.decode_chunks(recs, x, s, rows, 1.0, 0.0, agg=agg, phi=orc.PHI_IDENTITY)
+        R = scipy.fft.idct(want, type=2, norm="ortho")
+        assert np.max(np.abs(out["R"][0] - R)) < 1e-14
+        assert np.max(np.abs(out["x_new"][0] - (x[0] - R))) < 1e-14  # phi = identity, lr = 1, wd = 0
+
+
+def test_count_mean_limits_and_identity_update():
+    s, rows, k, W = 8, 8, 5, 4
+    M = s * s
+    rng = np.random.default_rng(41)
+    x = rng.standard_normal((2, M)) * 0.02
+    # disjoint index sets: count-normalised == sum; identical index sets: count-normalised == mean
+    dis = np.zeros((W, 2, k), dtype=orc.RECORD_DTYPE)
+    same = np.zeros((W, 2, k), dtype=orc.RECORD_DTYPE)
+    for w in range(W):
+        for c in range(2):
+            dis[w, c]["idx"] = np.arange(w * k, (w + 1) * k)
+            same[w, c]["idx"] = np.arange(3, 3 + k)
+            dis[w, c]["val"] = rng.standard_normal(k).astype(np.float32)
+            same[w, c]["val"] = rng.standard_normal(k).astype(np.float32)
+    a = orc.decode_chunks(dis, x, s, rows, 1e-3, 0.1, agg=orc.AGG_COUNT_MEAN)
+    b = orc.decode_chunks(dis, x, s, rows, 1e-3, 0.1, agg=orc.AGG_SUM)
+    assert np.array_equal(a["R"], b["R"]) and np.array_equal(a["x_new"], b["x_new"])
+    a = orc.decode_chunks(same, x, s, rows, 1e-3, 0.1, agg=orc.AGG_COUNT_MEAN, phi=orc.PHI_IDENTITY)
+    b = orc.decode_chunks(same, x, s, rows, 1e-3, 0.1, agg=orc.AGG_MEAN, phi=orc.PHI_IDENTITY)
+    assert np.max(np.abs(a["R"] - b["R"])) < 1e-15
+    # the mean has the sign of the sum; identity applies R itself: x - lr (R + wd x)
+    c = orc.decode_chunks(same, x, s, rows, 1e-3, 0.1, agg=orc.AGG_SUM)
+    d = orc.decode_chunks(same, x, s, rows, 1e-3, 0.1, agg=orc.AGG_MEAN)
+    assert np.array_equal(c["x_new"], d["x_new"])
+    assert np.max(np.abs(b["x_new"] - (x - 1e-3 * (b["R"] + 0.1 * x)))) < 1e-16
+    assert np.max(np.abs(b["R"] - c["R"] / W)) < 1e-15
