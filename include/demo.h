@@ -188,6 +188,19 @@ demo_status demo_set_lr(demo_ctx *ctx, float lr);
  * next demo_compress.  Errors: INVALID_ARG. */
 demo_status demo_set_alpha(demo_ctx *ctx, float alpha);
 
+/* How demo_decode_apply combines the W payloads and which transform phi it applies (Section 2.1):
+ *   aggregation  DEMO_AGG_SUM         S = sum_w Q^w                         (Algorithm 1; default)
+ *                DEMO_AGG_MEAN        S = (1/W) sum_w Q^w                   (AvgAllGather)
+ *                DEMO_AGG_COUNT_MEAN  S[i] = sum_w Q^w[i] / #{w : i sent},  0/0 = 0
+ *                                     (appendix algorithm "Sparse Top-k Averaging")
+ *   phi          DEMO_PHI_SIGN        x <- x - lr (sign(R) + wd x)          (Signum; default)
+ *                DEMO_PHI_IDENTITY    x <- x - lr (R + wd x)                (SGD-style)
+ * with R = IDCT(S).  Takes effect for the next demo_decode_apply.
+ * Errors: INVALID_ARG; UNSUPPORTED (count-normalised mean with more than 65535 workers). */
+typedef enum { DEMO_AGG_SUM = 0, DEMO_AGG_MEAN = 1, DEMO_AGG_COUNT_MEAN = 2 } demo_aggregation;
+typedef enum { DEMO_PHI_SIGN = 0, DEMO_PHI_IDENTITY = 1 } demo_phi;
+demo_status demo_set_decode_mode(demo_ctx *ctx, int32_t aggregation, int32_t phi);
+
 /* Select the kernel family (see demo_path).  Errors: INVALID_ARG. */
 demo_status demo_set_path(demo_ctx *ctx, int32_t path);
 

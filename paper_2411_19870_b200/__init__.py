@@ -6,7 +6,12 @@ This package only marshals arguments: every step of the path runs in the library
 from .binding import (  # noqa: F401
     DEMO_BF16,
     DEMO_F32,
+    DEMO_AGG_COUNT_MEAN,
+    DEMO_AGG_MEAN,
+    DEMO_AGG_SUM,
     DEMO_PATH_AUTO,
+    DEMO_PHI_IDENTITY,
+    DEMO_PHI_SIGN,
     DEMO_PATH_GENERIC,
     DemoConfig,
     DemoError,

@@ -16,11 +16,13 @@ LIB_PATH = os.path.join(HERE, "libdemo_b200.so")
 
 DEMO_F32, DEMO_BF16 = 0, 1
 DEMO_PATH_AUTO, DEMO_PATH_GENERIC = 0, 1
+DEMO_AGG_SUM, DEMO_AGG_MEAN, DEMO_AGG_COUNT_MEAN = 0, 1, 2
+DEMO_PHI_SIGN, DEMO_PHI_IDENTITY = 0, 1
 RECORD_BYTES = 8
 
 EXPORTS = [
     "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
-    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
 ]
 
@@ -77,6 +79,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_set_lr.restype = i32
     lib.demo_set_alpha.argtypes = [vp, ctypes.c_float]
     lib.demo_set_alpha.restype = i32
+    lib.demo_set_decode_mode.argtypes = [vp, i32, i32]
+    lib.demo_set_decode_mode.restype = i32
     lib.demo_set_path.argtypes = [vp, i32]
     lib.demo_set_path.restype = i32
     lib.demo_launch_count.argtypes = [vp]
@@ -213,6 +217,11 @@ class DemoTransform:
         st = self.lib.demo_set_alpha(self._ctx, alpha)
         if st != 0:
             raise DemoError(st, "demo_set_alpha")
+
+    def set_decode_mode(self, aggregation: int, phi: int) -> None:
+        st = self.lib.demo_set_decode_mode(self._ctx, aggregation, phi)
+        if st != 0:
+            raise DemoError(st, "demo_set_decode_mode")
 
     def set_path(self, path: int) -> None:
         st = self.lib.demo_set_path(self._ctx, path)

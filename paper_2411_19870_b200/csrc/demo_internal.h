@@ -53,6 +53,9 @@ struct DemoDecodeArgs {
     float wd;
     int *status;
     const void *tmap_x;  // optional tensor maps of the parameter tensors (see DemoCompressArgs)
+    int agg;          // 0 sum, 1 mean over workers, 2 per-coordinate count-normalised mean (0/0 = 0)
+    int phi;          // 0 sign, 1 identity
+    float agg_scale;  // 1/W for the mean, else 1 (only the identity update sees it)
 };
 
 // Launchers (defined in the kernel translation units).  `s` is the chunk size, `two_d` selects

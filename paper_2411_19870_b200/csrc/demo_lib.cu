@@ -18,6 +18,7 @@ struct demo_ctx {
     int n_tensors = 0;
     int path = DEMO_PATH_AUTO;
     float alpha = 1.0f;  // momentum-subtraction coefficient
+    int aggregation = DEMO_AGG_SUM, phi = DEMO_PHI_SIGN;
     long long launches = 0;
     std::vector<demo_tensor_desc> descs;
     std::vector<long long> first_record, n_chunks, n_elems;
@@ -418,6 +419,9 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     a.wd = ctx->cfg.weight_decay;
     a.status = ctx->d_status;
     a.tmap_x = ctx->encode ? ctx->d_tm_x : nullptr;
+    a.agg = ctx->aggregation;
+    a.phi = ctx->phi;
+    a.agg_scale = (ctx->aggregation == DEMO_AGG_MEAN) ? 1.0f / (float)W : 1.0f;
     const int s = ctx->cfg.chunk;
     if (ctx->n2d) {
         a.entries = ctx->d_entries2d;
@@ -493,6 +497,18 @@ demo_status demo_set_alpha(demo_ctx *ctx, float alpha)
 {
     if (!ctx || !(alpha >= 0.0f && alpha <= 1.0f)) return DEMO_ERR_INVALID_ARG;
     ctx->alpha = alpha;
+    return DEMO_OK;
+}
+
+demo_status demo_set_decode_mode(demo_ctx *ctx, int32_t aggregation, int32_t phi)
+{
+    if (!ctx) return DEMO_ERR_INVALID_ARG;
+    if (aggregation != DEMO_AGG_SUM && aggregation != DEMO_AGG_MEAN && aggregation != DEMO_AGG_COUNT_MEAN)
+        return DEMO_ERR_INVALID_ARG;
+    if (phi != DEMO_PHI_SIGN && phi != DEMO_PHI_IDENTITY) return DEMO_ERR_INVALID_ARG;
+    if (aggregation == DEMO_AGG_COUNT_MEAN && ctx->cfg.num_workers > 65535) return DEMO_ERR_UNSUPPORTED;
+    ctx->aggregation = aggregation;
+    ctx->phi = phi;
     return DEMO_OK;
 }
 

@@ -605,10 +605,12 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
     }
 }
 
+// Bytes of one decode slot: the tile, the mbarrier and -- for the count-normalised mean -- one
+// 16-bit sender count per coordinate.
 template <int S>
-constexpr size_t decode_slot_bytes()
+__host__ __device__ constexpr size_t decode_slot_bytes(bool counts)
 {
-    return ((size_t)S * Cfg<S>::XS * 4 + 16 + 127) / 128 * 128;
+    return ((size_t)S * Cfg<S>::XS * 4 + 16 + (counts ? (size_t)S * S * 2 : 0) + 127) / 128 * 128;
 }
 
 template <int S, bool TMAP, int THREADS>
@@ -619,13 +621,15 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
     constexpr int M = S * S;
     extern __shared__ __align__(128) unsigned char smem_all[];
     const int slot = threadIdx.x / S;
-    unsigned char *smem_raw = smem_all + (size_t)slot * decode_slot_bytes<S>();
+    const bool counts = a.agg == 2;
+    unsigned char *smem_raw = smem_all + (size_t)slot * decode_slot_bytes<S>(counts);
     const SlotBarrier<S> sb{slot + 1};
     // One tile per slot: the aggregate S, then the row-stage output, and -- once column t has been
     // read back into registers -- the staging area of the x tile, fetched behind the second transform.
     float *St = reinterpret_cast<float *>(smem_raw);  // [S*XS]
     float *Xt = St;                                   // [S*S] (aliases St)
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XS);
+    unsigned short *Cn = reinterpret_cast<unsigned short *>(bar_mem + 2);  // [S*S] senders per coordinate (agg == 2)
 
     const int t = threadIdx.x % S;
     const uint32_t bar = smem_u32(bar_mem);
@@ -643,6 +647,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
     bool failed = false;
     const unsigned lr_bits = __float_as_uint(a.lr);
     const float decay = 1.f - a.lr * a.wd;
+    const float neg_lr_scale = -a.lr * a.agg_scale;
 
     const long long stride = (long long)gridDim.x * NCH;
     long long c = (long long)blockIdx.x * NCH + slot;
@@ -669,6 +674,8 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
             float4 *row = reinterpret_cast<float4 *>(St + t * XS);
 #pragma unroll
             for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (counts)
+                for (int v = 0; v < S; ++v) Cn[t * S + v] = 0;
         }
         sb.sync();
         // S = sum over workers in worker order; a barrier per worker fixes the order of additions.
@@ -684,14 +691,22 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
                 for (int j = 0; j < 8; ++j) {
                     if (w0 + j < a.W) {
                         if (mine) {
-                            if ((unsigned)r[j].idx < (unsigned)M)
+                            if ((unsigned)r[j].idx < (unsigned)M) {
                                 St[(r[j].idx >> C::LOG2S) * XS + (r[j].idx & (S - 1))] += r[j].val;
-                            else
+                                if (counts) Cn[r[j].idx] += 1;
+                            } else {
                                 atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                            }
                         }
                         sb.sync();
                     }
                 }
+            }
+        }
+        if (counts) {  // Sparse Top-k Averaging: sum / number of senders, 0/0 = 0 (row t is this thread's)
+            for (int v = 0; v < S; ++v) {
+                const unsigned short n = Cn[t * S + v];
+                if (n > 1) St[t * XS + v] = St[t * XS + v] / (float)n;
             }
         }
         // Two inverse passes through one copy of the unrolled transform (rolled loop): pass 0 along
@@ -751,6 +766,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
             const float rv = r[i];
             float stepv = __uint_as_float(lr_bits ^ (~__float_as_uint(rv) & 0x80000000u));
             stepv = (rv == 0.f) ? 0.f : stepv;
+            if (a.phi) stepv = rv * neg_lr_scale;  // phi = identity: -lr * R (R / W for the mean)
             x[base + (size_t)i * te.n1 + t] = fmaf(Xt[i * S + t], decay, stepv);
         }
         sb.sync();  // the tile is free again
@@ -803,7 +819,7 @@ cudaError_t launch_decode(const DemoDecodeArgs &a, int sm_count, cudaStream_t st
 {
     constexpr int TH = DECODE_THREADS;
     constexpr int NCH = TH / S;
-    const size_t smem = decode_slot_bytes<S>() * NCH;
+    const size_t smem = decode_slot_bytes<S>(a.agg == 2) * NCH;
     if (a.tmap_x != nullptr)
         return launch(decode_fast_kernel<S, true, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
     return launch(decode_fast_kernel<S, false, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);

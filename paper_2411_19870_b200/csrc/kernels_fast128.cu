@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
     }
 }
 
-constexpr size_t decode128_smem() { return (size_t)S * XS * 4 + 16; }
+constexpr size_t decode128_smem(bool counts) { return (size_t)S * XS * 4 + 16 + (counts ? (size_t)M * 2 : 0); }
 
 __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeArgs a)
 {
@@ -337,6 +337,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
     float *St = reinterpret_cast<float *>(smem_raw);  // [128*132] aggregate / intermediate; later the x tile [128*128]
     float *Xt = St;
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XS);
+    unsigned short *Cn = reinterpret_cast<unsigned short *>(bar_mem + 2);  // [M] senders per coordinate (agg == 2)
 
     const int tid = threadIdx.x, h = tid >> 7, j = tid & 127;
     const uint32_t bar = smem_u32(bar_mem);
@@ -351,6 +352,8 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
     unsigned phase = 0;
     const unsigned lr_bits = __float_as_uint(a.lr);
     const float decay = 1.f - a.lr * a.wd;
+    const float neg_lr_scale = -a.lr * a.agg_scale;
+    const bool counts = a.agg == 2;
 
     for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
         cur.seek(a.entries, a.n_entries, c);
@@ -365,6 +368,8 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
         if (tid == 0) tma_prefetch_2d(tm_x, k1 * S, k0 * S);
 
         for (int i = tid; i < S * XS / 4; i += THREADS) reinterpret_cast<float4 *>(St)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (counts)
+            for (int i = tid; i < M; i += THREADS) Cn[i] = 0;
         __syncthreads();
         // S = sum over workers in worker order (a barrier per worker fixes the order of additions)
         for (int kb = 0; kb < k_eff; kb += THREADS) {
@@ -378,15 +383,24 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
                 for (int q = 0; q < 8; ++q) {
                     if (w0 + q < a.W) {
                         if (mine) {
-                            if ((unsigned)r[q].idx < (unsigned)M)
+                            if ((unsigned)r[q].idx < (unsigned)M) {
                                 St[(r[q].idx >> 7) * XS + (r[q].idx & 127)] += r[q].val;
-                            else
+                                if (counts) Cn[r[q].idx] += 1;
+                            } else {
                                 atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                            }
                         }
                         __syncthreads();
                     }
                 }
             }
+        }
+        if (counts) {  // Sparse Top-k Averaging: sum / number of senders, 0/0 = 0
+            for (int i = tid; i < M; i += THREADS) {
+                const unsigned short n = Cn[i];
+                if (n > 1) St[(i >> 7) * XS + (i & 127)] /= (float)n;
+            }
+            __syncthreads();
         }
         // two inverse passes (rolled): pass 0 along row j, pass 1 down column j
         float in[H], out[H];
@@ -435,6 +449,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
             const float rv = out[n];
             float stepv = __uint_as_float(lr_bits ^ (~__float_as_uint(rv) & 0x80000000u));
             stepv = (rv == 0.f) ? 0.f : stepv;
+            if (a.phi) stepv = rv * neg_lr_scale;  // phi = identity
             x[base + (size_t)row * te.n1 + j] = fmaf(Xt[row * S + j], decay, stepv);
         }
         fence_proxy_async();
@@ -472,5 +487,5 @@ cudaError_t demo_launch_compress_fast128(const DemoCompressArgs &a, int sm_count
 cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
 {
     if (!a.tmap_x) return cudaErrorNotSupported;
-    return launch128(decode_fast128_kernel, decode128_smem(), a.n_chunks, sm_count, stream, &a);
+    return launch128(decode_fast128_kernel, decode128_smem(a.agg == 2), a.n_chunks, sm_count, stream, &a);
 }

@@ -254,7 +254,9 @@ __global__ void __launch_bounds__(GEN_THREADS) decode_generic_kernel(DemoDecodeA
     extern __shared__ float smem[];
     float *St = smem;
     float *X1 = St + M;
+    unsigned short *Cn = reinterpret_cast<unsigned short *>(X1 + M);  // [M] senders per coordinate (agg == 2 only)
     const int tid = threadIdx.x;
+    const bool counts = a.agg == 2;
 
     for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
         const DemoTensorEntry te = a.entries[demo_find_entry(a.entries, a.n_entries, c)];
@@ -266,7 +268,10 @@ __global__ void __launch_bounds__(GEN_THREADS) decode_generic_kernel(DemoDecodeA
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + lc * (long long)k_eff;
 
-        for (int i = tid; i < M; i += GEN_THREADS) St[i] = 0.f;
+        for (int i = tid; i < M; i += GEN_THREADS) {
+            St[i] = 0.f;
+            if (counts) Cn[i] = 0;
+        }
         __syncthreads();
         // aggregate: S = sum over workers, in worker order (Decompress&Aggregate); indices are
         // unique inside one worker's chunk, so a barrier per worker fixes the summation order
@@ -274,10 +279,19 @@ __global__ void __launch_bounds__(GEN_THREADS) decode_generic_kernel(DemoDecodeA
             const DemoRecord *rec = a.payloads[w] + rec_off;
             for (int i = tid; i < k_eff; i += GEN_THREADS) {
                 const DemoRecord r = rec[i];
-                if ((unsigned)r.idx < (unsigned)M)
+                if ((unsigned)r.idx < (unsigned)M) {
                     St[r.idx] += r.val;
-                else
+                    if (counts) Cn[r.idx] += 1;
+                } else {
                     atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                }
+            }
+            __syncthreads();
+        }
+        if (counts) {  // Sparse Top-k Averaging: sum / number of senders, 0/0 = 0
+            for (int i = tid; i < M; i += GEN_THREADS) {
+                const unsigned short n = Cn[i];
+                if (n > 1) St[i] = St[i] / (float)n;
             }
             __syncthreads();
         }
@@ -288,7 +302,7 @@ __global__ void __launch_bounds__(GEN_THREADS) decode_generic_kernel(DemoDecodeA
             const int r = i / S, j = i - r * S;
             const size_t off = base + (size_t)r * te.n1 + j;
             const float rv = R[i];
-            const float sg = (float)((rv > 0.f) - (rv < 0.f));
+            const float sg = a.phi ? rv * a.agg_scale : (float)((rv > 0.f) - (rv < 0.f));
             const float xv = x[off];
             x[off] = fmaf(-a.lr, fmaf(a.wd, xv, sg), xv);
         }
@@ -328,9 +342,9 @@ template <int S>
 cudaError_t decode_dispatch(int two_d, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
 {
     if (two_d)
-        return launch_persistent(decode_generic_kernel<S, S>, 2 * S * S * sizeof(float), a.n_chunks, sm_count,
+        return launch_persistent(decode_generic_kernel<S, S>, 2 * S * S * sizeof(float) + S * S * 2, a.n_chunks, sm_count,
                                  stream, &a);
-    return launch_persistent(decode_generic_kernel<S, 1>, 2 * S * sizeof(float), a.n_chunks, sm_count, stream, &a);
+    return launch_persistent(decode_generic_kernel<S, 1>, 2 * S * sizeof(float) + S * 2, a.n_chunks, sm_count, stream, &a);
 }
 
 }  // namespace
@@ -524,6 +538,9 @@ extern "C" demo_status demo_decode_apply_static(const demo_config *cfg, const de
         a.wd = cfg->weight_decay;
         a.status = reinterpret_cast<int *>(base + OFF_STATUS);
         a.tmap_x = nullptr;
+        a.agg = 0;
+        a.phi = 0;
+        a.agg_scale = 1.f;
         cudaError_t err = cudaSuccess;
         if (n2d) {
             a.entries = reinterpret_cast<const DemoTensorEntry *>(base + OFF_ENTRIES);

@@ -135,10 +135,20 @@ def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, repor
     return ref
 
 
-def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Report, what=""):
+def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Report, what="", agg=0, phi=0):
     """recs_gpu [W, n, k_eff] GPU-written records; x_* float64 [n, M]."""
-    ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd)
+    ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd, agg=agg, phi=phi)
     R = ref["R"]
+    if phi == orc.PHI_IDENTITY:
+        # no sign decision: the update is linear in R; the tolerance follows R's fp32 rounding
+        x_ref = ref["x_new"]
+        rinf = np.maximum(1.0, np.max(np.abs(R), axis=1, keepdims=True))
+        tol = RTOL * np.abs(x_ref) + ATOL * np.maximum(1.0, np.max(np.abs(x_ref), axis=1, keepdims=True)) + lr * (
+            RTOL * np.abs(R) + ATOL * rinf)
+        ok = np.abs(x_after - x_ref) <= tol
+        assert ok.all(), "%s: %d parameter(s) outside tolerance (identity update)" % (what, (~ok).sum())
+        report.add("decode_chunks", x_before.shape[0])
+        return ref
     rinf = np.maximum(1.0, np.max(np.abs(R), axis=1, keepdims=True))
     exempt = np.abs(R) < SIGN_EXEMPT * rinf
     x_ref = ref["x_new"]
@@ -164,7 +174,7 @@ def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Re
 class Runner:
     """Drives a workload through the C ABI and checks sampled (or all) chunks every step."""
 
-    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0, alpha=None):
+    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0, alpha=None, agg=0, phi=0):
         import paper_2411_19870_b200 as demo
         from paper_2411_19870_b200 import inputs
 
@@ -176,6 +186,9 @@ class Runner:
                                      device=self.device.index or 0)
         if path is not None:
             self.tr.set_path(path)
+        self.agg, self.phi = agg, phi
+        if agg or phi:
+            self.tr.set_decode_mode(agg, phi)
         self.alpha = 1.0
         if alpha is not None:
             self.tr.set_alpha(alpha)
@@ -219,7 +232,7 @@ class Runner:
                 recs = np.stack([gather_records(self.payloads[w], first, k_eff, self.ids[t])
                                  for w in range(wl.num_workers)])
                 check_decode_chunks(recs, xb[t], gather_tiles(self.params[t], s, self.ids[t]), s, rows, self.lr,
-                                    self.wd, self.report, what="decode t%d" % t)
+                                    self.wd, self.report, what="decode t%d" % t, agg=self.agg, phi=self.phi)
         st = self.tr.device_status()
         assert st == 0, "device status %d (%s)" % (st, self.demo.demo_status_string(st))
 

@@ -70,6 +70,7 @@ def test_null_arguments(lib):
     assert lib.demo_set_lr(None, 1.0) == 1
     assert lib.demo_set_path(None, 0) == 1
     assert lib.demo_set_alpha(None, 0.5) == 1
+    assert lib.demo_set_decode_mode(None, 0, 0) == 1
     assert lib.demo_device_status(None, None) == 1
     assert lib.demo_launch_count(None) == 0
     lib.demo_free(None)  # NULL-safe

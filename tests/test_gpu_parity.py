@@ -297,3 +297,19 @@ def test_alpha_scaled_momentum_subtraction(s, alpha):
             r2.tr.set_alpha(1.5)
         finally:
             r2.close()
+
+
+@pytest.mark.parametrize("s", [8, 64, 128])
+@pytest.mark.parametrize("agg,phi", [(1, 0), (2, 0), (0, 1), (1, 1), (2, 1)])
+def test_aggregation_and_phi_variants(s, agg, phi):
+    """Mean / count-normalised aggregation (Sparse Top-k Averaging) and phi = identity, both kernel
+    families; workers share gradient structure so that coordinates collide across workers."""
+    shapes = [(2 * s, 2 * s), (2 * s,)]
+    wl = inputs.Workload("agg", shapes, chunk=s, topk=max(2, s // 4), num_workers=5, grad_kind="normal", grad_std=0.01)
+    for path in PATHS:
+        r = parity.Runner(wl, max_chunks=10**9, path=path, agg=agg, phi=phi)
+        base = [g for g in r.streams[0].next()]
+        grads = [[(b.float() + 0.3 * o.float()).to(b.dtype) for b, o in zip(base, st.next())] for st in r.streams]
+        r.step(grads=grads)
+        r.step(grads=grads)
+        r.close()
