@@ -201,6 +201,13 @@ typedef enum { DEMO_AGG_SUM = 0, DEMO_AGG_MEAN = 1, DEMO_AGG_COUNT_MEAN = 2 } de
 typedef enum { DEMO_PHI_SIGN = 0, DEMO_PHI_IDENTITY = 1 } demo_phi;
 demo_status demo_set_decode_mode(demo_ctx *ctx, int32_t aggregation, int32_t phi);
 
+/* Self-test of the device-side failure path: enqueue a one-CTA kernel that waits, for at most
+ * limit_cycles SM clock cycles (1 .. 2e9), on a barrier that nothing completes -- the situation a lost
+ * tile copy would create -- using the same bounded wait as the production kernels.  The kernel records
+ * DEMO_ERR_TIMEOUT in the sticky device status and returns; the context stays usable.  Nothing is
+ * trapped, faulted or left spinning.  Errors: INVALID_ARG, CUDA. */
+demo_status demo_selftest_bounded_wait(demo_ctx *ctx, int64_t limit_cycles, void *cuda_stream);
+
 /* Select the kernel family (see demo_path).  Errors: INVALID_ARG. */
 demo_status demo_set_path(demo_ctx *ctx, int32_t path);
 

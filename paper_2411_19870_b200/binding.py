@@ -22,7 +22,7 @@ RECORD_BYTES = 8
 
 EXPORTS = [
     "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
-    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_selftest_bounded_wait", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
 ]
 
@@ -81,6 +81,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_set_alpha.restype = i32
     lib.demo_set_decode_mode.argtypes = [vp, i32, i32]
     lib.demo_set_decode_mode.restype = i32
+    lib.demo_selftest_bounded_wait.argtypes = [vp, i64, vp]
+    lib.demo_selftest_bounded_wait.restype = i32
     lib.demo_set_path.argtypes = [vp, i32]
     lib.demo_set_path.restype = i32
     lib.demo_launch_count.argtypes = [vp]
@@ -222,6 +224,11 @@ class DemoTransform:
         st = self.lib.demo_set_decode_mode(self._ctx, aggregation, phi)
         if st != 0:
             raise DemoError(st, "demo_set_decode_mode")
+
+    def selftest_bounded_wait(self, limit_cycles: int, stream=None) -> None:
+        st = self.lib.demo_selftest_bounded_wait(self._ctx, int(limit_cycles), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_selftest_bounded_wait")
 
     def set_path(self, path: int) -> None:
         st = self.lib.demo_set_path(self._ctx, path)

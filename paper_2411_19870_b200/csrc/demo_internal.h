@@ -72,6 +72,10 @@ cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count
 cudaError_t demo_launch_compress_fast128(const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
 cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream);
 
+// Self-test of the bounded wait (kernels_fast.cu): one CTA waits, for at most `limit_cycles`, on an
+// mbarrier that nothing completes, records DEMO_DEV_TIMEOUT in *status and returns.
+cudaError_t demo_launch_wait_selftest(int *status, long long limit_cycles, cudaStream_t stream);
+
 // Locate the tensor that owns chunk id c: the last entry with chunk_begin <= c.
 __device__ __forceinline__ int demo_find_entry(const DemoTensorEntry *entries, int n, long long c)
 {

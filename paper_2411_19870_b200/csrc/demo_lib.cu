@@ -512,6 +512,19 @@ demo_status demo_set_decode_mode(demo_ctx *ctx, int32_t aggregation, int32_t phi
     return DEMO_OK;
 }
 
+demo_status demo_selftest_bounded_wait(demo_ctx *ctx, int64_t limit_cycles, void *cuda_stream)
+{
+    if (!ctx || limit_cycles < 1 || limit_cycles > 2000000000LL) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    if (demo_launch_wait_selftest(ctx->d_status, limit_cycles, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return DEMO_OK;
+}
+
 demo_status demo_set_path(demo_ctx *ctx, int32_t path)
 {
     if (!ctx || (path != DEMO_PATH_AUTO && path != DEMO_PATH_GENERIC)) return DEMO_ERR_INVALID_ARG;

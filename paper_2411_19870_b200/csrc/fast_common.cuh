@@ -33,12 +33,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity)
     return ok != 0;
 }
 // Bounded wait: false if the phase did not complete within WAIT_LIMIT_CYCLES.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, unsigned parity, long long limit = WAIT_LIMIT_CYCLES)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }

@@ -825,7 +825,29 @@ cudaError_t launch_decode(const DemoDecodeArgs &a, int sm_count, cudaStream_t st
     return launch(decode_fast_kernel<S, false, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
 }
 
+// One CTA arms an mbarrier with a transaction count that no copy will ever satisfy and waits for it
+// with the same bounded wait the production kernels use.
+__global__ void wait_selftest_kernel(int *status, long long limit_cycles)
+{
+    __shared__ __align__(8) unsigned long long bar_mem;
+    const uint32_t bar = smem_u32(&bar_mem);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        fence_proxy_async();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_expect_tx(bar, 16);  // 16 bytes that never arrive
+    const bool arrived = mbar_wait_bounded(bar, 0, limit_cycles);
+    if (!__syncthreads_and(arrived) && threadIdx.x == 0) atomicMax(status, DEMO_DEV_TIMEOUT);
+}
+
 }  // namespace
+
+cudaError_t demo_launch_wait_selftest(int *status, long long limit_cycles, cudaStream_t stream)
+{
+    wait_selftest_kernel<<<1, 64, 0, stream>>>(status, limit_cycles);
+    return cudaGetLastError();
+}
 
 bool demo_fast_supported(int s) { return s == 128 || s == 64 || s == 32; }
 

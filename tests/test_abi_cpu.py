@@ -71,6 +71,7 @@ def test_null_arguments(lib):
     assert lib.demo_set_path(None, 0) == 1
     assert lib.demo_set_alpha(None, 0.5) == 1
     assert lib.demo_set_decode_mode(None, 0, 0) == 1
+    assert lib.demo_selftest_bounded_wait(None, 1000, None) == 1
     assert lib.demo_device_status(None, None) == 1
     assert lib.demo_launch_count(None) == 0
     lib.demo_free(None)  # NULL-safe

@@ -313,3 +313,16 @@ def test_aggregation_and_phi_variants(s, agg, phi):
         r.step(grads=grads)
         r.step(grads=grads)
         r.close()
+
+
+def test_bounded_wait_expires_into_a_status_and_the_context_survives():
+    """Failure detection without a GPU fault: a wait that nothing satisfies runs out after ~1 ms, the
+    kernel returns, the sticky status says TIMEOUT, and the same context then computes correctly."""
+    wl = inputs.small_decoder(num_workers=2)
+    r = parity.Runner(wl, max_chunks=16)
+    r.step()
+    r.tr.selftest_bounded_wait(2_000_000)  # ~1 ms of SM clock
+    assert r.tr.device_status() == 7       # DEMO_ERR_TIMEOUT ...
+    assert r.tr.device_status() == 0       # ... reported once, then cleared
+    r.step()                               # parity-checked step on the same context
+    r.close()
