@@ -124,8 +124,10 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
  * demo_step_host -- one whole optimizer step driven from HOST gradient buffers: for every worker
  * copy its gradients host->device into the caller's device staging tensors, compress, then decode
  * and apply, then (if host_payloads_out is not NULL) copy all W payloads device->host.  Everything
- * is enqueued on cuda_stream; the host buffers must stay valid until the stream has drained
- * (use pinned memory for the copies to be asynchronous).
+ * is ordered with cuda_stream; the host buffers must stay valid until the stream has drained
+ * (use pinned memory for the copies to be asynchronous).  The gradient copies run on an internal
+ * stream, created together with W events on the first call, so that the copy of worker w+1 overlaps
+ * the compress of worker w; they start only after the work already queued on cuda_stream.
  *   host_grads         host array [W * n_tensors] of HOST pointers (worker-major)
  *   dev_grads          host array [W * n_tensors] of DEVICE pointers receiving the copies
  *   momentum           host array [W * n_tensors] of DEVICE pointers (fp32)

@@ -50,6 +50,12 @@ struct demo_ctx {
     CUtensorMap *d_tm_g = nullptr, *d_tm_m = nullptr;  // [W][T]
     CUtensorMap *d_tm_x = nullptr;                     // [T]
     std::vector<CUtensorMap> h_tm;                     // staging, [T]
+
+    // demo_step_host: host->device gradient copies run on their own stream so that the copy of worker
+    // w+1 overlaps the compress of worker w (created on first use)
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_start = nullptr;
+    std::vector<cudaEvent_t> ev_copied;  // [W]
 };
 
 namespace {
@@ -124,6 +130,10 @@ void release(demo_ctx *c)
     cudaFree(c->d_tm_g);
     cudaFree(c->d_tm_m);
     cudaFree(c->d_tm_x);
+    for (cudaEvent_t e : c->ev_copied)
+        if (e) cudaEventDestroy(e);
+    if (c->ev_start) cudaEventDestroy(c->ev_start);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     delete c;
 }
 
@@ -459,14 +469,41 @@ demo_status demo_step_host(demo_ctx *ctx, const void *const *host_grads, void *c
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DEMO_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!ctx->copy_stream) {
+        bool ok = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) == cudaSuccess;
+        try {
+            ctx->ev_copied.assign((size_t)W, nullptr);
+        } catch (const std::bad_alloc &) {
+            ok = false;
+        }
+        for (int w = 0; ok && w < W; ++w)
+            ok = cudaEventCreateWithFlags(&ctx->ev_copied[w], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            return DEMO_ERR_ALLOC;
+        }
+    }
+    // the copies start once everything already queued on the caller's stream (the previous step, which
+    // reads the staging tensors) has finished, then run ahead of the compress calls
+    bool ok = cudaEventRecord(ctx->ev_start, stream) == cudaSuccess &&
+              cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_start, 0) == cudaSuccess;
+    for (int w = 0; ok && w < W; ++w) {
+        const size_t row = (size_t)w * T;
+        for (int t = 0; ok && t < T; ++t)
+            ok = cudaMemcpyAsync(dev_grads[row + t], host_grads[row + t], (size_t)ctx->n_elems[t] * gsize,
+                                 cudaMemcpyHostToDevice, ctx->copy_stream) == cudaSuccess;
+        ok = ok && cudaEventRecord(ctx->ev_copied[w], ctx->copy_stream) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
     for (int w = 0; w < W; ++w) {
         const size_t row = (size_t)w * T;
-        for (int t = 0; t < T; ++t) {
-            if (cudaMemcpyAsync(dev_grads[row + t], host_grads[row + t], (size_t)ctx->n_elems[t] * gsize,
-                                cudaMemcpyHostToDevice, stream) != cudaSuccess) {
-                cudaGetLastError();
-                return DEMO_ERR_CUDA;
-            }
+        if (cudaStreamWaitEvent(stream, ctx->ev_copied[w], 0) != cudaSuccess) {
+            cudaGetLastError();
+            return DEMO_ERR_CUDA;
         }
         demo_status st = demo_compress(ctx, w, const_cast<const void *const *>(dev_grads + row), momentum + row,
                                        payloads[w], cuda_stream);
