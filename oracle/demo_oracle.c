@@ -26,7 +26,9 @@
  *   - exactly k_eff coefficients per chunk (||Q_hat||_0 = k, Section 2.1); ties at the
  *     k-th magnitude go to the lowest flat index;
  *   - sign(0) = 0 (the sign lemmas of the appendix treat sign(y) = 0 as a legal case);
- *   - the DCT is the orthonormal DCT-II ("unitary", P^T = P^-1, appendix Sec. B.1.2).
+ *   - the DCT is the orthonormal DCT-II ("unitary", P^T = P^-1, appendix Sec. B.1.2);
+ *   - any other orthonormal basis (identity, Gram-Schmidt of a Gaussian matrix: Section 4.2) is passed
+ *     in as an s x s matrix whose ROWS are the basis vectors, and is used for both axes of a 2-D chunk.
  *
  * Parity pins live in tests/test_oracle_pins.py (closed forms, scipy's DCT, Parseval,
  * brute force on 8x8, the paper's 128x512 blocking example, the sqrt(1-k/M) bound with its
@@ -60,6 +62,46 @@ void oracle_dct_matrix(int s, double *C)
         for (int n = 0; n < s; ++n)
             C[(size_t)u * s + n] = a * cos(pi * (double)(2 * n + 1) * (double)u / (2.0 * (double)s));
     }
+}
+
+/* The transform of a chunk is any orthonormal s x s matrix P with rows as basis vectors (Q = P B P^T,
+ * inverse P^T Q P): the DCT above, the identity ("no transformation") or a random orthonormal matrix
+ * (Section 4.2, "Choice of Linear Projections").  `basis` NULL selects the DCT. */
+static void chunk_basis(int s, const double *basis, double *C)
+{
+    if (basis)
+        memcpy(C, basis, sizeof(double) * (size_t)s * s);
+    else
+        oracle_dct_matrix(s, C);
+}
+
+/* Gram-Schmidt process on the rows of G (s x s, entries drawn from N(0,1) by the caller with the step
+ * number as the seed, Section 4.2): row j of P is row j of G minus its components along rows 0..j-1 of
+ * P, scaled to unit length.  The components are removed one after the other from the running vector
+ * (the "modified" ordering, identical in exact arithmetic).  Returns -1 when a row has no component
+ * left (G singular to rounding), 0 otherwise. */
+int oracle_gram_schmidt(int s, const double *G, double *P)
+{
+    for (int j = 0; j < s; ++j) {
+        double *p = P + (size_t)j * s;
+        double scale = 0.0;
+        for (int n = 0; n < s; ++n) {
+            p[n] = G[(size_t)j * s + n];
+            scale += p[n] * p[n];
+        }
+        for (int i = 0; i < j; ++i) {
+            const double *q = P + (size_t)i * s;
+            double dot = 0.0;
+            for (int n = 0; n < s; ++n) dot += p[n] * q[n];
+            for (int n = 0; n < s; ++n) p[n] -= dot * q[n];
+        }
+        double nrm = 0.0;
+        for (int n = 0; n < s; ++n) nrm += p[n] * p[n];
+        if (!(nrm > 1e-24 * scale)) return -1;
+        nrm = sqrt(nrm);
+        for (int n = 0; n < s; ++n) p[n] /= nrm;
+    }
+    return 0;
 }
 
 /* ---------------------------------------------------------------------------------------
@@ -233,12 +275,12 @@ void oracle_compress_chunk(int s, int rows, int k, double beta, double alpha, co
 void oracle_compress_chunks(int64_t n, int s, int rows, int k, double beta, double alpha, const double *g,
                             const double *m, const int32_t *forced_idx, double *Q_out,
                             int32_t *idx_out, double *val_out, double *m_new, double *gap,
-                            int n_threads)
+                            int n_threads, const double *basis)
 {
     const int M = rows * s;
     const int k_eff = k < M ? k : M;
     double *C = (double *)malloc(sizeof(double) * (size_t)s * s);
-    oracle_dct_matrix(s, C);
+    chunk_basis(s, basis, C);
     (void)n_threads;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1) num_threads(n_threads > 0 ? n_threads : omp_get_max_threads())
@@ -263,7 +305,7 @@ void oracle_compress_chunks(int64_t n, int s, int rows, int k, double beta, doub
  * ------------------------------------------------------------------------------------- */
 int oracle_compress_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, double beta, double alpha, const double *g,
                            double *m, const int32_t *forced_idx, oracle_record *records, double *val64,
-                           double *gap, int n_threads)
+                           double *gap, int n_threads, const double *basis)
 {
     if (ndim != 1 && ndim != 2) return -1;
     if (ndim == 1) n0 = 1;
@@ -273,7 +315,7 @@ int oracle_compress_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, doubl
     const int M = rows * s;
     const int k_eff = k < M ? k : M;
     double *C = (double *)malloc(sizeof(double) * (size_t)s * s);
-    oracle_dct_matrix(s, C);
+    chunk_basis(s, basis, C);
     (void)n_threads;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 4) num_threads(n_threads > 0 ? n_threads : omp_get_max_threads())
@@ -347,11 +389,12 @@ void oracle_decode_chunk(int s, int rows, int k_eff, int W, int agg, int phi, co
 
 /* Batch of independent chunks: recs is [W][n][k_eff] contiguous; x, x_new, R_out are [n][M]. */
 void oracle_decode_chunks(int64_t n, int s, int rows, int k_eff, int W, int agg, int phi, const oracle_record *recs,
-                          const double *x, double lr, double wd, double *x_new, double *R_out, int n_threads)
+                          const double *x, double lr, double wd, double *x_new, double *R_out, int n_threads,
+                          const double *basis)
 {
     const int M = rows * s;
     double *C = (double *)malloc(sizeof(double) * (size_t)s * s);
-    oracle_dct_matrix(s, C);
+    chunk_basis(s, basis, C);
     (void)n_threads;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1) num_threads(n_threads > 0 ? n_threads : omp_get_max_threads())
@@ -370,7 +413,7 @@ void oracle_decode_chunks(int64_t n, int s, int rows, int k_eff, int W, int agg,
  * x is updated in place; R_out (nullable) receives the reconstructed global momentum. */
 int oracle_decode_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, int W, int agg, int phi,
                          const oracle_record *const *payloads, double *x, double lr, double wd, double *R_out,
-                         int n_threads)
+                         int n_threads, const double *basis)
 {
     if (ndim != 1 && ndim != 2) return -1;
     if (ndim == 1) n0 = 1;
@@ -380,7 +423,7 @@ int oracle_decode_tensor(int ndim, int64_t n0, int64_t n1, int s, int k, int W, 
     const int M = rows * s;
     const int k_eff = k < M ? k : M;
     double *C = (double *)malloc(sizeof(double) * (size_t)s * s);
-    oracle_dct_matrix(s, C);
+    chunk_basis(s, basis, C);
     (void)n_threads;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 4) num_threads(n_threads > 0 ? n_threads : omp_get_max_threads())

@@ -55,16 +55,18 @@ def _load():
             lib.oracle_topk.argtypes = [i32, i32, c_dp, c_ip, c_dp, c_dp]
             lib.oracle_topk.restype = None
             lib.oracle_compress_chunks.argtypes = [i64, i32, i32, i32, f64, f64, c_dp, c_dp, c_ip, c_dp, c_ip,
-                                                   c_dp, c_dp, c_dp, i32]
+                                                   c_dp, c_dp, c_dp, i32, c_dp]
             lib.oracle_compress_chunks.restype = None
             lib.oracle_compress_tensor.argtypes = [i32, i64, i64, i32, i32, f64, f64, c_dp, c_dp, c_ip, vp, c_dp,
-                                                   c_dp, i32]
+                                                   c_dp, i32, c_dp]
             lib.oracle_compress_tensor.restype = i32
-            lib.oracle_decode_chunks.argtypes = [i64, i32, i32, i32, i32, i32, i32, vp, c_dp, f64, f64, c_dp, c_dp, i32]
+            lib.oracle_decode_chunks.argtypes = [i64, i32, i32, i32, i32, i32, i32, vp, c_dp, f64, f64, c_dp, c_dp, i32, c_dp]
             lib.oracle_decode_chunks.restype = None
             lib.oracle_decode_tensor.argtypes = [i32, i64, i64, i32, i32, i32, i32, i32, ctypes.POINTER(vp), c_dp, f64,
-                                                 f64, c_dp, i32]
+                                                 f64, c_dp, i32, c_dp]
             lib.oracle_decode_tensor.restype = i32
+            lib.oracle_gram_schmidt.argtypes = [i32, c_dp, c_dp]
+            lib.oracle_gram_schmidt.restype = i32
             lib.oracle_max_threads.argtypes = []
             lib.oracle_max_threads.restype = i32
             _lib = lib
@@ -81,6 +83,28 @@ def _ip(a):
 
 def _f64(a):
     return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _basis(basis, s):
+    """(keep-alive array, pointer) of an optional s x s basis (rows = basis vectors); None = DCT."""
+    if basis is None:
+        return None, None
+    b = _f64(basis)
+    if b.shape != (s, s):
+        raise ValueError("basis must be s x s")
+    return b, _dp(b)
+
+
+def gram_schmidt(G: np.ndarray) -> np.ndarray:
+    """Rows of the square matrix G orthonormalised in order (Gram-Schmidt process)."""
+    G = _f64(G)
+    s = G.shape[0]
+    if G.shape != (s, s):
+        raise ValueError("G must be square")
+    P = np.empty_like(G)
+    if _load().oracle_gram_schmidt(s, _dp(G), _dp(P)) != 0:
+        raise ValueError("G is singular to rounding")
+    return P
 
 
 def max_threads() -> int:
@@ -137,7 +161,7 @@ def topk(Q: np.ndarray, k: int):
 
 
 def compress_chunks(g, m, s: int, rows: int, k: int, beta: float, forced_idx=None, n_threads: int = 0,
-                    alpha: float = 1.0):
+                    alpha: float = 1.0, basis=None):
     """Independent chunks given as tiles [n, rows*s].
 
     Returns dict(Q [n,M], idx [n,k_eff] int32, val [n,k_eff] fp64, m_new [n,M], gap [n,2])."""
@@ -157,11 +181,12 @@ def compress_chunks(g, m, s: int, rows: int, k: int, beta: float, forced_idx=Non
     if forced_idx is not None:
         fi = np.ascontiguousarray(forced_idx, dtype=np.int32).reshape(n, k_eff)
     _load().oracle_compress_chunks(n, s, rows, k, float(beta), float(alpha), _dp(g), _dp(m), _ip(fi) if fi is not None else None,
-                                   _dp(Q), _ip(idx), _dp(val), _dp(m_new), _dp(gap), n_threads)
+                                   _dp(Q), _ip(idx), _dp(val), _dp(m_new), _dp(gap), n_threads, _basis(basis, s)[1])
     return dict(Q=Q, idx=idx, val=val, m_new=m_new, gap=gap)
 
 
-def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_threads: int = 0, alpha: float = 1.0):
+def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_threads: int = 0, alpha: float = 1.0,
+                    basis=None):
     """One tensor (1-D or 2-D), one worker.  Returns dict(m_new, records [n_chunks,k_eff], val64, gap)."""
     g = _f64(g)
     m_new = _f64(m).copy()
@@ -181,7 +206,7 @@ def compress_tensor(g, m, s: int, k: int, beta: float, forced_idx=None, n_thread
         fi = np.ascontiguousarray(forced_idx, dtype=np.int32).reshape(n_chunks, k_eff)
     rc = _load().oracle_compress_tensor(ndim, n0, n1, s, k, float(beta), float(alpha), _dp(g), _dp(m_new),
                                         _ip(fi) if fi is not None else None, rec.ctypes.data_as(ctypes.c_void_p),
-                                        _dp(val64), _dp(gap), n_threads)
+                                        _dp(val64), _dp(gap), n_threads, _basis(basis, s)[1])
     if rc != 0:
         raise ValueError("oracle_compress_tensor rejected the shape")
     return dict(m_new=m_new, records=rec, val64=val64, gap=gap)
@@ -191,7 +216,8 @@ AGG_SUM, AGG_MEAN, AGG_COUNT_MEAN = 0, 1, 2
 PHI_SIGN, PHI_IDENTITY = 0, 1
 
 
-def decode_chunks(records, x, s: int, rows: int, lr: float, wd: float, n_threads: int = 0, agg: int = 0, phi: int = 0):
+def decode_chunks(records, x, s: int, rows: int, lr: float, wd: float, n_threads: int = 0, agg: int = 0, phi: int = 0,
+                  basis=None):
     """records [W, n, k_eff] (RECORD_DTYPE), x [n, rows*s] -> dict(x_new [n,M], R [n,M])."""
     records = np.ascontiguousarray(records, dtype=RECORD_DTYPE)
     W, n, k_eff = records.shape
@@ -200,11 +226,12 @@ def decode_chunks(records, x, s: int, rows: int, lr: float, wd: float, n_threads
     x_new = np.empty_like(x)
     R = np.empty_like(x)
     _load().oracle_decode_chunks(n, s, rows, k_eff, W, agg, phi, records.ctypes.data_as(ctypes.c_void_p), _dp(x), float(lr),
-                                 float(wd), _dp(x_new), _dp(R), n_threads)
+                                 float(wd), _dp(x_new), _dp(R), n_threads, _basis(basis, s)[1])
     return dict(x_new=x_new, R=R)
 
 
-def decode_tensor(payloads, x, s: int, k: int, lr: float, wd: float, n_threads: int = 0, agg: int = 0, phi: int = 0):
+def decode_tensor(payloads, x, s: int, k: int, lr: float, wd: float, n_threads: int = 0, agg: int = 0, phi: int = 0,
+                  basis=None):
     """payloads: list over workers of [n_chunks, k_eff] record arrays for this tensor.
 
     Returns dict(x_new, R) with R the reconstructed global momentum of the tensor."""
@@ -216,7 +243,7 @@ def decode_tensor(payloads, x, s: int, k: int, lr: float, wd: float, n_threads: 
     arr = (ctypes.c_void_p * W)(*[p.ctypes.data for p in keep])
     R = np.empty_like(x_new)
     rc = _load().oracle_decode_tensor(ndim, n0, n1, s, k, W, agg, phi, arr, _dp(x_new), float(lr), float(wd), _dp(R),
-                                      n_threads)
+                                      n_threads, _basis(basis, s)[1])
     if rc != 0:
         raise ValueError("oracle_decode_tensor rejected the shape")
     return dict(x_new=x_new, R=R)

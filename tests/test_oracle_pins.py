@@ -472,3 +472,104 @@ def test_count_mean_limits_and_identity_update():
     assert np.array_equal(c["x_new"], d["x_new"])
     assert np.max(np.abs(b["x_new"] - (x - 1e-3 * (b["R"] + 0.1 * x)))) < 1e-16
     assert np.max(np.abs(b["R"] - c["R"] / W)) < 1e-15
+
+
+# --------------------------------------------------------------------------------------------
+# Other orthonormal bases (Section 4.2, "Choice of Linear Projections"): identity, and a Gaussian
+# matrix orthonormalised by the Gram-Schmidt process
+# --------------------------------------------------------------------------------------------
+def test_gram_schmidt_hand_example_and_library_qr():
+    # 2 x 2 by hand: rows (3,4), (1,0) -> (0.6,0.8), then (1,0) - 0.6*(0.6,0.8) = (0.64,-0.48) -> (0.8,-0.6)
+    P = orc.gram_schmidt(np.array([[3.0, 4.0], [1.0, 0.0]]))
+    assert np.max(np.abs(P - np.array([[0.6, 0.8], [0.8, -0.6]]))) < 1e-15
+    rng = np.random.default_rng(5)
+    for s in (8, 32, 64, 128):
+        G = rng.standard_normal((s, s))
+        P = orc.gram_schmidt(G)
+        assert np.max(np.abs(P @ P.T - np.eye(s))) < 1e-12
+        # rows orthonormalised in order: G = L P with L lower triangular, positive diagonal
+        L = G @ P.T
+        assert np.max(np.abs(np.triu(L, 1))) < 1e-11 and np.all(np.diag(L) > 0)
+        assert np.max(np.abs(P[0] - G[0] / np.linalg.norm(G[0]))) < 1e-15
+        # the library's QR of G^T gives the same vectors once its signs are fixed
+        Qm, Rm = np.linalg.qr(G.T)
+        assert np.max(np.abs(P - (Qm * np.sign(np.diag(Rm))).T)) < 1e-10
+    with pytest.raises(ValueError):
+        orc.gram_schmidt(np.ones((4, 4)))
+
+
+def test_identity_basis_is_plain_topk_of_the_momentum():
+    s, rows, k, n = 8, 8, 5, 6
+    M = s * s
+    rng = np.random.default_rng(6)
+    g, m = rng.standard_normal((n, M)), rng.standard_normal((n, M))
+    out = orc.compress_chunks(g, m, s, rows, k, 0.9, basis=np.eye(s))
+    B = 0.9 * m + g
+    for c in range(n):
+        want = np.sort(np.argsort(-np.abs(B[c]), kind="stable")[:k])
+        assert np.array_equal(out["idx"][c], want)
+        assert np.array_equal(out["val"][c], B[c][want]) and np.array_equal(out["Q"][c], B[c])
+        keep = B[c].copy()
+        keep[want] = 0.0
+        assert np.array_equal(out["m_new"][c], keep)
+    # decode with the identity: the scattered sum itself drives the update
+    recs = np.zeros((2, n, k), dtype=orc.RECORD_DTYPE)
+    recs[0]["idx"], recs[0]["val"] = out["idx"], out["val"].astype(np.float32)
+    recs[1]["idx"], recs[1]["val"] = out["idx"], (2.0 * out["val"]).astype(np.float32)
+    x = rng.standard_normal((n, M)) * 0.02
+    dec = orc.decode_chunks(recs, x, s, rows, 1e-3, 0.1, basis=np.eye(s))
+    S = np.zeros((n, M))
+    for c in range(n):
+        S[c][out["idx"][c]] = recs[0][c]["val"].astype(np.float64) + recs[1][c]["val"].astype(np.float64)
+    assert np.array_equal(dec["R"], S)
+    assert np.max(np.abs(dec["x_new"] - (x - 1e-3 * (np.sign(S) + 0.1 * x)))) < 1e-17
+
+
+@pytest.mark.parametrize("s,rows", [(8, 8), (32, 32), (64, 1)])
+def test_random_orthonormal_basis_identities(s, rows):
+    M, k, n = s * rows, 7, 3
+    rng = np.random.default_rng(7)
+    P = orc.gram_schmidt(rng.standard_normal((s, s)))
+    g, m = rng.standard_normal((n, M)), rng.standard_normal((n, M))
+    out = orc.compress_chunks(g, m, s, rows, k, 0.999, basis=P)
+    B = 0.999 * m + g
+    for c in range(n):
+        # rows of P are the basis vectors: Q = P B P^T (2-D), q = P b (1-D); P is not symmetric, so
+        # a transposed operand fails here
+        Qw = P @ B[c].reshape(rows, s) @ P.T if rows > 1 else P @ B[c]
+        assert np.max(np.abs(out["Q"][c] - Qw.reshape(-1))) < 1e-12
+        assert abs(np.sum(out["Q"][c] ** 2) - np.sum(B[c] ** 2)) < 1e-10 * np.sum(B[c] ** 2)
+        Qs = np.zeros(M)
+        Qs[out["idx"][c]] = out["val"][c]
+        back = P.T @ Qs.reshape(rows, s) @ P if rows > 1 else P.T @ Qs
+        assert np.max(np.abs(back.reshape(-1) + out["m_new"][c] - B[c])) < 1e-12
+    # W = 1 decode rebuilds what compress removed
+    recs = np.zeros((1, n, k), dtype=orc.RECORD_DTYPE)
+    recs[0]["idx"], recs[0]["val"] = out["idx"], out["val"].astype(np.float32)
+    dec = orc.decode_chunks(recs, np.zeros((n, M)), s, rows, 1.0, 0.0, basis=P, phi=orc.PHI_IDENTITY)
+    assert np.max(np.abs(dec["R"] - (B - out["m_new"]))) < 1e-6
+
+
+def test_explicit_dct_basis_equals_default_and_tensor_driver_takes_a_basis():
+    s, k = 8, 4
+    rng = np.random.default_rng(8)
+    g, m = rng.standard_normal((16, 24)), rng.standard_normal((16, 24))
+    a = orc.compress_tensor(g, m, s, k, 0.9)
+    b = orc.compress_tensor(g, m, s, k, 0.9, basis=orc.dct_matrix(s))
+    assert np.array_equal(a["records"], b["records"]) and np.array_equal(a["m_new"], b["m_new"])
+    P = orc.gram_schmidt(rng.standard_normal((s, s)))
+    t = orc.compress_tensor(g, m, s, k, 0.9, basis=P)
+    # chunk (1, 2) of the tensor driver == the chunk routine on that tile
+    tile = lambda X: orc.block_extract(X, s, s, 1, 2).reshape(1, -1)
+    c = orc.compress_chunks(tile(g), tile(m), s, s, k, 0.9, basis=P)
+    assert np.array_equal(t["records"][1 * 3 + 2]["idx"], c["idx"][0])
+    assert np.array_equal(orc.block_extract(t["m_new"], s, s, 1, 2).reshape(-1), c["m_new"][0])
+    x = rng.standard_normal((16, 24)) * 0.02
+    d1 = orc.decode_tensor([a["records"]], x, s, k, 1e-3, 0.1)
+    d2 = orc.decode_tensor([a["records"]], x, s, k, 1e-3, 0.1, basis=orc.dct_matrix(s))
+    assert np.array_equal(d1["x_new"], d2["x_new"])
+    d3 = orc.decode_tensor([t["records"]], x, s, k, 1e-3, 0.1, basis=P)
+    R = orc.block_extract(d3["R"], s, s, 1, 2)
+    Qs = np.zeros(s * s)
+    Qs[c["idx"][0]] = c["val"][0].astype(np.float32)
+    assert np.max(np.abs(R - P.T @ Qs.reshape(s, s) @ P)) < 1e-12
