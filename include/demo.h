@@ -203,6 +203,29 @@ typedef enum { DEMO_AGG_SUM = 0, DEMO_AGG_MEAN = 1, DEMO_AGG_COUNT_MEAN = 2 } de
 typedef enum { DEMO_PHI_SIGN = 0, DEMO_PHI_IDENTITY = 1 } demo_phi;
 demo_status demo_set_decode_mode(demo_ctx *ctx, int32_t aggregation, int32_t phi);
 
+/* Other orthonormal bases (Section 4.2, "Choice of Linear Projections": identity mapping, random
+ * orthonormal projection).  The basis is an s x s row-major fp32 matrix P whose ROWS are the basis
+ * vectors; it replaces the DCT matrix on both axes of a 2-D chunk (Q = P B P^T, inverse P^T Q P) and on
+ * 1-D segments (q = P b).  While a caller-supplied basis is active every tensor goes through the
+ * dense-transform kernels (the fast kernels hard-code the DCT factorisation).
+ *
+ * demo_set_basis: basis_host = HOST pointer to P, read during the call and not retained; NULL restores
+ * the DCT.  The rows must be orthonormal to 1e-5 (INVALID_ARG otherwise).  The upload is enqueued on
+ * cuda_stream, so the new basis applies to calls enqueued after it on that stream.
+ *
+ * demo_set_basis_gaussian: gauss_host = HOST pointer to an s x s row-major matrix of N(0,1) draws (the
+ * paper seeds them with the step number so that all workers agree).  Its rows are orthonormalised in
+ * order by the Gram-Schmidt process on the device (fp64, one small kernel) and the result becomes the
+ * active basis.  Synchronises cuda_stream.  INVALID_ARG when a row has no component left (singular
+ * matrix); the previous basis then stays in force.
+ *
+ * demo_get_basis: copies the active basis (DCT or caller-supplied) to basis_host_out (HOST, s*s floats)
+ * and synchronises cuda_stream.
+ * Errors: INVALID_ARG, CUDA. */
+demo_status demo_set_basis(demo_ctx *ctx, const float *basis_host, void *cuda_stream);
+demo_status demo_set_basis_gaussian(demo_ctx *ctx, const float *gauss_host, void *cuda_stream);
+demo_status demo_get_basis(demo_ctx *ctx, float *basis_host_out, void *cuda_stream);
+
 /* Self-test of the device-side failure path: enqueue a one-CTA kernel that waits, for at most
  * limit_cycles SM clock cycles (1 .. 2e9), on a barrier that nothing completes -- the situation a lost
  * tile copy would create -- using the same bounded wait as the production kernels.  The kernel records

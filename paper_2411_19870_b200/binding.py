@@ -11,6 +11,8 @@ import ctypes
 import os
 from typing import List, Optional, Sequence
 
+import torch
+
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libdemo_b200.so")
 
@@ -22,7 +24,8 @@ RECORD_BYTES = 8
 
 EXPORTS = [
     "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
-    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_selftest_bounded_wait", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_set_basis",
+    "demo_set_basis_gaussian", "demo_get_basis", "demo_selftest_bounded_wait", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
 ]
 
@@ -81,6 +84,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_set_alpha.restype = i32
     lib.demo_set_decode_mode.argtypes = [vp, i32, i32]
     lib.demo_set_decode_mode.restype = i32
+    lib.demo_set_basis.argtypes = [vp, vp, vp]
+    lib.demo_set_basis.restype = i32
+    lib.demo_set_basis_gaussian.argtypes = [vp, vp, vp]
+    lib.demo_set_basis_gaussian.restype = i32
+    lib.demo_get_basis.argtypes = [vp, vp, vp]
+    lib.demo_get_basis.restype = i32
     lib.demo_selftest_bounded_wait.argtypes = [vp, i64, vp]
     lib.demo_selftest_bounded_wait.restype = i32
     lib.demo_set_path.argtypes = [vp, i32]
@@ -224,6 +233,35 @@ class DemoTransform:
         st = self.lib.demo_set_decode_mode(self._ctx, aggregation, phi)
         if st != 0:
             raise DemoError(st, "demo_set_decode_mode")
+
+    def _host_matrix(self, a):
+        a = a.detach().to("cpu", torch.float32).contiguous() if isinstance(a, torch.Tensor) else torch.tensor(a, dtype=torch.float32)
+        s = self.cfg.chunk
+        if tuple(a.shape) != (s, s):
+            raise ValueError("expected an s x s matrix")
+        return a
+
+    def set_basis(self, basis=None, stream=None) -> None:
+        """s x s matrix whose rows are the basis vectors (host or device tensor); None restores the DCT."""
+        keep = None if basis is None else self._host_matrix(basis)
+        st = self.lib.demo_set_basis(self._ctx, None if keep is None else keep.data_ptr(), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_set_basis")
+
+    def set_basis_gaussian(self, gauss, stream=None) -> None:
+        """Gram-Schmidt (on the device) of the rows of an s x s matrix of N(0,1) draws."""
+        keep = self._host_matrix(gauss)
+        st = self.lib.demo_set_basis_gaussian(self._ctx, keep.data_ptr(), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_set_basis_gaussian")
+
+    def get_basis(self, stream=None) -> torch.Tensor:
+        s = self.cfg.chunk
+        out = torch.empty((s, s), dtype=torch.float32)
+        st = self.lib.demo_get_basis(self._ctx, out.data_ptr(), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_get_basis")
+        return out
 
     def selftest_bounded_wait(self, limit_cycles: int, stream=None) -> None:
         st = self.lib.demo_selftest_bounded_wait(self._ctx, int(limit_cycles), self._stream(stream))

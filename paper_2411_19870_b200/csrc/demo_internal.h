@@ -76,6 +76,10 @@ cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cu
 // mbarrier that nothing completes, records DEMO_DEV_TIMEOUT in *status and returns.
 cudaError_t demo_launch_wait_selftest(int *status, long long limit_cycles, cudaStream_t stream);
 
+// Gram-Schmidt process on the rows of the s x s matrix `gauss` (device, fp32) in fp64; writes the
+// orthonormal rows to `basis` (device, fp32) and 1 to *flag when a row has no component left.
+cudaError_t demo_launch_gram_schmidt(const float *gauss, float *basis, int *flag, int s, cudaStream_t stream);
+
 // Locate the tensor that owns chunk id c: the last entry with chunk_begin <= c.
 __device__ __forceinline__ int demo_find_entry(const DemoTensorEntry *entries, int n, long long c)
 {

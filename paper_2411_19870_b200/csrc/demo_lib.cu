@@ -33,6 +33,12 @@ struct demo_ctx {
     float *d_C = nullptr;
     int *d_status = nullptr;
 
+    // caller-supplied orthonormal basis (rows = basis vectors); while `custom_basis` is set every
+    // tensor goes through the dense-transform kernels, which read the basis from memory
+    float *d_P = nullptr, *d_P_stage = nullptr;  // [s*s], [2*s*s]
+    int *d_basis_flag = nullptr;
+    bool custom_basis = false;
+
     // device pointer tables and their host mirrors (uploaded only when the caller's pointers change)
     const void **d_g = nullptr;      // [W][T]
     float **d_m = nullptr;           // [W][T]
@@ -122,6 +128,9 @@ void release(demo_ctx *c)
     cudaFree(c->d_entries2d);
     cudaFree(c->d_entries1d);
     cudaFree(c->d_C);
+    cudaFree(c->d_P);
+    cudaFree(c->d_P_stage);
+    cudaFree(c->d_basis_flag);
     cudaFree(c->d_status);
     cudaFree((void *)c->d_g);
     cudaFree((void *)c->d_m);
@@ -259,6 +268,9 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
     bool ok = true;
     ok = ok && cudaMalloc(&c->d_C, C.size() * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_P, C.size() * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_P_stage, 2 * C.size() * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_basis_flag, sizeof(int)) == cudaSuccess;
     if (ok && c->n2d) ok = cudaMalloc(&c->d_entries2d, e2d.size() * sizeof(DemoTensorEntry)) == cudaSuccess;
     if (ok && c->n1d) ok = cudaMalloc(&c->d_entries1d, e1d.size() * sizeof(DemoTensorEntry)) == cudaSuccess;
     ok = ok && cudaMalloc((void **)&c->d_g, W * T * sizeof(void *)) == cudaSuccess;
@@ -318,6 +330,13 @@ demo_status demo_payload_layout(const demo_ctx *ctx, int32_t tensor, int64_t *fi
     return DEMO_OK;
 }
 
+// The fast kernels hard-code the DCT factorisation; any other basis takes the dense-transform kernels.
+static bool use_fast_path(const demo_ctx *ctx)
+{
+    const int s = ctx->cfg.chunk;
+    return ctx->path == DEMO_PATH_AUTO && !ctx->custom_basis && demo_fast_supported(s) && (s != 128 || ctx->encode);
+}
+
 demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grads, float *const *momentum,
                           void *payload_out, void *cuda_stream)
 {
@@ -358,7 +377,7 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
     a.g_ptrs = ctx->d_g + row;
     a.m_ptrs = ctx->d_m + row;
     a.payload = static_cast<DemoRecord *>(payload_out);
-    a.C = ctx->d_C;
+    a.C = ctx->custom_basis ? ctx->d_P : ctx->d_C;
     a.beta = ctx->cfg.beta;
     a.alpha = ctx->alpha;
     a.grad_bf16 = ctx->cfg.grad_dtype == DEMO_BF16;
@@ -370,7 +389,7 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
-        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s) && (s != 128 || ctx->encode))
+        if (use_fast_path(ctx))
             err = demo_launch_compress_fast(s, a, ctx->sm_count, stream);
         else
             err = demo_launch_compress_generic(s, 1, a, ctx->sm_count, stream);
@@ -424,7 +443,7 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     a.payloads = ctx->d_p;
     a.W = W;
     a.x_ptrs = ctx->d_x;
-    a.C = ctx->d_C;
+    a.C = ctx->custom_basis ? ctx->d_P : ctx->d_C;
     a.lr = ctx->cfg.lr;
     a.wd = ctx->cfg.weight_decay;
     a.status = ctx->d_status;
@@ -437,7 +456,7 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
-        if (ctx->path == DEMO_PATH_AUTO && demo_fast_supported(s) && (s != 128 || ctx->encode))
+        if (use_fast_path(ctx))
             err = demo_launch_decode_fast(s, a, ctx->sm_count, stream);
         else
             err = demo_launch_decode_generic(s, 1, a, ctx->sm_count, stream);
@@ -559,6 +578,76 @@ demo_status demo_selftest_bounded_wait(demo_ctx *ctx, int64_t limit_cycles, void
         return DEMO_ERR_CUDA;
     }
     ctx->launches += 1;
+    return DEMO_OK;
+}
+
+demo_status demo_set_basis(demo_ctx *ctx, const float *basis_host, void *cuda_stream)
+{
+    if (!ctx) return DEMO_ERR_INVALID_ARG;
+    if (!basis_host) {
+        ctx->custom_basis = false;
+        return DEMO_OK;
+    }
+    const int s = ctx->cfg.chunk;
+    // rows must be orthonormal: |<p_u, p_v> - delta_uv| <= 1e-5 (fp32 entries carry ~6e-8 each)
+    for (int u = 0; u < s; ++u)
+        for (int v = u; v < s; ++v) {
+            double dot = 0.0;
+            for (int n = 0; n < s; ++n) dot += (double)basis_host[(size_t)u * s + n] * basis_host[(size_t)v * s + n];
+            if (!(std::fabs(dot - (u == v ? 1.0 : 0.0)) <= 1e-5)) return DEMO_ERR_INVALID_ARG;
+        }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    if (cudaMemcpyAsync(ctx->d_P, basis_host, sizeof(float) * (size_t)s * s, cudaMemcpyHostToDevice,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    ctx->custom_basis = true;
+    return DEMO_OK;
+}
+
+demo_status demo_set_basis_gaussian(demo_ctx *ctx, const float *gauss_host, void *cuda_stream)
+{
+    if (!ctx || !gauss_host) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int s = ctx->cfg.chunk;
+    const size_t n = (size_t)s * s;
+    // staging = [Gaussian input | orthonormalised output]; the active table is replaced only after the
+    // kernel's verdict, so a singular matrix leaves the previous basis in force
+    float *gauss = ctx->d_P_stage, *out = ctx->d_P_stage + n;
+    int flag = 0;
+    bool ok = cudaMemcpyAsync(gauss, gauss_host, n * sizeof(float), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaMemsetAsync(ctx->d_basis_flag, 0, sizeof(int), stream) == cudaSuccess;
+    ok = ok && demo_launch_gram_schmidt(gauss, out, ctx->d_basis_flag, s, stream) == cudaSuccess;
+    if (ok) ctx->launches += 1;
+    ok = ok && cudaMemcpyAsync(&flag, ctx->d_basis_flag, sizeof(int), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    if (ok && flag) return DEMO_ERR_INVALID_ARG;
+    ok = ok && cudaMemcpyAsync(ctx->d_P, out, n * sizeof(float), cudaMemcpyDeviceToDevice, stream) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    ctx->custom_basis = true;
+    return DEMO_OK;
+}
+
+demo_status demo_get_basis(demo_ctx *ctx, float *basis_host_out, void *cuda_stream)
+{
+    if (!ctx || !basis_host_out) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t bytes = sizeof(float) * (size_t)ctx->cfg.chunk * ctx->cfg.chunk;
+    if (cudaMemcpyAsync(basis_host_out, ctx->custom_basis ? ctx->d_P : ctx->d_C, bytes, cudaMemcpyDeviceToHost,
+                        stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
     return DEMO_OK;
 }
 

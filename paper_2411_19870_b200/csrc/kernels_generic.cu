@@ -376,6 +376,85 @@ cudaError_t demo_launch_decode_generic(int s, int two_d, const DemoDecodeArgs &a
 }
 
 // =================================================================================================
+// Random orthonormal basis (Section 4.2, "Choice of Linear Projections"): Gram-Schmidt process on the
+// rows of a Gaussian matrix, in fp64, one CTA.  Right-looking order: once row j is final its component
+// is removed from every later row, so each row loses its components along rows 0..j-1 one after the
+// other -- the same operations as the row-by-row statement of the process.
+// =================================================================================================
+constexpr int GS_THREADS = 1024;
+
+__global__ void __launch_bounds__(GS_THREADS) gram_schmidt_kernel(const float *__restrict__ gauss,
+                                                                  float *__restrict__ basis, int *flag, int s)
+{
+    extern __shared__ double gs_A[];  // [s][s + 1]
+    __shared__ double scale[128];     // squared length of each input row
+    __shared__ double inv_len;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int WARPS = GS_THREADS / 32;
+    const int ld = s + 1;
+    for (int i = tid; i < s * s; i += GS_THREADS) gs_A[(i / s) * ld + (i % s)] = (double)gauss[i];
+    __syncthreads();
+    for (int r = warp; r < s; r += WARPS) {
+        double acc = 0.0;
+        for (int n = lane; n < s; n += 32) acc += gs_A[r * ld + n] * gs_A[r * ld + n];
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+        if (lane == 0) scale[r] = acc;
+    }
+    __syncthreads();
+    bool bad = false;
+    for (int j = 0; j < s; ++j) {
+        if (warp == 0) {
+            double acc = 0.0;
+            for (int n = lane; n < s; n += 32) acc += gs_A[j * ld + n] * gs_A[j * ld + n];
+            for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+            if (lane == 0) inv_len = (acc > 1e-24 * scale[j]) ? 1.0 / sqrt(acc) : 0.0;
+        }
+        __syncthreads();
+        const double inv = inv_len;
+        if (inv == 0.0) {
+            bad = true;
+            break;
+        }
+        double p[4];  // s <= 128: at most 4 entries of row j per lane
+#pragma unroll
+        for (int t = 0; t < 4; ++t) p[t] = (lane + 32 * t < s) ? gs_A[j * ld + lane + 32 * t] * inv : 0.0;
+        for (int r = j + 1 + warp; r < s; r += WARPS) {
+            double dot = 0.0;
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if (lane + 32 * t < s) dot += gs_A[r * ld + lane + 32 * t] * p[t];
+            for (int d = 16; d > 0; d >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, d);
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if (lane + 32 * t < s) gs_A[r * ld + lane + 32 * t] -= dot * p[t];
+        }
+        __syncthreads();
+        if (warp == 0) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if (lane + 32 * t < s) gs_A[j * ld + lane + 32 * t] = p[t];
+        }
+    }
+    __syncthreads();
+    if (bad) {
+        if (tid == 0) *flag = 1;
+        return;
+    }
+    for (int i = tid; i < s * s; i += GS_THREADS) basis[i] = (float)gs_A[(i / s) * ld + (i % s)];
+}
+
+cudaError_t demo_launch_gram_schmidt(const float *gauss, float *basis, int *flag, int s, cudaStream_t stream)
+{
+    if (s < 1 || s > 128) return cudaErrorInvalidValue;
+    const size_t smem = sizeof(double) * (size_t)s * (s + 1);
+    cudaError_t err =
+        cudaFuncSetAttribute(gram_schmidt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    gram_schmidt_kernel<<<1, GS_THREADS, smem, stream>>>(gauss, basis, flag, s);
+    return cudaGetLastError();
+}
+
+// =================================================================================================
 // demo_decode_apply_static: the decode + update step for callers that must not allocate.
 //
 // The generic decode kernels above read four small tables from global memory besides the caller's

@@ -207,3 +207,11 @@ class GradStream:
 
     def next(self) -> List[torch.Tensor]:
         return [self._draw(t, shp).to(self.wl.grad_dtype) for t, shp in enumerate(self.wl.shapes)]
+
+
+def basis_gaussian(step: int, s: int) -> torch.Tensor:
+    """s x s matrix of N(0,1) draws for the random orthonormal basis of one step; the seed is the step
+    number, so every worker draws the same matrix (Section 4.2)."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(int(step))
+    return torch.randn((s, s), generator=gen, dtype=torch.float32)

@@ -66,12 +66,13 @@ class Report(dict):
         self[key] = self.get(key, 0) + int(n)
 
 
-def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, report: Report, what="", alpha=1.0):
+def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, report: Report, what="", alpha=1.0,
+                          basis=None):
     """All arguments are per-chunk arrays of the same n chunks (float64 / records)."""
     M = rows * s
     k_eff = min(k, M)
     n = g.shape[0]
-    ref = orc.compress_chunks(g, m_before, s, rows, k, beta, alpha=alpha)
+    ref = orc.compress_chunks(g, m_before, s, rows, k, beta, alpha=alpha, basis=basis)
     Q = ref["Q"]
     qinf = np.max(np.abs(Q), axis=1)
     floor = FLOOR_REL * qinf
@@ -121,7 +122,8 @@ def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, repor
     # residual momentum: oracle continued from the GPU's index set where the sets differ
     m_ref = ref["m_new"]
     if len(diff):
-        forced = orc.compress_chunks(g[diff], m_before[diff], s, rows, k, beta, forced_idx=idx_gpu[diff].astype(np.int32), alpha=alpha)
+        forced = orc.compress_chunks(g[diff], m_before[diff], s, rows, k, beta, forced_idx=idx_gpu[diff].astype(np.int32), alpha=alpha,
+                                     basis=basis)
         m_ref = m_ref.copy()
         m_ref[diff] = forced["m_new"]
     # the abs tolerance is scaled by the chunk's pre-subtraction magnitude (the fp32 rounding of
@@ -135,9 +137,10 @@ def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, repor
     return ref
 
 
-def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Report, what="", agg=0, phi=0):
+def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Report, what="", agg=0, phi=0,
+                         basis=None):
     """recs_gpu [W, n, k_eff] GPU-written records; x_* float64 [n, M]."""
-    ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd, agg=agg, phi=phi)
+    ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd, agg=agg, phi=phi, basis=basis)
     R = ref["R"]
     if phi == orc.PHI_IDENTITY:
         # no sign decision: the update is linear in R; the tolerance follows R's fp32 rounding
@@ -174,7 +177,8 @@ def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Re
 class Runner:
     """Drives a workload through the C ABI and checks sampled (or all) chunks every step."""
 
-    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0, alpha=None, agg=0, phi=0):
+    def __init__(self, wl, device="cuda", max_chunks=256, path=None, seed=0, alpha=None, agg=0, phi=0, basis=None,
+                 gauss=None):
         import paper_2411_19870_b200 as demo
         from paper_2411_19870_b200 import inputs
 
@@ -189,6 +193,10 @@ class Runner:
         self.agg, self.phi = agg, phi
         if agg or phi:
             self.tr.set_decode_mode(agg, phi)
+        # other bases: `basis` (s x s, rows = vectors) is handed to both sides; `gauss` is orthonormalised
+        # by each side with its own Gram-Schmidt
+        self.basis = None
+        self.set_basis(basis, gauss)
         self.alpha = 1.0
         if alpha is not None:
             self.tr.set_alpha(alpha)
@@ -206,6 +214,19 @@ class Runner:
         self.lr = float(np.float32(wl.lr))
         self.wd = float(np.float32(wl.weight_decay))
 
+    def set_basis(self, basis=None, gauss=None):
+        if gauss is not None:
+            g32 = np.ascontiguousarray(gauss, dtype=np.float32)
+            self.tr.set_basis_gaussian(torch.from_numpy(g32))
+            self.basis = orc.gram_schmidt(g32.astype(np.float64))
+        elif basis is not None:
+            b32 = np.ascontiguousarray(basis, dtype=np.float32)
+            self.tr.set_basis(torch.from_numpy(b32))
+            self.basis = b32.astype(np.float64)
+        else:
+            self.tr.set_basis(None)
+            self.basis = None
+
     def step(self, check=True, grads=None):
         wl, s = self.wl, self.wl.chunk
         T = len(wl.shapes)
@@ -221,7 +242,7 @@ class Runner:
                     check_compress_chunks(
                         gather_tiles(g[t], s, self.ids[t]), before[t], gather_tiles(self.mom[w][t], s, self.ids[t]),
                         gather_records(self.payloads[w], first, k_eff, self.ids[t]), s, rows, wl.topk, self.beta,
-                        self.report, what="compress w%d t%d" % (w, t), alpha=self.alpha)
+                        self.report, what="compress w%d t%d" % (w, t), alpha=self.alpha, basis=self.basis)
         if check:
             xb = [gather_tiles(self.params[t], s, self.ids[t]) for t in range(T)]
         self.tr.decode_apply(self.payloads, self.params)
@@ -232,7 +253,7 @@ class Runner:
                 recs = np.stack([gather_records(self.payloads[w], first, k_eff, self.ids[t])
                                  for w in range(wl.num_workers)])
                 check_decode_chunks(recs, xb[t], gather_tiles(self.params[t], s, self.ids[t]), s, rows, self.lr,
-                                    self.wd, self.report, what="decode t%d" % t, agg=self.agg, phi=self.phi)
+                                    self.wd, self.report, what="decode t%d" % t, agg=self.agg, phi=self.phi, basis=self.basis)
         st = self.tr.device_status()
         assert st == 0, "device status %d (%s)" % (st, self.demo.demo_status_string(st))
 

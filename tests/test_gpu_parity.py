@@ -315,6 +315,52 @@ def test_aggregation_and_phi_variants(s, agg, phi):
         r.close()
 
 
+@pytest.mark.parametrize("s", [8, 64, 128])
+def test_identity_basis(s):
+    """Section 4.2's baseline P = I: top-k of the momentum itself, sign of the scattered sum."""
+    shapes = [(2 * s, 3 * s), (2 * s,)]
+    wl = inputs.Workload("ident", shapes, chunk=s, topk=max(2, s // 2), num_workers=3, grad_kind="normal", grad_std=0.01)
+    r = parity.Runner(wl, max_chunks=10**9, basis=np.eye(s))
+    r.step()
+    r.step()
+    assert torch.equal(r.tr.get_basis(), torch.eye(s))
+    r.close()
+
+
+@pytest.mark.parametrize("s", [8, 32, 64, 128])
+def test_random_orthonormal_basis_redrawn_every_step(s):
+    """Gaussian matrix seeded by the step number, Gram-Schmidt on the device vs the oracle's own."""
+    shapes = [(2 * s, 3 * s), (4 * s,)]
+    wl = inputs.Workload("randp", shapes, chunk=s, topk=max(2, s // 2), num_workers=2, grad_kind="normal", grad_std=0.01)
+    r = parity.Runner(wl, max_chunks=10**9)
+    for step in (1, 2, 3):
+        r.set_basis(gauss=inputs.basis_gaussian(step, s).numpy())
+        P = r.tr.get_basis().double().numpy()
+        assert np.max(np.abs(P - r.basis)) < 2e-7
+        assert np.max(np.abs(P @ P.T - np.eye(s))) < 2e-6
+        r.step()
+    # back to the DCT (and, where there is one, to the fast kernel family)
+    r.set_basis()
+    r.step()
+    r.close()
+
+
+def test_basis_argument_errors_keep_the_previous_basis():
+    s = 8
+    wl = inputs.Workload("basis-err", [(2 * s, 2 * s)], chunk=s, topk=4, num_workers=1, grad_kind="normal", grad_std=0.01)
+    r = parity.Runner(wl, max_chunks=10**9, gauss=inputs.basis_gaussian(7, s).numpy())
+    before = r.tr.get_basis()
+    with pytest.raises(demo.DemoError):
+        r.tr.set_basis(torch.ones((s, s)))  # rows not orthonormal
+    with pytest.raises(demo.DemoError):
+        r.tr.set_basis_gaussian(torch.ones((s, s)))  # singular: the second row has nothing left
+    with pytest.raises(ValueError):
+        r.tr.set_basis(torch.eye(s + 1))
+    assert torch.equal(r.tr.get_basis(), before)
+    r.step()
+    r.close()
+
+
 def test_bounded_wait_expires_into_a_status_and_the_context_survives():
     """Failure detection without a GPU fault: a wait that nothing satisfies runs out after ~1 ms, the
     kernel returns, the sticky status says TIMEOUT, and the same context then computes correctly."""
