@@ -11,6 +11,12 @@
  * there is no global state and no CPU fallback: without a CUDA device every compute entry point
  * fails with DEMO_ERR_CUDA.
  *
+ * CUDA graphs: demo_compress and demo_decode_apply copy their pointer arrays to device tables only
+ * when a pointer differs from the previous call with the same worker index.  After one ordinary call
+ * with the same buffers they enqueue kernel launches only and may be captured into a CUDA graph on
+ * the capturing stream; the graph is valid while the buffers and the context live and the context's
+ * settings (learning rate, alpha, decode mode, basis, path) are those of the capture.
+ *
  * Notation (the paper's): s chunk size, k coefficients kept per chunk, M = s*s (2-D tensors) or
  * s (1-D tensors) elements per chunk, k_eff = min(k, M), W workers, beta momentum decay,
  * lr learning rate (eta), weight_decay (lambda).

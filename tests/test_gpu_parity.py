@@ -233,6 +233,51 @@ def test_step_host_matches_separate_calls():
     r.close()
 
 
+@pytest.mark.parametrize("path", [None, demo.DEMO_PATH_GENERIC])
+def test_cuda_graph_replay_matches_eager_calls(path):
+    """The whole step (W compress calls + decode) captured into one CUDA graph after a warm-up call (which
+    uploads the pointer tables) and replayed twice gives the same bits as two eager steps."""
+    wl = inputs.small_decoder(num_workers=2)
+    r = parity.Runner(wl, max_chunks=4, path=path)
+    grads = [st.next() for st in r.streams]
+
+    def one_step():
+        for w in range(wl.num_workers):
+            r.tr.compress(w, grads[w], r.mom[w], r.payloads[w])
+        r.tr.decode_apply(r.payloads, r.params)
+
+    def reset(state=None):
+        for mw in r.mom:
+            for m in mw:
+                m.zero_()
+        if state is not None:
+            for p, s in zip(r.params, state):
+                p.copy_(s)
+
+    x0 = [p.clone() for p in r.params]
+    one_step()
+    one_step()
+    torch.cuda.synchronize()
+    want_x = [p.clone() for p in r.params]
+    want_m = [[m.clone() for m in mw] for mw in r.mom]
+    want_p = [p.clone() for p in r.payloads]
+    reset(x0)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        one_step()
+    reset(x0)  # capture records the launches without running them; start both replays from the same state
+    for p in r.payloads:
+        p.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert r.tr.device_status() == 0
+    assert all(torch.equal(a, b) for a, b in zip(want_x, r.params))
+    assert all(torch.equal(a, b) for aw, bw in zip(want_m, r.mom) for a, b in zip(aw, bw))
+    assert all(torch.equal(a, b) for a, b in zip(want_p, r.payloads))
+    r.close()
+
+
 @pytest.mark.parametrize("k", [32, 128])
 def test_decode_fan_in_64_workers(k):
     """Config 5's W=64 cell on the 4096 x 4096 matrix: one step from zero momentum (m = g), every
