@@ -3,6 +3,8 @@
 The product is ``libdemo_b200.so`` (hand-written CUDA for sm_100a behind ``include/demo.h``).
 This package only marshals arguments: every step of the path runs in the library's kernels.
 """
+# ``paper_2411_19870_b200.distributed`` (one worker per rank, all-gather of the payloads) is imported on
+# demand: it needs ``torch.distributed``.
 from .binding import (  # noqa: F401
     DEMO_BF16,
     DEMO_F32,

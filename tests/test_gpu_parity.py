@@ -233,6 +233,42 @@ def test_step_host_matches_separate_calls():
     r.close()
 
 
+def test_one_worker_per_rank_in_a_world_of_one():
+    """The deployed form (one worker per rank, NCCL all-gather of the payloads, decode on every rank)
+    through a single-rank NCCL group: same bits as compress + decode called directly with W = 1."""
+    import os
+
+    import torch.distributed as dist
+
+    from paper_2411_19870_b200.distributed import DistributedDemo
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(35500 + (os.getpid() % 2000))
+    wl = inputs.small_decoder(num_workers=1)
+    r = parity.Runner(wl, max_chunks=8)
+    grads = r.streams[0].next()
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        dd = DistributedDemo(wl.shapes, chunk=wl.chunk, topk=wl.topk, beta=wl.beta, lr=wl.lr, weight_decay=wl.weight_decay,
+                             grad_dtype=r.tr.cfg.grad_dtype)
+        mom = [torch.zeros_like(m) for m in r.mom[0]]
+        params = [p.clone() for p in r.params]
+        for _ in range(2):
+            dd.step(grads, mom, params)
+        torch.cuda.synchronize()
+        assert dd.tr.device_status() == 0
+        for _ in range(2):
+            r.step(check=True, grads=[grads])
+        torch.cuda.synchronize()
+        assert all(torch.equal(a, b) for a, b in zip(params, r.params))
+        assert all(torch.equal(a, b) for a, b in zip(mom, r.mom[0]))
+        assert torch.equal(dd.slices[0], r.payloads[0])
+        dd.close()
+    finally:
+        dist.destroy_process_group()
+    r.close()
+
+
 @pytest.mark.parametrize("path", [None, demo.DEMO_PATH_GENERIC])
 def test_cuda_graph_replay_matches_eager_calls(path):
     """The whole step (W compress calls + decode) captured into one CUDA graph after a warm-up call (which
