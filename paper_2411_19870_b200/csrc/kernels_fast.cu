@@ -332,18 +332,19 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             sb.sync();
             unsigned lmin;
             {
-                const unsigned okey = (NW > 1) ? tk[t ^ 32] : tkey;
-                unsigned gtc = 0, gto = 0;
-                const uint4 *t4 = reinterpret_cast<const uint4 *>(tk);
+                // bit-by-bit search, most significant first, for the largest L (low 15 mantissa bits zero)
+                // that still has k_eff maxima at or above it: every warp holds all S keys (its own and
+                // the partner warp's), so two ballots count them without a second exchange
+                const unsigned okey = (NW > 1) ? tk[t ^ 32] : 0u;
+                unsigned prefix = 0u;
 #pragma unroll
-                for (int j4 = 0; j4 < S / 4; ++j4) {
-                    const uint4 o = t4[j4];
-                    gtc += (o.x > tkey) + (o.y > tkey) + (o.z > tkey) + (o.w > tkey);
-                    if (NW > 1) gto += (o.x > okey) + (o.y > okey) + (o.z > okey) + (o.w > okey);
+                for (int b = 30; b >= 15; --b) {
+                    const unsigned cand = prefix | (1u << b);
+                    unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand));
+                    if (NW > 1) cnt += __popc(__ballot_sync(0xffffffffu, okey >= cand));
+                    prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
                 }
-                unsigned cnd = (gtc < (unsigned)k_eff) ? tkey : 0xffffffffu;
-                if (NW > 1) cnd = min(cnd, (gto < (unsigned)k_eff) ? okey : 0xffffffffu);
-                lmin = __reduce_min_sync(0xffffffffu, cnd);
+                lmin = prefix;
             }
             const float L = __uint_as_float(lmin);
             // candidates: coefficients with magnitude >= L (at least k_eff of them exist).
