@@ -336,9 +336,15 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                 // that still has k_eff maxima at or above it: every warp holds all S keys (its own and
                 // the partner warp's), so two ballots count them without a second exchange
                 const unsigned okey = (NW > 1) ? tk[t ^ 32] : 0u;
-                unsigned prefix = 0u;
-#pragma unroll
-                for (int b = 30; b >= 15; --b) {
+                // the answer lies between the smallest and the largest maximum: their common leading
+                // bits are settled, the search starts at the first bit where the two differ
+                const unsigned both_min = min(tkey, (NW > 1) ? okey : tkey), both_max = max(tkey, okey);
+                const unsigned lo_all = __reduce_min_sync(0xffffffffu, both_min);
+                const unsigned hi_all = __reduce_max_sync(0xffffffffu, both_max);
+                const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
+                unsigned prefix = lo_all & ~((2u << b0) - 1u);
+#pragma unroll 1
+                for (int b = b0; b >= 15; --b) {
                     const unsigned cand = prefix | (1u << b);
                     unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand));
                     if (NW > 1) cnt += __popc(__ballot_sync(0xffffffffu, okey >= cand));
