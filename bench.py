@@ -179,6 +179,10 @@ def run_ours(args, rank, world):
                             grad_dtype=demo.DEMO_BF16 if gbytes == 2 else demo.DEMO_F32, device=local)
     if args.path == "generic":
         tr.set_path(demo.DEMO_PATH_GENERIC)
+    if args.basis == "identity":
+        tr.set_basis(torch.eye(wl.chunk))
+    elif args.basis == "random":  # Gaussian draws seeded by a step number, orthonormalised on the device
+        tr.set_basis_gaussian(inputs.basis_gaussian(1, wl.chunk))
     params = inputs.make_params(wl, dev)
     mom = [inputs.make_momentum(wl, dev) for _ in range(W)]
     grads = [inputs.GradStream(wl, w, dev).next() for w in range(W)]  # one seeded set per worker, reused
@@ -282,7 +286,8 @@ def run_ours(args, rank, world):
                        "num_workers": W, "beta": wl.beta, "grad_dtype": "bf16" if gbytes == 2 else "f32",
                        "parallelism": "replicas only (one GPU per replica, no collective)" if world > 1 else "1 GPU",
                        "worker_params_per_s": value * W, "l2": "inputs (%.1f GB resident in HBM) are larger than the 126 MB L2; no flush needed" % (
-                           (W * P * (gbytes + 4) + 4 * P + W * tr.payload_bytes) / 1e9), "kernel_path": args.path},
+                           (W * P * (gbytes + 4) + 4 * P + W * tr.payload_bytes) / 1e9), "kernel_path": args.path,
+                       "basis": args.basis},
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
         }
         if base is not None:
@@ -399,6 +404,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="decoder_1b")
     ap.add_argument("--path", default="auto", choices=["auto", "generic"])
+    ap.add_argument("--basis", default="dct", choices=["dct", "identity", "random"],
+                    help="transform basis; anything but dct takes the dense-transform kernels (not the headline)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -72,6 +72,12 @@ cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count
 cudaError_t demo_launch_compress_fast128(const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
 cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream);
 
+// Tensor-core kernels for 2-D tensors under a caller-supplied basis (kernels_tc.cu): tcgen05 MMAs with
+// 3xTF32 splitting, chunk size 64 only.
+bool demo_tc_supported(int s);
+cudaError_t demo_launch_compress_tc(const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
+cudaError_t demo_launch_decode_tc(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream);
+
 // Self-test of the bounded wait (kernels_fast.cu): one CTA waits, for at most `limit_cycles`, on an
 // mbarrier that nothing completes, records DEMO_DEV_TIMEOUT in *status and returns.
 cudaError_t demo_launch_wait_selftest(int *status, long long limit_cycles, cudaStream_t stream);

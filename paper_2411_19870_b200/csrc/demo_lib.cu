@@ -337,6 +337,13 @@ static bool use_fast_path(const demo_ctx *ctx)
     return ctx->path == DEMO_PATH_AUTO && !ctx->custom_basis && demo_fast_supported(s) && (s != 128 || ctx->encode);
 }
 
+// A caller-supplied basis has no fast factorisation: its dense transforms run on the tensor cores where
+// there is a kernel for the chunk size, else on the CUDA cores.
+static bool use_tc_path(const demo_ctx *ctx)
+{
+    return ctx->path == DEMO_PATH_AUTO && ctx->custom_basis && demo_tc_supported(ctx->cfg.chunk);
+}
+
 demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grads, float *const *momentum,
                           void *payload_out, void *cuda_stream)
 {
@@ -391,6 +398,8 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
         a.n_chunks = ctx->chunks2d;
         if (use_fast_path(ctx))
             err = demo_launch_compress_fast(s, a, ctx->sm_count, stream);
+        else if (use_tc_path(ctx))
+            err = demo_launch_compress_tc(a, ctx->sm_count, stream);
         else
             err = demo_launch_compress_generic(s, 1, a, ctx->sm_count, stream);
         ctx->launches += 1;
@@ -458,6 +467,8 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
         a.n_chunks = ctx->chunks2d;
         if (use_fast_path(ctx))
             err = demo_launch_decode_fast(s, a, ctx->sm_count, stream);
+        else if (use_tc_path(ctx))
+            err = demo_launch_decode_tc(a, ctx->sm_count, stream);
         else
             err = demo_launch_decode_generic(s, 1, a, ctx->sm_count, stream);
         ctx->launches += 1;

@@ -27,36 +27,6 @@ namespace {
 using namespace fastk;
 
 constexpr int CAP = 128;                          // candidate capacity of the fast top-k
-// A CTA hosts NCH independent "slots" of S threads, one chunk each.  Threads of a slot meet at the
-// slot's own named barrier (a warp-level barrier when the slot is a single warp); all slots meet once
-// per chunk at the CTA barrier, which keeps the warps of the CTA in the same region of the (large,
-// fully unrolled) code so that instruction fetches are shared instead of streamed once per warp.
-template <int S>
-struct SlotBarrier {
-    int id;  // named barrier 1..15
-    __device__ __forceinline__ void sync() const
-    {
-        if (S == 32)
-            __syncwarp();
-        else
-            asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(S) : "memory");
-    }
-    __device__ __forceinline__ bool sync_and(bool pred) const
-    {
-        if (S == 32) return __all_sync(0xffffffffu, pred);
-        unsigned r;
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\t"
-            "setp.ne.u32 q, %3, 0;\n\t"
-            "bar.red.and.pred p, %1, %2, q;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(r)
-            : "r"(id), "n"(S), "r"((unsigned)pred)
-            : "memory");
-        return r != 0;
-    }
-};
-
 template <int S>
 struct Cfg {
     static constexpr int XS = S + 4;  // row stride of the transpose tile: conflict-free scalar
@@ -64,62 +34,6 @@ struct Cfg {
     static constexpr int NW = S / 32;
     static constexpr int LOG2S = (S == 64) ? 6 : 5;
 };
-
-// ------------------------------------------------------------------------------------------------
-// Exact radix select over the S x S coefficient tile stored at X[u*XS + v] (S threads).  Returns the
-// magnitude key of the k-th largest and how many coefficients equal to it belong to the top-k.
-// ------------------------------------------------------------------------------------------------
-template <int S>
-__device__ __forceinline__ void radix_select_tile(const float *X, int k_eff, unsigned *hist, unsigned *s_state,
-                                                  unsigned *thr, unsigned *need_eq, int t, SlotBarrier<S> sb)
-{
-    constexpr int XS = Cfg<S>::XS;
-    if (t == 0) {
-        s_state[0] = 0u;
-        s_state[1] = (unsigned)k_eff;
-    }
-#pragma unroll 1
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = 24 - 8 * pass;
-        const unsigned mask = (pass == 0) ? 0u : (0xffffffffu << (shift + 8));
-        for (int i = t; i < 256; i += S) hist[i] = 0u;
-        sb.sync();
-        const unsigned prefix = s_state[0];
-#pragma unroll 1
-        for (int v = 0; v < S; ++v) {
-            const unsigned key = mag_key(X[t * XS + v]);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
-        sb.sync();
-        if (t < 32) {
-            const unsigned rem = s_state[1];
-            unsigned local = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) local += hist[255 - 8 * t - j];
-            unsigned inc = local;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                unsigned n = __shfl_up_sync(0xffffffffu, inc, d);
-                if (t >= d) inc += n;
-            }
-            const unsigned before = inc - local;
-            if (before < rem && rem <= inc) {
-                unsigned cum = before;
-                int b = 255 - 8 * t;
-                for (int j = 0; j < 8; ++j, --b) {
-                    const unsigned h = hist[b];
-                    if (cum + h >= rem) break;
-                    cum += h;
-                }
-                s_state[1] = rem - cum;
-                s_state[0] = prefix | ((unsigned)b << shift);
-            }
-        }
-        sb.sync();
-    }
-    *thr = s_state[0];
-    *need_eq = s_state[1];
-}
 
 // Bytes of the tile area of the compress kernel: the staged m and g tiles, or the padded transpose
 // tile that later aliases them, whichever is larger.
@@ -483,7 +397,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
         if (use_fallback) {
             sb.sync();  // coefficient tile complete in X
             unsigned thr, need_eq;
-            radix_select_tile<S>(X, k_eff, hist, misc, &thr, &need_eq, t, sb);
+            radix_select_tile<S, XS>(X, k_eff, hist, misc, &thr, &need_eq, t, sb);
             unsigned gt = 0, eq = 0;
 #pragma unroll 1
             for (int v = 0; v < S; ++v) {

@@ -396,24 +396,27 @@ def test_aggregation_and_phi_variants(s, agg, phi):
         r.close()
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("s", [8, 64, 128])
-def test_identity_basis(s):
-    """Section 4.2's baseline P = I: top-k of the momentum itself, sign of the scattered sum."""
+def test_identity_basis(s, path):
+    """Section 4.2's baseline P = I: top-k of the momentum itself, sign of the scattered sum (at s = 64
+    on the tensor-core kernels by default, on the CUDA-core dense kernels when forced)."""
     shapes = [(2 * s, 3 * s), (2 * s,)]
     wl = inputs.Workload("ident", shapes, chunk=s, topk=max(2, s // 2), num_workers=3, grad_kind="normal", grad_std=0.01)
-    r = parity.Runner(wl, max_chunks=10**9, basis=np.eye(s))
+    r = parity.Runner(wl, max_chunks=10**9, basis=np.eye(s), path=path)
     r.step()
     r.step()
     assert torch.equal(r.tr.get_basis(), torch.eye(s))
     r.close()
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("s", [8, 32, 64, 128])
-def test_random_orthonormal_basis_redrawn_every_step(s):
+def test_random_orthonormal_basis_redrawn_every_step(s, path):
     """Gaussian matrix seeded by the step number, Gram-Schmidt on the device vs the oracle's own."""
     shapes = [(2 * s, 3 * s), (4 * s,)]
     wl = inputs.Workload("randp", shapes, chunk=s, topk=max(2, s // 2), num_workers=2, grad_kind="normal", grad_std=0.01)
-    r = parity.Runner(wl, max_chunks=10**9)
+    r = parity.Runner(wl, max_chunks=10**9, path=path)
     for step in (1, 2, 3):
         r.set_basis(gauss=inputs.basis_gaussian(step, s).numpy())
         P = r.tr.get_basis().double().numpy()
@@ -423,6 +426,25 @@ def test_random_orthonormal_basis_redrawn_every_step(s):
     # back to the DCT (and, where there is one, to the fast kernel family)
     r.set_basis()
     r.step()
+    r.close()
+
+
+@pytest.mark.parametrize("k,alpha,agg,phi", [(32, None, 0, 0), (1, 0.2, 1, 1), (200, None, 2, 0), (4096, 0.5, 2, 1)])
+def test_tensor_core_kernels_under_a_random_basis(k, alpha, agg, phi):
+    """s = 64 with a caller-supplied basis runs on the tcgen05 kernels: odd number of chunks (the last
+    pair is half empty), several tensors, bf16 gradients, k below and above 64 up to lossless, alpha and
+    the aggregation / phi variants, five workers with colliding coordinates."""
+    s = 64
+    shapes = [(s, 3 * s), (2 * s, 2 * s), (s,)]  # 3 + 4 = 7 chunks: an odd count
+    wl = inputs.Workload("tc", shapes, chunk=s, topk=k, num_workers=5, grad_kind="normal", grad_std=0.01)
+    r = parity.Runner(wl, max_chunks=10**9, gauss=inputs.basis_gaussian(11, s).numpy(), alpha=alpha, agg=agg, phi=phi)
+    base = [g for g in r.streams[0].next()]
+    grads = [[(b.float() + 0.3 * o.float()).to(b.dtype) for b, o in zip(base, st.next())] for st in r.streams]
+    before = r.tr.launch_count
+    r.step(grads=grads)
+    r.step(grads=grads)
+    assert r.tr.launch_count - before == 2 * (wl.num_workers + 1) * 2  # 2-D list + 1-D list per call
+    assert r.tr.device_status() == 0
     r.close()
 
 
