@@ -212,8 +212,9 @@ demo_status demo_set_decode_mode(demo_ctx *ctx, int32_t aggregation, int32_t phi
 /* Other orthonormal bases (Section 4.2, "Choice of Linear Projections": identity mapping, random
  * orthonormal projection).  The basis is an s x s row-major fp32 matrix P whose ROWS are the basis
  * vectors; it replaces the DCT matrix on both axes of a 2-D chunk (Q = P B P^T, inverse P^T Q P) and on
- * 1-D segments (q = P b).  While a caller-supplied basis is active every tensor goes through the
- * dense-transform kernels (the fast kernels hard-code the DCT factorisation).
+ * 1-D segments (q = P b).  While a caller-supplied basis is active the fast kernels (which hard-code the
+ * DCT factorisation) are out: 2-D tensors at chunk size 64 run on tensor-core kernels (3xTF32, fp32
+ * accuracy), everything else on the dense CUDA-core kernels; DEMO_PATH_GENERIC forces the latter.
  *
  * demo_set_basis: basis_host = HOST pointer to P, read during the call and not retained; NULL restores
  * the DCT.  The rows must be orthonormal to 1e-5 (INVALID_ARG otherwise).  The upload is enqueued on
