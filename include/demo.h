@@ -108,7 +108,10 @@ demo_status demo_payload_layout(const demo_ctx *ctx, int32_t tensor, int64_t *fi
  *   cuda_stream  cudaStream_t (NULL = default stream)
  * Device buffers must be 16-byte aligned and must not alias each other.  The pointer arrays are
  * host memory, read during the call and not retained.  Calls on one context must be issued in
- * stream order (one stream, or streams the caller orders).  Errors: INVALID_ARG, CUDA.
+ * stream order (one stream, or streams the caller orders).  Gradients or momenta that hold NaN or Inf
+ * give unspecified values for the chunks they touch, but every chunk still gets k_eff records with
+ * distinct, ascending, in-range indices, other chunks are unaffected and nothing hangs or traps.
+ * Errors: INVALID_ARG, CUDA.
  */
 demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grads,
                           float *const *momentum, void *payload_out, void *cuda_stream);

@@ -313,12 +313,17 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                 if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
             }
             sb.sync();
-            unsigned n_w[NW];
+            unsigned n_w[NW], n_all = 0;
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
                 n_w[w] = misc[w];
+                n_all += n_w[w];
                 use_fallback = use_fallback || (n_w[w] > CAPW);
             }
+            // Fewer than k_eff candidates cannot happen with finite data (the k_eff largest maxima are
+            // candidates themselves); with NaN coefficients the comparisons above fail, and the select on
+            // the integer keys, which orders every bit pattern, takes over.
+            use_fallback = use_fallback || (n_all < (unsigned)k_eff);
             if (!use_fallback) {
                 // rank among all candidates by magnitude only.  If exactly k_eff candidates have
                 // fewer than k_eff larger ones, no tie straddles the threshold and that set is the

@@ -464,6 +464,43 @@ def test_basis_argument_errors_keep_the_previous_basis():
     r.close()
 
 
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("s", [64, 128])
+def test_nan_and_inf_gradients_neither_hang_nor_corrupt_other_tensors(s, path):
+    """Results for chunks that contain NaN or Inf are unspecified, but the kernels must finish, every
+    chunk must still carry k_eff records with distinct, ascending, in-range indices (a consumer relies on
+    that), and tensors without such values must come out bit-identical to a clean run."""
+    shapes = [(2 * s, 2 * s), (2 * s, 4 * s), (2 * s,), (4 * s,)]
+    wl = inputs.Workload("nonfinite", shapes, chunk=s, topk=8, num_workers=2, grad_kind="normal", grad_std=0.01)
+    clean = parity.Runner(wl, max_chunks=10**9, path=path)
+    dirty = parity.Runner(wl, max_chunks=10**9, path=path)
+    grads = [st.next() for st in clean.streams]
+    bad = [[g.clone() for g in gw] for gw in grads]
+    for w in range(wl.num_workers):
+        bad[w][0][3, 5] = float("nan")          # one chunk of the first matrix
+        bad[w][0][s + 1, s + 2] = float("inf")  # another one
+        bad[w][0][s + 7, 9] = float("-inf")     # and a third
+        bad[w][2][3] = float("nan")             # one segment of the first vector
+    clean.step(check=True, grads=grads)
+    dirty.step(check=False, grads=bad)
+    torch.cuda.synchronize()
+    assert dirty.tr.device_status() == 0
+    for tns in (1, 3):  # untouched tensors: same bits as the clean run
+        assert torch.equal(clean.params[tns], dirty.params[tns])
+        for w in range(wl.num_workers):
+            assert torch.equal(clean.mom[w][tns], dirty.mom[w][tns])
+    for w in range(wl.num_workers):
+        raw = dirty.payloads[w].cpu().numpy().view(parity.orc.RECORD_DTYPE)
+        for tns, shp in enumerate(shapes):
+            first, n_chunks, k_eff = dirty.layout[tns]
+            idx = raw["idx"][first:first + n_chunks * k_eff].reshape(n_chunks, k_eff)
+            M = s * s if len(shp) == 2 else s
+            assert idx.min() >= 0 and idx.max() < M
+            assert np.all(np.diff(idx, axis=1) > 0)
+    clean.close()
+    dirty.close()
+
+
 def test_bounded_wait_expires_into_a_status_and_the_context_survives():
     """Failure detection without a GPU fault: a wait that nothing satisfies runs out after ~1 ms, the
     kernel returns, the sticky status says TIMEOUT, and the same context then computes correctly."""
