@@ -465,7 +465,7 @@ def test_basis_argument_errors_keep_the_previous_basis():
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("s", [64, 128])
+@pytest.mark.parametrize("s", [8, 32, 64, 128])
 def test_nan_and_inf_gradients_neither_hang_nor_corrupt_other_tensors(s, path):
     """Results for chunks that contain NaN or Inf are unspecified, but the kernels must finish, every
     chunk must still carry k_eff records with distinct, ascending, in-range indices (a consumer relies on
