@@ -119,6 +119,22 @@ def _tensor_ptrs(tensors) -> List[int]:
     return [int(t.data_ptr()) for t in tensors]
 
 
+def validate_tensors(tensors, shapes, dtype, device_index: Optional[int], what: str) -> None:
+    """The C ABI takes bare pointers, so the layout it assumes is checked here: one contiguous tensor per
+    shape, of the given dtype, on CUDA device ``device_index`` (``None``: any device; used by CPU tests)."""
+    if len(tensors) != len(shapes):
+        raise ValueError("%s: expected %d tensors, got %d" % (what, len(shapes), len(tensors)))
+    for i, (t, shp) in enumerate(zip(tensors, shapes)):
+        if tuple(t.shape) != tuple(shp):
+            raise ValueError("%s[%d]: shape %s, expected %s" % (what, i, tuple(t.shape), tuple(shp)))
+        if t.dtype != dtype:
+            raise ValueError("%s[%d]: dtype %s, expected %s" % (what, i, t.dtype, dtype))
+        if not t.is_contiguous():
+            raise ValueError("%s[%d]: not contiguous" % (what, i))
+        if device_index is not None and (not t.is_cuda or t.device.index != device_index):
+            raise ValueError("%s[%d]: on %s, expected cuda:%d" % (what, i, t.device, device_index))
+
+
 def decode_apply_static(shapes, payloads, params, *, chunk: int, topk: int, lr: float, weight_decay: float,
                         device: int = 0, stream=None) -> None:
     """``demo_decode_apply_static``: decode + update without a context and without any allocation by
@@ -159,11 +175,14 @@ class DemoTransform:
             self._ctx = ctypes.c_void_p()
             raise DemoError(st, "demo_init")
         self._ptr_cache = {}
+        self._payload_bytes = int(self.lib.demo_payload_bytes(self._ctx))
+        self._payload_ok = set()   # (data pointer, size) of payload buffers already checked
+        self._gdtype = torch.bfloat16 if grad_dtype == DEMO_BF16 else torch.float32
 
     # --- queries -------------------------------------------------------------------------------
     @property
     def payload_bytes(self) -> int:
-        return int(self.lib.demo_payload_bytes(self._ctx))
+        return self._payload_bytes
 
     def payload_layout(self, tensor: int):
         first, n_chunks, k_eff = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int32()
@@ -178,14 +197,32 @@ class DemoTransform:
         return int(self.lib.demo_launch_count(self._ctx))
 
     # --- marshalling helpers -------------------------------------------------------------------
-    def _array(self, key, tensors):
-        """Pointer array for a list of tensors, cached per list identity and data pointers."""
+    def _array(self, key, tensors, check=None):
+        """Pointer array for a list of tensors, cached per key and data pointers.  ``check`` = (shapes,
+        dtype, on_device) is verified whenever the pointers are new."""
         ptrs = tuple(_tensor_ptrs(tensors))
         hit = self._ptr_cache.get(key)
         if hit is None or hit[0] != ptrs:
+            if check is not None:
+                shapes, dtype, on_device = check
+                validate_tensors(tensors, shapes, dtype, self.device if on_device else None, str(key))
             hit = (ptrs, _ptr_array(ptrs))
             self._ptr_cache[key] = hit
         return hit[1]
+
+    def _check_payloads(self, payloads) -> None:
+        for i, p in enumerate(payloads):  # (the library itself checks their number)
+            self._check_payload(p, "payloads[%d]" % i)
+
+    def _check_payload(self, p, what: str) -> None:
+        ptr = (p.data_ptr(), p.numel())
+        if ptr in self._payload_ok:
+            return
+        if p.dtype != torch.uint8 or not p.is_contiguous() or p.numel() < self.payload_bytes or not p.is_cuda \
+                or p.device.index != self.device:
+            raise ValueError("%s: need a contiguous uint8 tensor of at least %d bytes on cuda:%d"
+                             % (what, self.payload_bytes, self.device))
+        self._payload_ok.add(ptr)
 
     @staticmethod
     def _stream(stream) -> ctypes.c_void_p:
@@ -197,15 +234,17 @@ class DemoTransform:
 
     # --- the ABI calls -------------------------------------------------------------------------
     def compress(self, worker: int, grads, momentum, payload_out, stream=None) -> None:
-        st = self.lib.demo_compress(self._ctx, worker, self._array(("g", worker), grads),
-                                    self._array(("m", worker), momentum), ctypes.c_void_p(payload_out.data_ptr()),
-                                    self._stream(stream))
+        self._check_payload(payload_out, "payload_out")
+        st = self.lib.demo_compress(self._ctx, worker, self._array(("g", worker), grads, (self.shapes, self._gdtype, True)),
+                                    self._array(("m", worker), momentum, (self.shapes, torch.float32, True)),
+                                    ctypes.c_void_p(payload_out.data_ptr()), self._stream(stream))
         if st != 0:
             raise DemoError(st, "demo_compress")
 
     def decode_apply(self, payloads, params, stream=None) -> None:
+        self._check_payloads(payloads)
         st = self.lib.demo_decode_apply(self._ctx, self._array("p", payloads), len(payloads),
-                                        self._array("x", params), self._stream(stream))
+                                        self._array("x", params, (self.shapes, torch.float32, True)), self._stream(stream))
         if st != 0:
             raise DemoError(st, "demo_decode_apply")
 

@@ -90,3 +90,25 @@ def test_no_cpu_fallback_without_device(lib):
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(RuntimeError):
         demo.load_library(str(tmp_path / "libnot_there.so"))
+
+
+def test_binding_checks_the_layout_the_abi_assumes():
+    """The C ABI takes bare pointers; the binding refuses tensors whose layout differs from the shapes
+    the context was built for (checked without a GPU: the device test is skipped with None)."""
+    import torch
+
+    from paper_2411_19870_b200.binding import validate_tensors
+
+    shapes = [(4, 6), (8,)]
+    good = [torch.zeros(4, 6), torch.zeros(8)]
+    validate_tensors(good, shapes, torch.float32, None, "m")
+    with pytest.raises(ValueError, match="expected 2 tensors"):
+        validate_tensors(good[:1], shapes, torch.float32, None, "m")
+    with pytest.raises(ValueError, match="shape"):
+        validate_tensors([torch.zeros(6, 4), good[1]], shapes, torch.float32, None, "m")
+    with pytest.raises(ValueError, match="dtype"):
+        validate_tensors([good[0].double(), good[1]], shapes, torch.float32, None, "m")
+    with pytest.raises(ValueError, match="not contiguous"):
+        validate_tensors([torch.zeros(6, 4).t(), good[1]], shapes, torch.float32, None, "m")
+    with pytest.raises(ValueError, match="expected cuda:0"):
+        validate_tensors(good, shapes, torch.float32, 0, "m")

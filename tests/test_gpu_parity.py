@@ -201,6 +201,30 @@ def test_abi_runtime_argument_errors():
     tr.close()
 
 
+def test_binding_refuses_tensors_of_the_wrong_layout():
+    shapes = [(64, 128)]
+    tr = demo.DemoTransform(shapes, chunk=64, topk=8, beta=0.9, lr=1e-3, weight_decay=0.0, num_workers=1)
+    g = [torch.zeros(64, 128, device="cuda", dtype=torch.bfloat16)]
+    m = [torch.zeros(64, 128, device="cuda")]
+    p = torch.zeros(tr.payload_bytes, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ValueError, match="not contiguous"):
+        tr.compress(0, [torch.zeros(128, 64, device="cuda", dtype=torch.bfloat16).t()], m, p)
+    with pytest.raises(ValueError, match="dtype"):
+        tr.compress(0, [g[0].float()], m, p)
+    with pytest.raises(ValueError, match="shape"):
+        tr.compress(0, g, [torch.zeros(128, 64, device="cuda")], p)
+    with pytest.raises(ValueError, match="expected cuda:0"):
+        tr.compress(0, g, [torch.zeros(64, 128)], p)
+    with pytest.raises(ValueError, match="payload_out"):
+        tr.compress(0, g, m, p[:-8])
+    with pytest.raises(ValueError, match="payloads"):
+        tr.decode_apply([p.cpu()], m)
+    tr.compress(0, g, m, p)
+    tr.decode_apply([p], m)
+    assert tr.device_status() == 0
+    tr.close()
+
+
 def test_bad_payload_index_is_reported_not_faulted():
     shapes = [(64, 64)]
     tr = demo.DemoTransform(shapes, chunk=64, topk=4, beta=0.9, lr=1e-3, weight_decay=0.0, num_workers=1)
