@@ -27,6 +27,8 @@ namespace {
 using namespace fastk;
 
 constexpr int S = 128, H = 64, XS = S + 4, M = S * S, THREADS = 256;
+constexpr int CAP128 = 256;           // candidate capacity of the fast top-k (one per thread)
+constexpr int CAP128P = CAP128 + 4;   // padded for 128-bit key loads
 using SC = fdct::ScaleOrtho<S>;
 
 __device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned *warp_tot /*[8]*/)
@@ -72,7 +74,7 @@ constexpr size_t compress128_tile_bytes()
 template <typename GT>
 constexpr size_t compress128_smem()
 {
-    return compress128_tile_bytes<GT>() + (256 + 8 + 4) * 4 + 128 * 16 + 16;
+    return compress128_tile_bytes<GT>() + (256 + 8 + 4) * 4 + 128 * 16 + 3 * CAP128P * 4 + 16;
 }
 
 template <typename GT>
@@ -87,7 +89,10 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
     unsigned *warp_tot = hist + 256;                                                         // [8]
     unsigned *s_state = warp_tot + 8;                                                        // [4]
     int4 *recs4 = reinterpret_cast<int4 *>(s_state + 4);                                     // [128]
-    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(recs4 + 128);
+    unsigned *cand_key = reinterpret_cast<unsigned *>(recs4 + 128);                          // [CAP128P]
+    float *cand_val = reinterpret_cast<float *>(cand_key + CAP128P);                         // [CAP128P]
+    int *cand_idx = reinterpret_cast<int *>(cand_val + CAP128P);                             // [CAP128P]
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(cand_idx + CAP128P);
 
     const int tid = threadIdx.x, h = tid >> 7, j = tid & 127;
     const uint32_t bar = smem_u32(bar_mem);
@@ -171,9 +176,112 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
             __syncthreads();
         }
 
-        // ---- exact top-k: radix select on the magnitude bits, then index-ordered compaction --------
-        unsigned thr, need_eq;
-        {
+        // ---- exact top-k ---------------------------------------------------------------------------
+        // thread tid scans the half row [tid/2][64*(tid&1) .. +64): flat indices 64*tid .. 64*tid+63.
+        // Fast path (k_eff <= 256): the k_eff-th largest of the 256 per-thread maxima is a lower bound L of
+        // the k_eff-th largest coefficient (256 groups: the bound is tight, a few dozen candidates); the
+        // candidates are listed in index order and ranked exactly, ties to the lowest index.  Everything
+        // compares integer magnitude keys, so NaN and Inf are ordered like any other bit pattern.  More
+        // than CAP128 candidates (tied or degenerate chunks) or k_eff > 256: radix select below.
+        bool use_radix = k_eff > 256;
+        if (!use_radix) {
+            const float4 *mine4 = reinterpret_cast<const float4 *>(X + (tid >> 1) * XS + 64 * (tid & 1));
+            const int lane = tid & 31, warp = tid >> 5;
+            // the two halves of a row sit 256 bytes apart (same banks): the odd one starts 4 pieces later
+            const int rot = 4 * (tid & 1);
+            unsigned tkey = 0u;
+#pragma unroll
+            for (int i4 = 0; i4 < 16; ++i4) {
+                const float4 f = mine4[(i4 + rot) & 15];
+                tkey = max(max(tkey, mag_key(f.x)), max(mag_key(f.y), max(mag_key(f.z), mag_key(f.w))));
+            }
+            hist[tid] = tkey;
+            __syncthreads();
+            if (warp == 0) {
+                unsigned k8[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) k8[i] = hist[lane + 32 * i];
+                unsigned lo = k8[0], hi = k8[0];
+#pragma unroll
+                for (int i = 1; i < 8; ++i) {
+                    lo = min(lo, k8[i]);
+                    hi = max(hi, k8[i]);
+                }
+                lo = __reduce_min_sync(0xffffffffu, lo);
+                hi = __reduce_max_sync(0xffffffffu, hi);
+                const int b0 = 31 - __clz((lo ^ hi) | 0x8000u);  // >= 15
+                unsigned prefix = lo & ~((2u << b0) - 1u);
+#pragma unroll 1
+                for (int b = b0; b >= 15; --b) {
+                    const unsigned cand = prefix | (1u << b);
+                    unsigned cnt = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) cnt += __popc(__ballot_sync(0xffffffffu, k8[i] >= cand));
+                    prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
+                }
+                if (lane == 0) s_state[2] = prefix;
+            }
+            __syncthreads();
+            const unsigned lmin = s_state[2];
+            // candidates of this thread as a bit mask over its 64 values
+            unsigned long long mask = 0ull;
+#pragma unroll
+            for (int i4 = 0; i4 < 16; ++i4) {
+                const float4 f = mine4[i4];
+                const unsigned nib = (unsigned)(mag_key(f.x) >= lmin) | ((unsigned)(mag_key(f.y) >= lmin) << 1) |
+                                     ((unsigned)(mag_key(f.z) >= lmin) << 2) | ((unsigned)(mag_key(f.w) >= lmin) << 3);
+                mask |= (unsigned long long)nib << (4 * i4);
+            }
+            const unsigned cnt = (unsigned)__popcll(mask);
+            unsigned o = block_exclusive_scan(cnt, warp_tot);
+            if (tid == THREADS - 1) s_state[3] = o + cnt;
+            __syncthreads();
+            const unsigned n_cand = s_state[3];
+            use_radix = n_cand > (unsigned)CAP128 || n_cand < (unsigned)k_eff;
+            if (!use_radix) {
+                const float *mine = reinterpret_cast<const float *>(mine4);
+                while (mask) {
+                    const int e = __ffsll((long long)mask) - 1;
+                    mask &= mask - 1ull;
+                    const float val = mine[e];
+                    cand_key[o] = mag_key(val);
+                    cand_val[o] = val;
+                    cand_idx[o] = 64 * tid + e;
+                    ++o;
+                }
+                if (tid < 4) cand_key[n_cand + tid] = 0u;  // pad for the vector loads
+                __syncthreads();
+                // exact rank of candidate tid among all candidates (list order = index order)
+                bool sel = false;
+                if ((unsigned)tid < n_cand) {
+                    const unsigned key = cand_key[tid];
+                    unsigned rank = 0;
+                    const uint4 *keys4 = reinterpret_cast<const uint4 *>(cand_key);
+                    const unsigned n4 = (n_cand + 3u) >> 2;
+                    for (unsigned c4 = 0; c4 < n4; ++c4) {
+                        const uint4 k4 = keys4[c4];
+                        const unsigned j0 = 4u * c4;
+                        rank += (k4.x > key) || (k4.x == key && j0 < (unsigned)tid);
+                        rank += (k4.y > key) || (k4.y == key && j0 + 1u < (unsigned)tid);
+                        rank += (k4.z > key) || (k4.z == key && j0 + 2u < (unsigned)tid);
+                        rank += (k4.w > key) || (k4.w == key && j0 + 3u < (unsigned)tid);
+                    }
+                    sel = rank < (unsigned)k_eff;
+                }
+                const unsigned pos = block_exclusive_scan(sel ? 1u : 0u, warp_tot);
+                if (sel) {
+                    DemoRecord r;
+                    r.idx = cand_idx[tid];
+                    r.val = cand_val[tid];
+                    rec[pos] = r;
+                    if (k_eff <= 128)
+                        recs4[pos] = make_int4((r.idx >> 7) * XS, (r.idx & 127) * S, __float_as_int(a.alpha * r.val), 0);
+                }
+            }
+        }
+        // ---- radix select on the magnitude bits, then index-ordered compaction -----------------------
+        if (use_radix) {
+            unsigned thr, need_eq;
             if (tid == 0) {
                 s_state[0] = 0u;
                 s_state[1] = (unsigned)k_eff;
