@@ -27,6 +27,10 @@ namespace {
 using namespace fastk;
 
 constexpr int S = 128, H = 64, XS = S + 4, M = S * S, THREADS = 256;
+// The decode tile is only ever accessed element-wise: an odd row stride keeps a warp whose lanes walk 32
+// different rows (the row pass) on 32 different banks; S + 4 (compress: 128-bit row accesses) gives 4-way
+// conflicts there.
+constexpr int XSD = S + 1;
 constexpr int CAP128 = 256;           // candidate capacity of the fast top-k (one per thread)
 constexpr int CAP128P = CAP128 + 4;   // padded for 128-bit key loads
 using SC = fdct::ScaleOrtho<S>;
@@ -437,14 +441,14 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
     }
 }
 
-constexpr size_t decode128_smem(bool counts) { return (size_t)S * XS * 4 + 16 + (counts ? (size_t)M * 2 : 0); }
+constexpr size_t decode128_smem(bool counts) { return (size_t)S * XSD * 4 + 16 + (counts ? (size_t)M * 2 : 0); }
 
 __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float *St = reinterpret_cast<float *>(smem_raw);  // [128*132] aggregate / intermediate; later the x tile [128*128]
     float *Xt = St;
-    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XS);
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XSD);
     unsigned short *Cn = reinterpret_cast<unsigned short *>(bar_mem + 2);  // [M] senders per coordinate (agg == 2)
 
     const int tid = threadIdx.x, h = tid >> 7, j = tid & 127;
@@ -475,7 +479,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
         const char *tm_x = static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES;
         if (tid == 0) tma_prefetch_2d(tm_x, k1 * S, k0 * S);
 
-        for (int i = tid; i < S * XS / 4; i += THREADS) reinterpret_cast<float4 *>(St)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = tid; i < S * XSD / 4; i += THREADS) reinterpret_cast<float4 *>(St)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (counts)
             for (int i = tid; i < M; i += THREADS) Cn[i] = 0;
         __syncthreads();
@@ -492,7 +496,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
                     if (w0 + q < a.W) {
                         if (mine) {
                             if ((unsigned)r[q].idx < (unsigned)M) {
-                                St[(r[q].idx >> 7) * XS + (r[q].idx & 127)] += r[q].val;
+                                St[(r[q].idx >> 7) * XSD + (r[q].idx & 127)] += r[q].val;
                                 if (counts) Cn[r[q].idx] += 1;
                             } else {
                                 atomicMax(a.status, DEMO_DEV_PAYLOAD);
@@ -506,7 +510,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
         if (counts) {  // Sparse Top-k Averaging: sum / number of senders, 0/0 = 0
             for (int i = tid; i < M; i += THREADS) {
                 const unsigned short n = Cn[i];
-                if (n > 1) St[(i >> 7) * XS + (i & 127)] /= (float)n;
+                if (n > 1) St[(i >> 7) * XSD + (i & 127)] /= (float)n;
             }
             __syncthreads();
         }
@@ -515,8 +519,8 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
         bool arrived = true;
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
-            const int line = pass == 0 ? j * XS : j;   // start of line j
-            const int step = pass == 0 ? 1 : XS;       // distance between consecutive elements of the line
+            const int line = pass == 0 ? j * XSD : j;   // start of line j
+            const int step = pass == 0 ? 1 : XSD;       // distance between consecutive elements of the line
 #pragma unroll
             for (int p = 0; p < H; ++p) in[p] = St[line + (2 * p + h) * step];
             fence_proxy_async();
