@@ -227,32 +227,37 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
         unsigned n_cw = 0, off = 0;
         unsigned mlo = 0u, mhi = 0u;
         if (!use_fallback) {
-            // per-thread maximum magnitude: independent chains of 16 with 3-input max
-            float tm = 0.f;
+            // per-thread maximum magnitude: independent chains of 16 with 3-input max.  With S = 32 the two
+            // chains stay apart (two maxima per thread): 64 groups again, so that the bound is still useful
+            // at k_eff = 32.
+            float tm = 0.f, tm2 = 0.f;
 #pragma unroll
             for (int ch = 0; ch < S / 16; ++ch) {
                 const int b0 = 16 * ch;
                 float c = max3abs(q[b0], q[b0 + 1], q[b0 + 2]);
 #pragma unroll
                 for (int j = 3; j + 1 < 16; j += 2) c = max3f(c, fabsf(q[b0 + j]), fabsf(q[b0 + j + 1]));
-                tm = max3f(tm, c, fabsf(q[b0 + 15]));
+                if (S == 32 && ch == 1)
+                    tm2 = max3f(tm2, c, fabsf(q[b0 + 15]));
+                else
+                    tm = max3f(tm, c, fabsf(q[b0 + 15]));
             }
-            // L = the k_eff-th largest of the S per-thread maxima = the smallest maximum that has
-            // fewer than k_eff strictly larger ones.  Every warp ranks all S maxima (its own and the
-            // partner warp's) so that no second exchange is needed.
+            // L = the k_eff-th largest of the 64 maxima.  Every warp holds all of them -- its own and the
+            // partner warp's (S = 64), or its two per thread (S = 32) -- so that no second exchange is needed.
             const unsigned tkey = __float_as_uint(tm);
             unsigned *tk = reinterpret_cast<unsigned *>(tmax);
-            tk[t] = tkey;
-            sb.sync();
+            if (NW > 1) {
+                tk[t] = tkey;
+                sb.sync();
+            }
             unsigned lmin;
             {
                 // bit-by-bit search, most significant first, for the largest L (low 15 mantissa bits zero)
-                // that still has k_eff maxima at or above it: every warp holds all S keys (its own and
-                // the partner warp's), so two ballots count them without a second exchange
-                const unsigned okey = (NW > 1) ? tk[t ^ 32] : 0u;
+                // that still has k_eff maxima at or above it: two ballots per step count them
+                const unsigned okey = (NW > 1) ? tk[t ^ 32] : __float_as_uint(tm2);
                 // the answer lies between the smallest and the largest maximum: their common leading
                 // bits are settled, the search starts at the first bit where the two differ
-                const unsigned both_min = min(tkey, (NW > 1) ? okey : tkey), both_max = max(tkey, okey);
+                const unsigned both_min = min(tkey, okey), both_max = max(tkey, okey);
                 const unsigned lo_all = __reduce_min_sync(0xffffffffu, both_min);
                 const unsigned hi_all = __reduce_max_sync(0xffffffffu, both_max);
                 const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
@@ -260,8 +265,8 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
 #pragma unroll 1
                 for (int b = b0; b >= 15; --b) {
                     const unsigned cand = prefix | (1u << b);
-                    unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand));
-                    if (NW > 1) cnt += __popc(__ballot_sync(0xffffffffu, okey >= cand));
+                    const unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand)) +
+                                         __popc(__ballot_sync(0xffffffffu, okey >= cand));
                     prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
                 }
                 lmin = prefix;
