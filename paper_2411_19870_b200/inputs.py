@@ -162,7 +162,9 @@ class GradStream:
         self.row_factors = None
         if wl.grad_kind == "row_lognormal":
             rg = _gen(device, ROW_FACTOR_SEED)
-            self.row_factors = [torch.exp(torch.randn((shp[0], 1), generator=rg, device=device)) for shp in wl.shapes]
+            # one factor per row of a matrix, per element of a vector (its "rows" have one element)
+            self.row_factors = [torch.exp(torch.randn((shp[0], 1) if len(shp) == 2 else (shp[0],), generator=rg, device=device))
+                                for shp in wl.shapes]
         self.tie_gen = _gen(device, TIE_MASK_SEED + worker) if wl.grad_kind == "student_t_ties" else None
 
     def _draw(self, t: int, shp: Shape) -> torch.Tensor:
