@@ -506,6 +506,28 @@ def test_tensor_core_kernels_under_a_random_basis(k, alpha, agg, phi):
     r.close()
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_randomized_tensor_core_cases(seed):
+    """Seeded random configurations at s = 64 under a random orthonormal basis (tensor-core kernels), the
+    basis redrawn before each of the two steps."""
+    rng = np.random.default_rng(5000 + seed)
+    s = 64
+    k = int(rng.choice([1, 5, 31, 32, 33, 64, 65, 130, 1000, 4096]))
+    W = int(rng.integers(1, 5))
+    shapes = [(s * int(rng.integers(1, 4)), s * int(rng.integers(1, 4))) for _ in range(int(rng.integers(1, 4)))]
+    shapes += [(s * int(rng.integers(1, 4)),) for _ in range(int(rng.integers(0, 2)))]
+    dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+    alpha = None if rng.random() < 0.5 else float(rng.choice([0.2, 0.5]))
+    agg, phi = int(rng.integers(0, 3)), int(rng.integers(0, 2))
+    wl = inputs.Workload("tc-random%d" % seed, shapes, chunk=s, topk=k, num_workers=W, grad_kind="tensor_scaled",
+                         grad_std=0.01, grad_dtype=dtype)
+    r = parity.Runner(wl, max_chunks=10**9, seed=seed, alpha=alpha, agg=agg, phi=phi)
+    for step in (1, 2):
+        r.set_basis(gauss=inputs.basis_gaussian(100 * seed + step, s).numpy())
+        r.step()
+    r.close()
+
+
 def test_basis_argument_errors_keep_the_previous_basis():
     s = 8
     wl = inputs.Workload("basis-err", [(2 * s, 2 * s)], chunk=s, topk=4, num_workers=1, grad_kind="normal", grad_std=0.01)
