@@ -94,9 +94,10 @@ def algorithmic_bytes(wl, gbytes: int):
     return core, payload
 
 
-def cpu_baseline(wl, target_s: float = 20.0):
-    """Time the oracle, as it stands, on a bounded sample: n chunks of 2-D tiles through W compress
-    passes and one decode.  Returns params/s on that sample."""
+def cpu_sample(wl, target_s: float):
+    """A bounded sample of the workload for the oracle: n chunks of 2-D tiles through W compress passes
+    and one decode, n sized by a short probe so that one pass takes about target_s seconds.  The inputs
+    are drawn once (the values do not change the work); returns (timed pass, n, cores)."""
     import numpy as np
 
     from oracle import demo_oracle as orc
@@ -105,10 +106,13 @@ def cpu_baseline(wl, target_s: float = 20.0):
     M = s * s
     rng = np.random.default_rng(0)
 
-    def run(n):
-        g = rng.standard_normal((W, n, M)) * 1e-3
-        m = rng.standard_normal((W, n, M)) * 1e-2
-        x = rng.standard_normal((n, M)) * 0.02
+    def draw(n):
+        return (rng.standard_normal((W, n, M)) * 1e-3, rng.standard_normal((W, n, M)) * 1e-2,
+                rng.standard_normal((n, M)) * 0.02)
+
+    def run(data):
+        g, m, x = data
+        n = x.shape[0]
         recs = np.zeros((W, n, min(k, M)), dtype=orc.RECORD_DTYPE)
         t0 = time.perf_counter()
         for w in range(W):
@@ -120,9 +124,18 @@ def cpu_baseline(wl, target_s: float = 20.0):
 
     cores = orc.max_threads()
     n0 = max(cores, 16)
-    t_probe = run(n0)
+    t_probe = run(draw(n0))
     n = int(min(max(n0, n0 * target_s / max(t_probe, 1e-6)), 1 << 16))
-    t = run(n)
+    data = draw(n)
+    return (lambda: run(data)), n, cores
+
+
+def cpu_baseline(wl, target_s: float = 20.0, sample=None):
+    """Time the oracle, as it stands, on a bounded sample.  Returns (record, parameters, seconds)."""
+    s, k, W = wl.chunk, wl.topk, wl.num_workers
+    M = s * s
+    run, n, cores = sample if sample is not None else cpu_sample(wl, target_s)
+    t = run()
     return {"value": n * M / t, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "%d chunks of %dx%d (k=%d) through W=%d compress passes + 1 decode, %.1f s" % (n, s, s, k, W, t)}, n * M, t
 
@@ -136,8 +149,9 @@ def run_reference(args, rank):
     times, units = [], 0
     base = None
     per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    sample = cpu_sample(wl, per_step)  # sized and drawn once: every step is one pass over the same sample
     for i in range(args.warmup + args.steps):
-        base, n_par, t = cpu_baseline(wl, target_s=per_step)
+        base, n_par, t = cpu_baseline(wl, sample=sample)
         if i >= args.warmup:
             times.append(t)
             units += n_par
