@@ -49,7 +49,9 @@ constexpr int OFF_BK_LO = OFF_BK_HI + 2 * BLK;
 constexpr int OFF_BM_HI = OFF_BK_LO + 2 * BLK;    // basis, MN-major operand (2 blocks)
 constexpr int OFF_BM_LO = OFF_BM_HI + 2 * BLK;
 constexpr int OFF_MISC = OFF_BM_LO + 2 * BLK;     // per chunk: hist[256], state[16]; then mbarriers, tensor-memory slot
-constexpr int MISC_PER_CHUNK = (256 + 16) * 4;
+constexpr int CAPT = 128;                        // candidate capacity of the fast top-k
+constexpr int HIST_WORDS = 2 * (CAPT + 4);       // radix histogram [256], or candidate keys [CAPT + 4] + indices [CAPT + 4]
+constexpr int MISC_PER_CHUNK = (HIST_WORDS + 80 + 128) * 4;  // + misc[80] + rowmask[128]
 constexpr int OFF_BARS = OFF_MISC + 2 * GROUPS * MISC_PER_CHUNK;
 constexpr int TC_SMEM_BYTES = OFF_BARS + 64 + 1024;  // + alignment slack
 
@@ -319,7 +321,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) compress_tc_kernel(DemoCompress
     const SlotBarrier<S> sb{1 + GROUPS + 2 * f.g + c};    // the 64 threads of one chunk
     float *X = reinterpret_cast<float *>(f.op + (c ? OFF_OP_LO : OFF_OP_HI));  // plain tile of chunk c (aliases the operands)
     unsigned *hist = reinterpret_cast<unsigned *>(f.sm + OFF_MISC + (2 * f.g + c) * MISC_PER_CHUNK);
-    unsigned *misc = hist + 256;
+    unsigned *misc = hist + HIST_WORDS;  // [80]: counts, select state, the 64 row maxima
+    unsigned *rowmask = misc + 80;     // [128]: per row, the kept coefficients as a 64-bit mask
     bool ok = true;
 
     const long long n_pairs = (a.n_chunks + 1) / 2;
@@ -371,76 +374,150 @@ __global__ void __launch_bounds__(TC_THREADS, 1) compress_tc_kernel(DemoCompress
         ok = tc_transform(f, pb, c, r, v, 0);
         if (!ok) break;
 
-        // ---- exact top-k of the chunk (radix select, ties to the lowest index), records in index order ---
+        // ---- exact top-k of the chunk, ties to the lowest index, records in index order ------------------
+        // Fast path (k_eff <= 64): the k_eff-th largest of the 64 per-row maxima bounds the k_eff-th largest
+        // coefficient from below; the coefficients at or above it (a few dozen) are listed in index order
+        // and ranked exactly.  Everything compares integer magnitude keys (NaN and Inf are ordered like any
+        // other bit pattern).  Too many candidates (tied chunks) or k_eff > 64: radix select over the tile.
+        // `keep` collects, per row, which coefficients were kept: the inverse below takes them from there.
         DemoRecord *rec = a.payload + cr.te.rec_begin + cr.lc * (long long)k_eff;
+        unsigned long long keep = 0ull;
         if (cr.valid) {
             write_own_row(X, r, v);
-            sb.sync();
-            unsigned thr, need_eq;
-            radix_select_tile<S, XS>(X, k_eff, hist, misc, &thr, &need_eq, r, sb);
-            unsigned gt = 0, eq = 0;
+            unsigned *cand_key = hist, *cand_idx = hist + CAPT + 4;  // the histogram area doubles as the candidate lists
+            bool use_radix = k_eff > S;
+            if (!use_radix) {
+                unsigned tkey = 0u;
 #pragma unroll
-            for (int j = 0; j < S; ++j) {
-                const unsigned key = mag_key(v[j]);
-                gt += key > thr;
-                eq += key == thr;
-            }
-            const unsigned packed = gt | (eq << 16);
-            const unsigned inc = warp_inclusive_scan(packed, lane);
-            sb.sync();  // the select's last reads of misc are done
-            if (lane == 31) misc[warp2] = inc;
-            sb.sync();
-            unsigned before = inc - packed;
-            if (warp2 == 1) before += misc[0];
-            unsigned gb = before & 0xffffu, eb = before >> 16;
-#pragma unroll
-            for (int j = 0; j < S; ++j) {
-                const unsigned key = mag_key(v[j]);
-                bool s = false;
-                unsigned pos = 0;
-                if (key > thr) {
-                    pos = gb + min(eb, need_eq);
-                    ++gb;
-                    s = true;
-                } else if (key == thr) {
-                    if (eb < need_eq) {
-                        pos = gb + eb;
-                        s = true;
-                    }
-                    ++eb;
+                for (int j = 0; j < S; ++j) tkey = max(tkey, mag_key(v[j]));
+                rowmask[2 * r] = 0u;
+                rowmask[2 * r + 1] = 0u;
+                misc[4 + r] = tkey;  // misc[4 .. 4 + 64): the maxima of the chunk's rows
+                sb.sync();
+                const unsigned okey = misc[4 + (r ^ 32)];
+                const unsigned lo_all = __reduce_min_sync(0xffffffffu, min(tkey, okey));
+                const unsigned hi_all = __reduce_max_sync(0xffffffffu, max(tkey, okey));
+                const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
+                unsigned lmin = lo_all & ~((2u << b0) - 1u);
+#pragma unroll 1
+                for (int bit = b0; bit >= 15; --bit) {
+                    const unsigned cand = lmin | (1u << bit);
+                    const unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand)) +
+                                         __popc(__ballot_sync(0xffffffffu, okey >= cand));
+                    lmin = (cnt >= (unsigned)k_eff) ? cand : lmin;
                 }
-                if (s) {
-                    DemoRecord rc;
-                    rc.idx = r * S + j;
-                    rc.val = v[j];
-                    rec[pos] = rc;
+                unsigned long long mask = 0ull;
+#pragma unroll
+                for (int j = 0; j < S; ++j) mask |= (unsigned long long)(mag_key(v[j]) >= lmin) << j;
+                const unsigned cnt = (unsigned)__popcll(mask);
+                const unsigned inc = warp_inclusive_scan(cnt, lane);
+                if (lane == 31) misc[warp2] = inc;
+                sb.sync();
+                const unsigned n0 = misc[0], n_all = n0 + misc[1];
+                use_radix = n_all > (unsigned)CAPT || n_all < (unsigned)k_eff;
+                if (!use_radix) {
+                    unsigned o = inc - cnt + (warp2 ? n0 : 0u);
+                    while (mask) {
+                        const int j = __ffsll((long long)mask) - 1;
+                        mask &= mask - 1ull;
+                        cand_key[o] = mag_key(X[r * XS + j]);
+                        cand_idx[o] = (unsigned)(r * S + j);
+                        ++o;
+                    }
+                    if (r < 4) cand_key[n_all + r] = 0u;  // pad for the vector loads
+                    sb.sync();
+                    // candidates r and r + 64 of the list (list order = index order)
+                    unsigned selbits = 0u;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const unsigned me = (unsigned)(r + 64 * e);
+                        if (me < n_all) {
+                            const unsigned key = cand_key[me];
+                            unsigned rank = 0;
+                            const uint4 *keys4 = reinterpret_cast<const uint4 *>(cand_key);
+                            for (unsigned c4 = 0; c4 < ((n_all + 3u) >> 2); ++c4) {
+                                const uint4 k4 = keys4[c4];
+                                const unsigned j0 = 4u * c4;
+                                rank += (k4.x > key) || (k4.x == key && j0 < me);
+                                rank += (k4.y > key) || (k4.y == key && j0 + 1u < me);
+                                rank += (k4.z > key) || (k4.z == key && j0 + 2u < me);
+                                rank += (k4.w > key) || (k4.w == key && j0 + 3u < me);
+                            }
+                            selbits |= (unsigned)(rank < (unsigned)k_eff) << (16 * e);
+                        }
+                    }
+                    // positions: all kept among list entries 0..63 first (thread order), then among 64..127
+                    const unsigned sinc = warp_inclusive_scan(selbits, lane);
+                    if (lane == 31) misc[2 + warp2] = sinc;
+                    sb.sync();
+                    unsigned before = sinc - selbits + (warp2 ? misc[2] : 0u);
+                    const unsigned tot = misc[2] + misc[3];
+                    const unsigned pos_e[2] = {before & 0xffffu, (tot & 0xffffu) + (before >> 16)};
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        if ((selbits >> (16 * e)) & 1u) {
+                            const unsigned idx = cand_idx[r + 64 * e];
+                            DemoRecord rc;
+                            rc.idx = (int)idx;
+                            rc.val = X[(idx >> 6) * XS + (idx & (S - 1))];
+                            rec[pos_e[e]] = rc;
+                            atomicOr(&rowmask[2 * (idx >> 6) + ((idx >> 5) & 1u)], 1u << (idx & 31u));
+                        }
+                    }
+                    sb.sync();
+                    keep = ((unsigned long long)rowmask[2 * r + 1] << 32) | rowmask[2 * r];
+                }
+            }
+            if (use_radix) {
+                sb.sync();  // the coefficient tile is complete; the candidate path (if it ran) is done with its lists
+                unsigned thr, need_eq;
+                radix_select_tile<S, XS>(X, k_eff, hist, misc, &thr, &need_eq, r, sb);
+                unsigned gt = 0, eq = 0;
+#pragma unroll
+                for (int j = 0; j < S; ++j) {
+                    const unsigned key = mag_key(v[j]);
+                    gt += key > thr;
+                    eq += key == thr;
+                }
+                const unsigned packed = gt | (eq << 16);
+                const unsigned inc = warp_inclusive_scan(packed, lane);
+                sb.sync();  // the select's last reads of misc are done
+                if (lane == 31) misc[warp2] = inc;
+                sb.sync();
+                unsigned before = inc - packed;
+                if (warp2 == 1) before += misc[0];
+                unsigned gb = before & 0xffffu, eb = before >> 16;
+#pragma unroll
+                for (int j = 0; j < S; ++j) {
+                    const unsigned key = mag_key(v[j]);
+                    bool s = false;
+                    unsigned pos = 0;
+                    if (key > thr) {
+                        pos = gb + min(eb, need_eq);
+                        ++gb;
+                        s = true;
+                    } else if (key == thr) {
+                        if (eb < need_eq) {
+                            pos = gb + eb;
+                            s = true;
+                        }
+                        ++eb;
+                    }
+                    if (s) {
+                        DemoRecord rc;
+                        rc.idx = r * S + j;
+                        rc.val = v[j];
+                        rec[pos] = rc;
+                        keep |= 1ull << j;
+                    }
                 }
             }
         }
-        pb.sync();  // records of both chunks are written (visible inside the CTA); the tiles are free
+        pb.sync();  // both chunks are done with the tiles (coefficient tile, lists): they become operand space
 
         // ---- kept coefficients as a dense tile: row u of Q_sp (zero except the kept entries) --------------
 #pragma unroll
-        for (int j = 0; j < S; ++j) v[j] = 0.f;
-        if (cr.valid) {
-            // the records of the chunk are sorted by index, i.e. grouped by row: find this row's by bisection
-            int lo = 0, hi = k_eff;
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if ((rec[mid].idx >> 6) < r)
-                    lo = mid + 1;
-                else
-                    hi = mid;
-            }
-            for (int i = lo; i < k_eff; ++i) {
-                const DemoRecord rc = rec[i];
-                if ((rc.idx >> 6) != r) break;
-                const int col = rc.idx & (S - 1);
-#pragma unroll
-                for (int j = 0; j < S; ++j)
-                    if (j == col) v[j] = rc.val;
-            }
-        }
+        for (int j = 0; j < S; ++j) v[j] = ((keep >> j) & 1ull) ? v[j] : 0.f;
         // ---- R = P^T Q_sp P; momentum subtraction  m <- B - alpha R  (Section 2.1) -----------------------
         ok = tc_transform(f, pb, c, r, v, 1);
         if (!ok) break;
