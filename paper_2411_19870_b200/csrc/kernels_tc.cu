@@ -331,6 +331,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) compress_tc_kernel(DemoCompress
         const int k_eff = cr.te.k_eff;
         const size_t n1 = (size_t)cr.te.n1;
         float *m_tile = a.m_ptrs[cr.te.tensor] + cr.tile_off;
+        {
+            // pull the next pair's tiles into L2 while this pair is worked on: 64 threads x 3 lines of 128 bytes
+            // cover the 64 x 256 bytes of m and the 64 x 128 (bf16) or 64 x 256 (fp32) bytes of g
+            const ChunkRef nx = locate(a.entries, a.n_entries, a.n_chunks, 2 * (p + (long long)gridDim.x * GROUPS) + c);
+            if (nx.valid) {
+                const char *nm = reinterpret_cast<const char *>(a.m_ptrs[nx.te.tensor] + nx.tile_off) +
+                                 (size_t)r * nx.te.n1 * sizeof(float);
+                const size_t gsz = a.grad_bf16 ? 2 : 4;
+                const char *ng = static_cast<const char *>(a.g_ptrs[nx.te.tensor]) + (nx.tile_off + (size_t)r * nx.te.n1) * gsz;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nm));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nm + 128));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(ng));
+                if (!a.grad_bf16) asm volatile("prefetch.global.L2 [%0];" ::"l"(ng + 128));
+            }
+        }
         float b[S], v[S];
         if (cr.valid) {
             // momentum update, tile-wise and coalesced:  B = beta * m + g  (Algorithm 1, worker side)
@@ -555,6 +570,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) decode_tc_kernel(DemoDecodeArgs
     for (long long p = (long long)blockIdx.x * GROUPS + f.g; p < n_pairs; p += (long long)gridDim.x * GROUPS) {
         const ChunkRef cr = locate(a.entries, a.n_entries, a.n_chunks, 2 * p + c);
         const int k_eff = cr.te.k_eff;
+        {
+            // pull the next pair's parameter tiles into L2 while this pair is worked on
+            const ChunkRef nx = locate(a.entries, a.n_entries, a.n_chunks, 2 * (p + (long long)gridDim.x * GROUPS) + c);
+            if (nx.valid) {
+                const char *nxp = reinterpret_cast<const char *>(a.x_ptrs[nx.te.tensor] + nx.tile_off) +
+                                  (size_t)r * nx.te.n1 * sizeof(float);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nxp));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(nxp + 128));
+            }
+        }
         float v[S];
         if (cr.valid) {
             float4 *row = reinterpret_cast<float4 *>(St + r * XS);
