@@ -166,6 +166,7 @@ class GradStream:
             self.row_factors = [torch.exp(torch.randn((shp[0], 1) if len(shp) == 2 else (shp[0],), generator=rg, device=device))
                                 for shp in wl.shapes]
         self.tie_gen = _gen(device, TIE_MASK_SEED + worker) if wl.grad_kind == "student_t_ties" else None
+        self.tie_fraction = 0.05  # share of chunks replaced by tie-makers (student_t_ties)
 
     def _draw(self, t: int, shp: Shape) -> torch.Tensor:
         wl = self.wl
@@ -193,7 +194,7 @@ class GradStream:
         else:
             c0, c1 = 1, shp[0] // s
             tiles = g.view(1, c1, 1, s)
-        pick = torch.rand((c0, c1), generator=self.tie_gen, device=self.device) < 0.05
+        pick = torch.rand((c0, c1), generator=self.tie_gen, device=self.device) < self.tie_fraction
         kind = torch.randint(0, 4, (c0, c1), generator=self.tie_gen, device=self.device)
         a = 1e-3
         sign = torch.where(torch.rand(tiles.shape, generator=self.tie_gen, device=self.device) < 0.5, -a, a)

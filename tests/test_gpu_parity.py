@@ -528,6 +528,23 @@ def test_randomized_tensor_core_cases(seed):
     r.close()
 
 
+@pytest.mark.parametrize("basis_kind", ["identity", "random"])
+def test_tensor_core_kernels_on_tie_maker_chunks(basis_kind):
+    """All-zero, constant, symmetric and +-a tiles (the stress configuration's tie-makers, here in 30 % of the
+    chunks) through the tensor-core kernels: under the identity basis the ties survive the transform, so the
+    candidate path overflows and the radix select with the index tie-break has to take over."""
+    s = 64
+    wl = inputs.Workload("tc-ties", [(4 * s, 4 * s), (2 * s, 3 * s)], chunk=s, topk=32, num_workers=3,
+                         grad_kind="student_t_ties", grad_std=1e-3)
+    kw = dict(basis=np.eye(s)) if basis_kind == "identity" else dict(gauss=inputs.basis_gaussian(3, s).numpy())
+    r = parity.Runner(wl, max_chunks=10**9, **kw)
+    for st in r.streams:
+        st.tie_fraction = 0.3
+    r.step()
+    r.step()
+    r.close()
+
+
 def test_basis_argument_errors_keep_the_previous_basis():
     s = 8
     wl = inputs.Workload("basis-err", [(2 * s, 2 * s)], chunk=s, topk=4, num_workers=1, grad_kind="normal", grad_std=0.01)
