@@ -11,6 +11,10 @@
  * there is no global state and no CPU fallback: without a CUDA device every compute entry point
  * fails with DEMO_ERR_CUDA.
  *
+ * Streams: when a context holds both 2-D and 1-D tensors, the small kernel of the 1-D tensors runs on a
+ * stream of the context beside the kernel of the 2-D tensors: it starts after everything already queued on
+ * cuda_stream and cuda_stream continues only when it has finished, so the caller sees plain stream order.
+ *
  * CUDA graphs: demo_compress and demo_decode_apply copy their pointer arrays to device tables only
  * when a pointer differs from the previous call with the same worker index.  After one ordinary call
  * with the same buffers they enqueue kernel launches only and may be captured into a CUDA graph on

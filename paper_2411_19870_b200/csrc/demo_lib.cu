@@ -57,6 +57,11 @@ struct demo_ctx {
     CUtensorMap *d_tm_x = nullptr;                     // [T]
     std::vector<CUtensorMap> h_tm;                     // staging, [T]
 
+    // The small kernel of the 1-D tensors runs on a side stream beside the kernel of the 2-D tensors
+    // (fork / join by events; also legal inside a stream capture).  NULL: both on the caller's stream.
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+
     // demo_step_host: host->device gradient copies run on their own stream so that the copy of worker
     // w+1 overlaps the compress of worker w (created on first use)
     cudaStream_t copy_stream = nullptr;
@@ -142,6 +147,9 @@ void release(demo_ctx *c)
     for (cudaEvent_t e : c->ev_copied)
         if (e) cudaEventDestroy(e);
     if (c->ev_start) cudaEventDestroy(c->ev_start);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side_stream) cudaStreamDestroy(c->side_stream);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     delete c;
 }
@@ -303,6 +311,16 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
     }
     ok = ok && cudaMemcpy(c->d_C, C.data(), C.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+    if (ok && c->n2d && c->n1d) {
+        // optional: without them the two kernels of a call simply run one after the other
+        if (cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            if (c->side_stream) cudaStreamDestroy(c->side_stream);
+            c->side_stream = nullptr;
+        }
+    }
     if (ok && c->n2d)
         ok = cudaMemcpy(c->d_entries2d, e2d.data(), e2d.size() * sizeof(DemoTensorEntry), cudaMemcpyHostToDevice) ==
              cudaSuccess;
@@ -328,6 +346,26 @@ demo_status demo_payload_layout(const demo_ctx *ctx, int32_t tensor, int64_t *fi
     if (n_chunks) *n_chunks = ctx->n_chunks[tensor];
     if (k_eff) *k_eff = ctx->k_eff[tensor];
     return DEMO_OK;
+}
+
+// The 1-D kernel of a call goes to the side stream: it is ordered after everything already queued on the
+// caller's stream (fork) and the caller's stream continues only when it is done (join).
+static cudaStream_t fork_side(demo_ctx *ctx, cudaStream_t stream)
+{
+    if (!ctx->side_stream || !ctx->n2d || !ctx->n1d) return stream;
+    if (cudaEventRecord(ctx->ev_fork, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return stream;
+    }
+    return ctx->side_stream;
+}
+static cudaError_t join_side(demo_ctx *ctx, cudaStream_t side, cudaStream_t stream)
+{
+    if (side == stream) return cudaSuccess;
+    cudaError_t err = cudaEventRecord(ctx->ev_join, side);
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(stream, ctx->ev_join, 0);
+    return err;
 }
 
 // The fast kernels hard-code the DCT factorisation; any other basis takes the dense-transform kernels.
@@ -392,7 +430,16 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
     a.tmap_m = ctx->encode ? ctx->d_tm_m + row : nullptr;
     a.tmap_g = ctx->encode ? ctx->d_tm_g + row : nullptr;
     const int s = ctx->cfg.chunk;
-    if (ctx->n2d) {
+    cudaStream_t side = stream;
+    if (ctx->n1d) {
+        side = fork_side(ctx, stream);
+        a.entries = ctx->d_entries1d;
+        a.n_entries = ctx->n1d;
+        a.n_chunks = ctx->chunks1d;
+        err = demo_launch_compress_generic(s, 0, a, ctx->sm_count, side);
+        ctx->launches += 1;
+    }
+    if (err == cudaSuccess && ctx->n2d) {
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
@@ -404,12 +451,9 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
             err = demo_launch_compress_generic(s, 1, a, ctx->sm_count, stream);
         ctx->launches += 1;
     }
-    if (err == cudaSuccess && ctx->n1d) {
-        a.entries = ctx->d_entries1d;
-        a.n_entries = ctx->n1d;
-        a.n_chunks = ctx->chunks1d;
-        err = demo_launch_compress_generic(s, 0, a, ctx->sm_count, stream);
-        ctx->launches += 1;
+    {
+        const cudaError_t jerr = join_side(ctx, side, stream);  // always, so that a fork never stays open
+        if (err == cudaSuccess) err = jerr;
     }
     if (err != cudaSuccess) {
         cudaGetLastError();
@@ -461,7 +505,16 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     a.phi = ctx->phi;
     a.agg_scale = (ctx->aggregation == DEMO_AGG_MEAN) ? 1.0f / (float)W : 1.0f;
     const int s = ctx->cfg.chunk;
-    if (ctx->n2d) {
+    cudaStream_t side = stream;
+    if (ctx->n1d) {
+        side = fork_side(ctx, stream);
+        a.entries = ctx->d_entries1d;
+        a.n_entries = ctx->n1d;
+        a.n_chunks = ctx->chunks1d;
+        err = demo_launch_decode_generic(s, 0, a, ctx->sm_count, side);
+        ctx->launches += 1;
+    }
+    if (err == cudaSuccess && ctx->n2d) {
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
@@ -473,12 +526,9 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
             err = demo_launch_decode_generic(s, 1, a, ctx->sm_count, stream);
         ctx->launches += 1;
     }
-    if (err == cudaSuccess && ctx->n1d) {
-        a.entries = ctx->d_entries1d;
-        a.n_entries = ctx->n1d;
-        a.n_chunks = ctx->chunks1d;
-        err = demo_launch_decode_generic(s, 0, a, ctx->sm_count, stream);
-        ctx->launches += 1;
+    {
+        const cudaError_t jerr = join_side(ctx, side, stream);
+        if (err == cudaSuccess) err = jerr;
     }
     if (err != cudaSuccess) {
         cudaGetLastError();
