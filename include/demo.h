@@ -94,6 +94,42 @@ typedef enum { DEMO_PATH_AUTO = 0, DEMO_PATH_GENERIC = 1 } demo_path;
 demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_desc *tensors,
                       int32_t n_tensors, int32_t cuda_device);
 
+/*
+ * Tensors of any order with rectangular chunks -- the general statement of the method in the paper's
+ * appendix ("Multilinear Transforms and Chunk-wise Tensor Blocking"): a tensor of shape
+ * n_0 x ... x n_{d-1} with n_a = c_a * s_a is cut by the blocking operator into c_0 * ... * c_{d-1}
+ * chunks of shape s_0 x ... x s_{d-1}; the chunk transform is the multilinear product
+ * T(B; C_0, ..., C_{d-1}) with the orthonormal DCT-II of dimension s_a on axis a (inverse: the
+ * transposes).  The paper's worked example, a 128 x 512 matrix in 16 x 32 blocks, is
+ * {ndim 2, shape {128, 512}, chunk {16, 32}}.
+ *
+ * A descriptor is a contiguous row-major tensor of order ndim (1 .. DEMO_ND_MAX_DIMS) with its own chunk
+ * shape: 1 <= chunk[a] <= DEMO_ND_MAX_EXTENT, shape[a] a multiple of chunk[a] (the paper assumes this
+ * and gives no rule for remainders), M = product of chunk[] <= DEMO_ND_MAX_CHUNK_ELEMS.
+ *
+ * demo_init_nd builds a context like demo_init (cfg->chunk is ignored; 1 <= cfg->topk <=
+ * DEMO_ND_MAX_CHUNK_ELEMS, k_eff = min(k, M) per tensor).  Every other entry point takes the context
+ * unchanged, with these differences: a record's idx is the row-major position inside the chunk
+ * (((j_0 * s_1 + j_1) * s_2 + j_2) ...), chunks are ordered row-major over the chunk grid
+ * (k_0, ..., k_{d-1}); all tensors run on one family of kernels that apply the transform axis by axis as
+ * dense contractions on the CUDA cores (no fast-DCT, tensor-core or side-stream path; demo_set_path has
+ * no effect); demo_set_basis, demo_set_basis_gaussian and demo_get_basis return UNSUPPORTED (one basis
+ * per chunk extent: only the DCT is built).  A descriptor with ndim <= 2 and equal chunk extents gives
+ * the same payload bytes as demo_init with that chunk size.
+ * Errors: INVALID_ARG, SHAPE (ndim, chunk[a] < 1, shape[a] not a multiple of chunk[a]), K,
+ * UNSUPPORTED (chunk extent or chunk too large, dtype, too many tensors), ALLOC, CUDA.
+ */
+#define DEMO_ND_MAX_DIMS 4
+#define DEMO_ND_MAX_EXTENT 128
+#define DEMO_ND_MAX_CHUNK_ELEMS 16384
+typedef struct {
+    int32_t ndim;
+    int64_t shape[DEMO_ND_MAX_DIMS];
+    int32_t chunk[DEMO_ND_MAX_DIMS];
+} demo_nd_tensor_desc;
+demo_status demo_init_nd(demo_ctx **out, const demo_config *cfg, const demo_nd_tensor_desc *tensors,
+                         int32_t n_tensors, int32_t cuda_device);
+
 /* Bytes of one worker's payload: sum over tensors of n_chunks * k_eff * 8.  0 if ctx is NULL. */
 size_t demo_payload_bytes(const demo_ctx *ctx);
 

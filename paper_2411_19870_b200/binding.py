@@ -23,7 +23,7 @@ DEMO_PHI_SIGN, DEMO_PHI_IDENTITY = 0, 1
 RECORD_BYTES = 8
 
 EXPORTS = [
-    "demo_init", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
+    "demo_init", "demo_init_nd", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
     "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_set_basis",
     "demo_set_basis_gaussian", "demo_get_basis", "demo_selftest_bounded_wait", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
@@ -32,6 +32,13 @@ EXPORTS = [
 
 class DemoTensorDesc(ctypes.Structure):
     _fields_ = [("ndim", ctypes.c_int32), ("shape", ctypes.c_int64 * 2)]
+
+
+ND_MAX_DIMS = 4
+
+
+class DemoNdTensorDesc(ctypes.Structure):
+    _fields_ = [("ndim", ctypes.c_int32), ("shape", ctypes.c_int64 * ND_MAX_DIMS), ("chunk", ctypes.c_int32 * ND_MAX_DIMS)]
 
 
 class DemoConfig(ctypes.Structure):
@@ -65,6 +72,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     pvp = ctypes.POINTER(ctypes.c_void_p)
     lib.demo_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(DemoConfig), ctypes.POINTER(DemoTensorDesc), i32, i32]
     lib.demo_init.restype = i32
+    lib.demo_init_nd.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(DemoConfig), ctypes.POINTER(DemoNdTensorDesc), i32, i32]
+    lib.demo_init_nd.restype = i32
     lib.demo_payload_bytes.argtypes = [vp]
     lib.demo_payload_bytes.restype = ctypes.c_size_t
     lib.demo_payload_layout.argtypes = [vp, i32, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i32)]
@@ -155,25 +164,40 @@ def decode_apply_static(shapes, payloads, params, *, chunk: int, topk: int, lr: 
 
 
 class DemoTransform:
-    """One ``demo_ctx``.  ``shapes`` is a list of 1-D / 2-D shapes in payload order."""
+    """One ``demo_ctx``.  ``shapes`` is a list of 1-D / 2-D shapes in payload order (``demo_init``).
+    With ``chunk_shapes`` (one tuple per tensor, same order as its shape) the context comes from
+    ``demo_init_nd``: tensors of any order up to 4 with rectangular chunks; ``chunk`` is then unused."""
 
-    def __init__(self, shapes, *, chunk: int, topk: int, beta: float, lr: float, weight_decay: float,
-                 num_workers: int, grad_dtype: int = DEMO_BF16, device: int = 0):
+    def __init__(self, shapes, *, chunk: int = 0, topk: int, beta: float, lr: float, weight_decay: float,
+                 num_workers: int, grad_dtype: int = DEMO_BF16, device: int = 0, chunk_shapes=None):
         self.lib = load_library()
         self.shapes = [tuple(int(d) for d in s) for s in shapes]
-        descs = (DemoTensorDesc * len(self.shapes))()
-        for d, s in zip(descs, self.shapes):
-            d.ndim = len(s)
-            for a in range(min(len(s), 2)):
-                d.shape[a] = s[a]
+        self.chunk_shapes = None if chunk_shapes is None else [tuple(int(d) for d in s) for s in chunk_shapes]
         self.cfg = DemoConfig(beta, chunk, topk, lr, weight_decay, num_workers, grad_dtype)
         self.num_workers = num_workers
         self.device = device
         self._ctx = ctypes.c_void_p()
-        st = self.lib.demo_init(ctypes.byref(self._ctx), ctypes.byref(self.cfg), descs, len(self.shapes), device)
+        if self.chunk_shapes is None:
+            descs = (DemoTensorDesc * len(self.shapes))()
+            for d, s in zip(descs, self.shapes):
+                d.ndim = len(s)
+                for a in range(min(len(s), 2)):
+                    d.shape[a] = s[a]
+            st = self.lib.demo_init(ctypes.byref(self._ctx), ctypes.byref(self.cfg), descs, len(self.shapes), device)
+        else:
+            if len(self.chunk_shapes) != len(self.shapes) or any(
+                    len(c) != len(s) for c, s in zip(self.chunk_shapes, self.shapes)):
+                raise ValueError("chunk_shapes: one chunk shape per tensor, of the tensor's order")
+            nd = (DemoNdTensorDesc * len(self.shapes))()
+            for d, s, c in zip(nd, self.shapes, self.chunk_shapes):
+                d.ndim = len(s)
+                for a in range(min(len(s), ND_MAX_DIMS)):
+                    d.shape[a] = s[a]
+                    d.chunk[a] = c[a]
+            st = self.lib.demo_init_nd(ctypes.byref(self._ctx), ctypes.byref(self.cfg), nd, len(self.shapes), device)
         if st != 0:
             self._ctx = ctypes.c_void_p()
-            raise DemoError(st, "demo_init")
+            raise DemoError(st, "demo_init" if self.chunk_shapes is None else "demo_init_nd")
         self._ptr_cache = {}
         self._payload_bytes = int(self.lib.demo_payload_bytes(self._ctx))
         self._payload_ok = set()   # (data pointer, size) of payload buffers already checked

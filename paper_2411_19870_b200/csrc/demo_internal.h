@@ -86,6 +86,54 @@ cudaError_t demo_launch_wait_selftest(int *status, long long limit_cycles, cudaS
 // orthonormal rows to `basis` (device, fp32) and 1 to *flag when a row has no component left.
 cudaError_t demo_launch_gram_schmidt(const float *gauss, float *basis, int *flag, int s, cudaStream_t stream);
 
+// ---- tensors of any order with rectangular chunks (appendix of the paper: blocking operator and
+// multilinear product; kernels_nd.cu) ---------------------------------------------------------------
+constexpr int DEMO_ND_DIMS = 4;  // lower orders are padded on the left with axes of extent 1
+
+struct DemoNdEntry {
+    long long chunk_begin;           // id of this tensor's first chunk inside the work list
+    long long rec_begin;             // index of this tensor's first record inside a payload
+    long long stride[DEMO_ND_DIMS];  // element stride of each axis of the (contiguous) tensor
+    int tensor;                      // position in the caller's pointer arrays
+    int k_eff;                       // min(k, M)
+    int M;                           // elements per chunk
+    int s[DEMO_ND_DIMS];             // chunk shape
+    int c[DEMO_ND_DIMS];             // chunk grid
+    int basis[DEMO_ND_DIMS];         // offset (floats) of the s[a] x s[a] DCT matrix inside the table
+};
+
+struct DemoNdCompressArgs {
+    const DemoNdEntry *entries;  // device
+    int n_entries;
+    long long n_chunks;
+    const void *const *g_ptrs;
+    float *const *m_ptrs;
+    DemoRecord *payload;
+    const float *tables;  // device, the DCT matrices of every chunk extent in use, C[u*s + n]
+    float beta, alpha;
+    int grad_bf16;
+    int max_M;  // largest chunk of the list (sizes the shared-memory buffers)
+    int *status;
+};
+
+struct DemoNdDecodeArgs {
+    const DemoNdEntry *entries;
+    int n_entries;
+    long long n_chunks;
+    const DemoRecord *const *payloads;
+    int W;
+    float *const *x_ptrs;
+    const float *tables;
+    float lr, wd;
+    int max_M;
+    int *status;
+    int agg, phi;
+    float agg_scale;
+};
+
+cudaError_t demo_launch_compress_nd(const DemoNdCompressArgs &a, int sm_count, cudaStream_t stream);
+cudaError_t demo_launch_decode_nd(const DemoNdDecodeArgs &a, int sm_count, cudaStream_t stream);
+
 // Locate the tensor that owns chunk id c: the last entry with chunk_begin <= c.
 __device__ __forceinline__ int demo_find_entry(const DemoTensorEntry *entries, int n, long long c)
 {

@@ -33,6 +33,14 @@ struct demo_ctx {
     float *d_C = nullptr;
     int *d_status = nullptr;
 
+    // contexts made by demo_init_nd: one work list of rectangular chunks of any order, the DCT matrices
+    // of every chunk extent in one table; the square-chunk lists above stay empty
+    bool nd = false;
+    int n_nd = 0, max_M = 0;
+    long long chunks_nd = 0;
+    DemoNdEntry *d_entries_nd = nullptr;
+    float *d_tables = nullptr;
+
     // caller-supplied orthonormal basis (rows = basis vectors); while `custom_basis` is set every
     // tensor goes through the dense-transform kernels, which read the basis from memory
     float *d_P = nullptr, *d_P_stage = nullptr;  // [s*s], [2*s*s]
@@ -68,6 +76,8 @@ struct demo_ctx {
     cudaEvent_t ev_start = nullptr;
     std::vector<cudaEvent_t> ev_copied;  // [W]
 };
+
+static_assert(DEMO_ND_DIMS == DEMO_ND_MAX_DIMS, "public and internal axis limits disagree");
 
 namespace {
 
@@ -133,6 +143,8 @@ void release(demo_ctx *c)
     cudaFree(c->d_entries2d);
     cudaFree(c->d_entries1d);
     cudaFree(c->d_C);
+    cudaFree(c->d_entries_nd);
+    cudaFree(c->d_tables);
     cudaFree(c->d_P);
     cudaFree(c->d_P_stage);
     cudaFree(c->d_basis_flag);
@@ -336,6 +348,150 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
     return DEMO_OK;
 }
 
+demo_status demo_init_nd(demo_ctx **out, const demo_config *cfg, const demo_nd_tensor_desc *tensors, int32_t n_tensors,
+                         int32_t cuda_device)
+{
+    if (out) *out = nullptr;
+    if (!out || !cfg || !tensors || n_tensors < 1 || cuda_device < 0) return DEMO_ERR_INVALID_ARG;
+    if (cfg->num_workers < 1 || cfg->num_workers > 4096) return DEMO_ERR_INVALID_ARG;
+    if (!std::isfinite(cfg->beta) || !std::isfinite(cfg->lr) || !std::isfinite(cfg->weight_decay))
+        return DEMO_ERR_INVALID_ARG;
+    if (cfg->grad_dtype != DEMO_F32 && cfg->grad_dtype != DEMO_BF16) return DEMO_ERR_UNSUPPORTED;
+    if (n_tensors > (1 << 20)) return DEMO_ERR_UNSUPPORTED;
+    if (cfg->topk < 1 || cfg->topk > DEMO_ND_MAX_CHUNK_ELEMS) return DEMO_ERR_K;
+    for (int t = 0; t < n_tensors; ++t) {
+        const demo_nd_tensor_desc &d = tensors[t];
+        if (d.ndim < 1 || d.ndim > DEMO_ND_MAX_DIMS) return DEMO_ERR_SHAPE;
+        long long M = 1, n_ch = 1, n_el = 1;
+        for (int a = 0; a < d.ndim; ++a) {
+            if (d.chunk[a] < 1) return DEMO_ERR_SHAPE;
+            if (d.chunk[a] > DEMO_ND_MAX_EXTENT) return DEMO_ERR_UNSUPPORTED;
+            if (d.shape[a] < d.chunk[a] || d.shape[a] % d.chunk[a] != 0 || d.shape[a] > (1LL << 31) - 1)
+                return DEMO_ERR_SHAPE;
+            M *= d.chunk[a];
+            n_ch *= d.shape[a] / d.chunk[a];
+            n_el *= d.shape[a];
+            if (M > DEMO_ND_MAX_CHUNK_ELEMS || n_ch > (1LL << 31) - 1 || n_el > (1LL << 40)) return DEMO_ERR_UNSUPPORTED;
+        }
+    }
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cuda_device >= n_dev) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    DeviceGuard guard(cuda_device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+
+    demo_ctx *c = new (std::nothrow) demo_ctx();
+    if (!c) return DEMO_ERR_ALLOC;
+    c->cfg = *cfg;
+    c->cfg.chunk = 0;  // chunk shapes are per tensor
+    c->device = cuda_device;
+    c->n_tensors = n_tensors;
+    c->nd = true;
+    if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cuda_device) != cudaSuccess) {
+        release(c);
+        return DEMO_ERR_CUDA;
+    }
+
+    // planner: the work list (axes padded on the left to DEMO_ND_DIMS), payload offsets, and one
+    // orthonormal DCT-II matrix per distinct chunk extent
+    std::vector<DemoNdEntry> entries;
+    std::vector<float> tables;
+    try {
+        int table_of[DEMO_ND_MAX_EXTENT + 1];
+        for (int &v : table_of) v = -1;
+        c->first_record.resize(n_tensors);
+        c->n_chunks.resize(n_tensors);
+        c->n_elems.resize(n_tensors);
+        c->k_eff.resize(n_tensors);
+        long long rec = 0;
+        for (int t = 0; t < n_tensors; ++t) {
+            const demo_nd_tensor_desc &d = tensors[t];
+            DemoNdEntry e;
+            const int pad = DEMO_ND_DIMS - d.ndim;
+            long long stride = 1, M = 1, n_ch = 1;
+            for (int a = DEMO_ND_DIMS - 1; a >= 0; --a) {
+                const bool real = a >= pad;
+                const int s = real ? d.chunk[a - pad] : 1;
+                const long long n = real ? d.shape[a - pad] : 1;
+                e.s[a] = s;
+                e.c[a] = (int)(n / s);
+                e.stride[a] = stride;
+                stride *= n;
+                M *= s;
+                n_ch *= n / s;
+                e.basis[a] = 0;
+                if (s > 1) {
+                    if (table_of[s] < 0) {
+                        table_of[s] = (int)tables.size();
+                        const double pi = 3.141592653589793238462643383279502884;
+                        for (int u = 0; u < s; ++u)
+                            for (int n2 = 0; n2 < s; ++n2) {
+                                const double au = (u == 0) ? std::sqrt(1.0 / s) : std::sqrt(2.0 / s);
+                                tables.push_back((float)(au * std::cos(pi * (2.0 * n2 + 1.0) * u / (2.0 * s))));
+                            }
+                    }
+                    e.basis[a] = table_of[s];
+                }
+            }
+            e.tensor = t;
+            e.M = (int)M;
+            e.k_eff = (int)(cfg->topk < M ? cfg->topk : M);
+            e.rec_begin = rec;
+            e.chunk_begin = c->chunks_nd;
+            c->chunks_nd += n_ch;
+            if (e.M > c->max_M) c->max_M = e.M;
+            entries.push_back(e);
+            c->first_record[t] = rec;
+            c->n_chunks[t] = n_ch;
+            c->n_elems[t] = stride;
+            c->k_eff[t] = e.k_eff;
+            rec += n_ch * e.k_eff;
+        }
+        c->total_records = rec;
+        if (tables.empty()) tables.push_back(1.0f);  // every extent is 1: no matrix is ever read
+        const size_t W = (size_t)cfg->num_workers, T = (size_t)n_tensors;
+        c->h_g.assign(W * T, nullptr);
+        c->h_m.assign(W * T, nullptr);
+        c->h_x.assign(T, nullptr);
+        c->h_p.assign(W, nullptr);
+        c->g_valid.assign(W, 0);
+        c->m_valid.assign(W, 0);
+    } catch (const std::bad_alloc &) {
+        release(c);
+        return DEMO_ERR_ALLOC;
+    }
+    c->n_nd = n_tensors;
+
+    const size_t W = (size_t)cfg->num_workers, T = (size_t)n_tensors;
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->d_tables, tables.size() * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_entries_nd, entries.size() * sizeof(DemoNdEntry)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_g, W * T * sizeof(void *)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_m, W * T * sizeof(void *)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_x, T * sizeof(void *)) == cudaSuccess;
+    ok = ok && cudaMalloc((void **)&c->d_p, W * sizeof(void *)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        release(c);
+        return DEMO_ERR_ALLOC;
+    }
+    ok = ok && cudaMemcpy(c->d_tables, tables.data(), tables.size() * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(c->d_entries_nd, entries.data(), entries.size() * sizeof(DemoNdEntry),
+                          cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        release(c);
+        return DEMO_ERR_CUDA;
+    }
+    *out = c;
+    return DEMO_OK;
+}
+
 size_t demo_payload_bytes(const demo_ctx *ctx) { return ctx ? (size_t)ctx->total_records * sizeof(DemoRecord) : 0; }
 
 demo_status demo_payload_layout(const demo_ctx *ctx, int32_t tensor, int64_t *first_record, int64_t *n_chunks,
@@ -418,6 +574,28 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
         return DEMO_ERR_CUDA;
     }
 
+    if (ctx->nd) {
+        DemoNdCompressArgs n;
+        n.entries = ctx->d_entries_nd;
+        n.n_entries = ctx->n_nd;
+        n.n_chunks = ctx->chunks_nd;
+        n.g_ptrs = ctx->d_g + row;
+        n.m_ptrs = ctx->d_m + row;
+        n.payload = static_cast<DemoRecord *>(payload_out);
+        n.tables = ctx->d_tables;
+        n.beta = ctx->cfg.beta;
+        n.alpha = ctx->alpha;
+        n.grad_bf16 = ctx->cfg.grad_dtype == DEMO_BF16;
+        n.max_M = ctx->max_M;
+        n.status = ctx->d_status;
+        if (demo_launch_compress_nd(n, ctx->sm_count, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return DEMO_ERR_CUDA;
+        }
+        ctx->launches += 1;
+        return DEMO_OK;
+    }
+
     DemoCompressArgs a;
     a.g_ptrs = ctx->d_g + row;
     a.m_ptrs = ctx->d_m + row;
@@ -490,6 +668,30 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     if (err != cudaSuccess) {
         cudaGetLastError();
         return DEMO_ERR_CUDA;
+    }
+
+    if (ctx->nd) {
+        DemoNdDecodeArgs n;
+        n.entries = ctx->d_entries_nd;
+        n.n_entries = ctx->n_nd;
+        n.n_chunks = ctx->chunks_nd;
+        n.payloads = ctx->d_p;
+        n.W = W;
+        n.x_ptrs = ctx->d_x;
+        n.tables = ctx->d_tables;
+        n.lr = ctx->cfg.lr;
+        n.wd = ctx->cfg.weight_decay;
+        n.max_M = ctx->max_M;
+        n.status = ctx->d_status;
+        n.agg = ctx->aggregation;
+        n.phi = ctx->phi;
+        n.agg_scale = (ctx->aggregation == DEMO_AGG_MEAN) ? 1.0f / (float)W : 1.0f;
+        if (demo_launch_decode_nd(n, ctx->sm_count, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return DEMO_ERR_CUDA;
+        }
+        ctx->launches += 1;
+        return DEMO_OK;
     }
 
     DemoDecodeArgs a;
@@ -645,6 +847,7 @@ demo_status demo_selftest_bounded_wait(demo_ctx *ctx, int64_t limit_cycles, void
 demo_status demo_set_basis(demo_ctx *ctx, const float *basis_host, void *cuda_stream)
 {
     if (!ctx) return DEMO_ERR_INVALID_ARG;
+    if (ctx->nd) return DEMO_ERR_UNSUPPORTED;  // one basis per chunk extent: only the DCT is built
     if (!basis_host) {
         ctx->custom_basis = false;
         return DEMO_OK;
@@ -671,6 +874,7 @@ demo_status demo_set_basis(demo_ctx *ctx, const float *basis_host, void *cuda_st
 demo_status demo_set_basis_gaussian(demo_ctx *ctx, const float *gauss_host, void *cuda_stream)
 {
     if (!ctx || !gauss_host) return DEMO_ERR_INVALID_ARG;
+    if (ctx->nd) return DEMO_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DEMO_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -699,6 +903,7 @@ demo_status demo_set_basis_gaussian(demo_ctx *ctx, const float *gauss_host, void
 demo_status demo_get_basis(demo_ctx *ctx, float *basis_host_out, void *cuda_stream)
 {
     if (!ctx || !basis_host_out) return DEMO_ERR_INVALID_ARG;
+    if (ctx->nd) return DEMO_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DEMO_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

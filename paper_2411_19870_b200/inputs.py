@@ -212,6 +212,11 @@ class GradStream:
         return [self._draw(t, shp).to(self.wl.grad_dtype) for t, shp in enumerate(self.wl.shapes)]
 
 
+def random_tensor(shape: Shape, seed: int, std: float, dtype: torch.dtype, device) -> torch.Tensor:
+    """N(0, std^2) tensor of any shape from its own seed (tensors of order > 2, rectangular chunks)."""
+    return (torch.randn(tuple(shape), generator=_gen(device, seed), device=device, dtype=torch.float32) * std).to(dtype)
+
+
 def basis_gaussian(step: int, s: int) -> torch.Tensor:
     """s x s matrix of N(0,1) draws for the random orthonormal basis of one step; the seed is the step
     number, so every worker draws the same matrix (Section 4.2)."""

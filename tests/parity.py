@@ -16,6 +16,7 @@ import numpy as np
 import torch
 
 from oracle import demo_oracle as orc
+from oracle import demo_oracle_nd as ond
 
 RTOL = 1e-5
 ATOL = 1e-7
@@ -67,12 +68,22 @@ class Report(dict):
 
 
 def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, report: Report, what="", alpha=1.0,
-                          basis=None):
-    """All arguments are per-chunk arrays of the same n chunks (float64 / records)."""
-    M = rows * s
+                          basis=None, chunk_shape=None):
+    """All arguments are per-chunk arrays of the same n chunks (float64 / records).  With `chunk_shape`
+    (rectangular chunks of any order; s and rows unused) the reference is the N-D oracle."""
+    if chunk_shape is not None:
+        M = int(np.prod(chunk_shape))
+
+        def oracle(gg, mm, forced_idx=None):
+            return ond.compress_chunks(gg, mm, chunk_shape, k, beta, forced_idx=forced_idx, alpha=alpha)
+    else:
+        M = rows * s
+
+        def oracle(gg, mm, forced_idx=None):
+            return orc.compress_chunks(gg, mm, s, rows, k, beta, forced_idx=forced_idx, alpha=alpha, basis=basis)
     k_eff = min(k, M)
     n = g.shape[0]
-    ref = orc.compress_chunks(g, m_before, s, rows, k, beta, alpha=alpha, basis=basis)
+    ref = oracle(g, m_before)
     Q = ref["Q"]
     qinf = np.max(np.abs(Q), axis=1)
     floor = FLOOR_REL * qinf
@@ -122,8 +133,7 @@ def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, repor
     # residual momentum: oracle continued from the GPU's index set where the sets differ
     m_ref = ref["m_new"]
     if len(diff):
-        forced = orc.compress_chunks(g[diff], m_before[diff], s, rows, k, beta, forced_idx=idx_gpu[diff].astype(np.int32), alpha=alpha,
-                                     basis=basis)
+        forced = oracle(g[diff], m_before[diff], forced_idx=idx_gpu[diff].astype(np.int32))
         m_ref = m_ref.copy()
         m_ref[diff] = forced["m_new"]
     # the abs tolerance is scaled by the chunk's pre-subtraction magnitude (the fp32 rounding of
@@ -138,9 +148,12 @@ def check_compress_chunks(g, m_before, m_after, rec_gpu, s, rows, k, beta, repor
 
 
 def check_decode_chunks(recs_gpu, x_before, x_after, s, rows, lr, wd, report: Report, what="", agg=0, phi=0,
-                         basis=None):
+                         basis=None, chunk_shape=None):
     """recs_gpu [W, n, k_eff] GPU-written records; x_* float64 [n, M]."""
-    ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd, agg=agg, phi=phi, basis=basis)
+    if chunk_shape is not None:
+        ref = ond.decode_chunks(recs_gpu, x_before, chunk_shape, lr, wd, agg=agg, phi=phi)
+    else:
+        ref = orc.decode_chunks(recs_gpu, x_before, s, rows, lr, wd, agg=agg, phi=phi, basis=basis)
     R = ref["R"]
     if phi == orc.PHI_IDENTITY:
         # no sign decision: the update is linear in R; the tolerance follows R's fp32 rounding
@@ -256,6 +269,77 @@ class Runner:
                                     self.wd, self.report, what="decode t%d" % t, agg=self.agg, phi=self.phi, basis=self.basis)
         st = self.tr.device_status()
         assert st == 0, "device status %d (%s)" % (st, self.demo.demo_status_string(st))
+
+    def close(self):
+        self.tr.close()
+
+
+class NdRunner:
+    """Tensors of any order with rectangular chunks (demo_init_nd) against the N-D oracle, every chunk of
+    every tensor, every step."""
+
+    def __init__(self, shapes, chunk_shapes, topk, num_workers=2, grad_dtype=torch.bfloat16, beta=0.999, lr=1e-3,
+                 weight_decay=0.1, grad_std=1e-3, seed=0, alpha=None, agg=0, phi=0, device="cuda"):
+        import paper_2411_19870_b200 as demo
+        from paper_2411_19870_b200 import inputs
+
+        self.demo, self.inputs = demo, inputs
+        self.shapes = [tuple(s) for s in shapes]
+        self.chunks = [tuple(c) for c in chunk_shapes]
+        self.k, self.W, self.gdtype, self.grad_std, self.seed = topk, num_workers, grad_dtype, grad_std, seed
+        self.device = torch.device(device)
+        gd = demo.DEMO_BF16 if grad_dtype == torch.bfloat16 else demo.DEMO_F32
+        self.tr = demo.DemoTransform(self.shapes, topk=topk, beta=beta, lr=lr, weight_decay=weight_decay,
+                                     num_workers=num_workers, grad_dtype=gd, device=self.device.index or 0,
+                                     chunk_shapes=self.chunks)
+        self.agg, self.phi = agg, phi
+        if agg or phi:
+            self.tr.set_decode_mode(agg, phi)
+        self.alpha = 1.0
+        if alpha is not None:
+            self.tr.set_alpha(alpha)
+            self.alpha = float(np.float32(alpha))
+        self.params = [inputs.random_tensor(s, inputs.PARAM_SEED + t, 0.02, torch.float32, self.device)
+                       for t, s in enumerate(self.shapes)]
+        self.mom = [[torch.zeros(s, dtype=torch.float32, device=self.device) for s in self.shapes]
+                    for _ in range(num_workers)]
+        self.payloads = [torch.zeros(self.tr.payload_bytes, dtype=torch.uint8, device=self.device)
+                         for _ in range(num_workers)]
+        self.layout = [self.tr.payload_layout(t) for t in range(len(self.shapes))]
+        self.report = Report()
+        self.beta, self.lr, self.wd = float(np.float32(beta)), float(np.float32(lr)), float(np.float32(weight_decay))
+        self.step_no = 0
+
+    def _tiles(self, t, tensor):
+        M = int(np.prod(self.chunks[t]))
+        return ond.blocks(tensor.to(torch.float64).cpu().numpy(), self.chunks[t]).reshape(-1, M)
+
+    def _records(self, w, t):
+        first, n_chunks, k_eff = self.layout[t]
+        return gather_records(self.payloads[w], first, k_eff, np.arange(n_chunks, dtype=np.int64))
+
+    def step(self):
+        T = len(self.shapes)
+        for w in range(self.W):
+            g = [self.inputs.random_tensor(s, self.seed + 1000 * self.step_no + 100 * w + t, self.grad_std, self.gdtype,
+                                           self.device) for t, s in enumerate(self.shapes)]
+            before = [self._tiles(t, self.mom[w][t]) for t in range(T)]
+            self.tr.compress(w, g, self.mom[w], self.payloads[w])
+            for t in range(T):
+                M = int(np.prod(self.chunks[t]))
+                assert self.layout[t][2] == min(self.k, M)
+                check_compress_chunks(self._tiles(t, g[t]), before[t], self._tiles(t, self.mom[w][t]), self._records(w, t),
+                                      0, 0, self.k, self.beta, self.report, what="nd compress w%d t%d" % (w, t),
+                                      alpha=self.alpha, chunk_shape=self.chunks[t])
+        xb = [self._tiles(t, self.params[t]) for t in range(T)]
+        self.tr.decode_apply(self.payloads, self.params)
+        for t in range(T):
+            recs = np.stack([self._records(w, t) for w in range(self.W)])
+            check_decode_chunks(recs, xb[t], self._tiles(t, self.params[t]), 0, 0, self.lr, self.wd, self.report,
+                                what="nd decode t%d" % t, agg=self.agg, phi=self.phi, chunk_shape=self.chunks[t])
+        st = self.tr.device_status()
+        assert st == 0, "device status %d (%s)" % (st, self.demo.demo_status_string(st))
+        self.step_no += 1
 
     def close(self):
         self.tr.close()
