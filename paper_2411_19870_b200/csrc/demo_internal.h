@@ -92,6 +92,7 @@ constexpr int DEMO_ND_DIMS = 4;  // lower orders are padded on the left with axe
 
 struct DemoNdEntry {
     long long chunk_begin;           // id of this tensor's first chunk inside the work list
+    long long chunk_end;             // chunk_begin + number of chunks of this tensor
     long long rec_begin;             // index of this tensor's first record inside a payload
     long long stride[DEMO_ND_DIMS];  // element stride of each axis of the (contiguous) tensor
     int tensor;                      // position in the caller's pointer arrays
@@ -99,7 +100,8 @@ struct DemoNdEntry {
     int M;                           // elements per chunk
     int s[DEMO_ND_DIMS];             // chunk shape
     int c[DEMO_ND_DIMS];             // chunk grid
-    int basis[DEMO_ND_DIMS];         // offset (floats) of the s[a] x s[a] DCT matrix inside the table
+    unsigned inv[DEMO_ND_DIMS];      // ceil(2^32 / s[a]) for s[a] > 1 (division by multiplication), else 0
+    int basis[DEMO_ND_DIMS];         // offset (floats, multiple of 4) of axis a's [C | C^T] inside the table
 };
 
 struct DemoNdCompressArgs {
@@ -109,7 +111,7 @@ struct DemoNdCompressArgs {
     const void *const *g_ptrs;
     float *const *m_ptrs;
     DemoRecord *payload;
-    const float *tables;  // device, the DCT matrices of every chunk extent in use, C[u*s + n]
+    const float *tables;  // device: per chunk extent s in use, C (s x s, C[u*s + n]) followed by C^T
     float beta, alpha;
     int grad_bf16;
     int max_M;  // largest chunk of the list (sizes the shared-memory buffers)

@@ -423,15 +423,22 @@ demo_status demo_init_nd(demo_ctx **out, const demo_config *cfg, const demo_nd_t
                 M *= s;
                 n_ch *= n / s;
                 e.basis[a] = 0;
+                e.inv[a] = s > 1 ? (unsigned)(((1ULL << 32) + (unsigned)s - 1) / (unsigned)s) : 0u;
                 if (s > 1) {
                     if (table_of[s] < 0) {
+                        // C then C^T, each s x s; every table starts on a 16-byte boundary
                         table_of[s] = (int)tables.size();
                         const double pi = 3.141592653589793238462643383279502884;
+                        std::vector<float> C((size_t)s * s);
                         for (int u = 0; u < s; ++u)
                             for (int n2 = 0; n2 < s; ++n2) {
                                 const double au = (u == 0) ? std::sqrt(1.0 / s) : std::sqrt(2.0 / s);
-                                tables.push_back((float)(au * std::cos(pi * (2.0 * n2 + 1.0) * u / (2.0 * s))));
+                                C[(size_t)u * s + n2] = (float)(au * std::cos(pi * (2.0 * n2 + 1.0) * u / (2.0 * s)));
                             }
+                        tables.insert(tables.end(), C.begin(), C.end());
+                        for (int n2 = 0; n2 < s; ++n2)
+                            for (int u = 0; u < s; ++u) tables.push_back(C[(size_t)u * s + n2]);
+                        while (tables.size() % 4) tables.push_back(0.f);
                     }
                     e.basis[a] = table_of[s];
                 }
@@ -442,7 +449,8 @@ demo_status demo_init_nd(demo_ctx **out, const demo_config *cfg, const demo_nd_t
             e.rec_begin = rec;
             e.chunk_begin = c->chunks_nd;
             c->chunks_nd += n_ch;
-            if (e.M > c->max_M) c->max_M = e.M;
+            e.chunk_end = c->chunks_nd;
+            if (((e.M + 3) & ~3) > c->max_M) c->max_M = (e.M + 3) & ~3;  // buffers stay 16-byte aligned
             entries.push_back(e);
             c->first_record[t] = rec;
             c->n_chunks[t] = n_ch;

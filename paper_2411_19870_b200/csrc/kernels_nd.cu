@@ -28,63 +28,128 @@ __device__ __forceinline__ int find_nd_entry(const DemoNdEntry *entries, int n, 
 }
 
 // Element offset of the chunk's first element: chunk id -> (k_0..k_3) row-major over the chunk grid,
-// offset = sum_a k_a s_a stride_a (blocking operator).
-__device__ __forceinline__ size_t chunk_base(const DemoNdEntry &e, long long lc)
+// offset = sum_a k_a s_a stride_a (blocking operator).  A tensor has fewer than 2^31 chunks.
+__device__ __forceinline__ size_t chunk_base(const DemoNdEntry &e, unsigned lc)
 {
     size_t base = 0;
 #pragma unroll
     for (int a = DEMO_ND_DIMS - 1; a >= 0; --a) {
-        const long long k = lc % e.c[a];
-        lc /= e.c[a];
+        const unsigned q = lc / (unsigned)e.c[a];
+        const unsigned k = lc - q * (unsigned)e.c[a];
+        lc = q;
         base += (size_t)k * (size_t)e.s[a] * (size_t)e.stride[a];
     }
     return base;
 }
 
-// Offset of element i (row-major inside the chunk) relative to the chunk's first element.
+// The entry and the base offset of the CTA's current chunk, looked up by one thread (the table is read
+// again only when the chunk belongs to another tensor than the previous one).
+struct ChunkSlot {
+    DemoNdEntry e;
+    size_t base;
+};
+
+__device__ __forceinline__ void locate_chunk(ChunkSlot *slot, const DemoNdEntry *entries, int n_entries, long long c)
+{
+    if (threadIdx.x == 0) {
+        if (c < slot->e.chunk_begin || c >= slot->e.chunk_end) slot->e = entries[find_nd_entry(entries, n_entries, c)];
+        slot->base = chunk_base(slot->e, (unsigned)(c - slot->e.chunk_begin));
+    }
+    __syncthreads();
+}
+
+// Offset of element i (row-major inside the chunk) relative to the chunk's first element.  The
+// divisions by the chunk extents are multiplications by inv[a] = ceil(2^32 / s_a), exact for
+// i < 2^14 and s_a <= 2^7.
 __device__ __forceinline__ size_t elem_offset(const DemoNdEntry &e, int i)
 {
     size_t off = 0;
+    unsigned r = (unsigned)i;
 #pragma unroll
     for (int a = DEMO_ND_DIMS - 1; a >= 0; --a) {
-        const int j = i % e.s[a];
-        i /= e.s[a];
-        off += (size_t)j * (size_t)e.stride[a];
+        if (e.s[a] > 1) {
+            const unsigned q = __umulhi(r, e.inv[a]);
+            off += (size_t)(r - q * (unsigned)e.s[a]) * (size_t)e.stride[a];
+            r = q;
+        }
     }
     return off;
 }
 
 // One axis of the multilinear product on a chunk in shared memory viewed as [outer][s][inner]:
-//   forward  dst[o][u][i] = sum_n P[u][n] src[o][n][i]
-//   inverse  dst[o][n][i] = sum_u P[u][n] src[o][u][i]
-// Each thread produces TU outputs that share their inputs.
-template <int TU>
+//   dst[o][j][i] = sum_n T[n][j] src[o][n][i]
+// with T = C^T for the forward transform (T[n][j] = C[j][n]) and T = C for the inverse; either way the
+// threads of a warp that differ in j read neighbouring table entries.  Each thread owns a TU x TV tile
+// of outputs: TU along j, TV along i (VI, vector loads) or along o.
+template <int TU, int TV, bool VI>
 __device__ __forceinline__ void axis_pass(float *__restrict__ dst, const float *__restrict__ src,
-                                          const float *__restrict__ P, int s, int inner, int M, bool inverse)
+                                          const float *__restrict__ T, int s, int inner, int outer)
 {
-    const int p_out = inverse ? 1 : s;  // step in P from one output to the next
-    const int p_in = inverse ? s : 1;   // step in P along the contracted index
-    const int groups = s / TU;
-    const int items = M / TU;
+    const int gj = s / TU;
+    const int gi = VI ? inner / TV : inner;
+    const int go = VI ? outer : outer / TV;
+    const int vstep = VI ? 1 : s * inner;  // distance between the TV inputs (and outputs) of a tile
+    const int items = go * gj * gi;
     for (int it = threadIdx.x; it < items; it += GEN_THREADS) {
-        const int i = it % inner;
-        const int t = it / inner;
-        const int ub = (t % groups) * TU;
-        const int o = t / groups;
-        const float *sp = src + (size_t)o * s * inner + i;
-        const float *pp = P + ub * p_out;
-        float acc[TU];
+        const int ii = it % gi;
+        const int t = it / gi;
+        const int j0 = (t % gj) * TU;
+        const int oo = t / gj;
+        const int o0 = VI ? oo : oo * TV;
+        const int i0 = VI ? ii * TV : ii;
+        const float *sp = src + (size_t)o0 * s * inner + i0;
+        const float *tp = T + j0;
+        float acc[TU][TV];
 #pragma unroll
-        for (int q = 0; q < TU; ++q) acc[q] = 0.f;
+        for (int q = 0; q < TU; ++q)
+#pragma unroll
+            for (int v = 0; v < TV; ++v) acc[q][v] = 0.f;
+#pragma unroll 2
         for (int n = 0; n < s; ++n) {
-            const float v = sp[n * inner];
+            float tv[TU], sv[TV];
+            if constexpr (TU == 4) {  // s, j0 and the table offset are multiples of 4
+                const float4 t4 = __ldg(reinterpret_cast<const float4 *>(tp + n * s));
+                tv[0] = t4.x, tv[1] = t4.y, tv[2] = t4.z, tv[3] = t4.w;
+            } else {
 #pragma unroll
-            for (int q = 0; q < TU; ++q) acc[q] = fmaf(__ldg(pp + q * p_out + n * p_in), v, acc[q]);
+                for (int q = 0; q < TU; ++q) tv[q] = __ldg(tp + n * s + q);
+            }
+            if constexpr (VI && TV == 4) {  // inner and i0 are multiples of 4, the buffers 16-byte aligned
+                const float4 s4 = *reinterpret_cast<const float4 *>(sp + n * inner);
+                sv[0] = s4.x, sv[1] = s4.y, sv[2] = s4.z, sv[3] = s4.w;
+            } else {
+#pragma unroll
+                for (int v = 0; v < TV; ++v) sv[v] = sp[n * inner + v * vstep];
+            }
+#pragma unroll
+            for (int q = 0; q < TU; ++q)
+#pragma unroll
+                for (int v = 0; v < TV; ++v) acc[q][v] = fmaf(tv[q], sv[v], acc[q][v]);
         }
-        float *dp = dst + (size_t)o * s * inner + (size_t)ub * inner + i;
+        float *dp = dst + (size_t)o0 * s * inner + (size_t)j0 * inner + i0;
 #pragma unroll
-        for (int q = 0; q < TU; ++q) dp[q * inner] = acc[q];
+        for (int q = 0; q < TU; ++q) {
+            if constexpr (VI && TV == 4) {
+                *reinterpret_cast<float4 *>(dp + q * inner) = make_float4(acc[q][0], acc[q][1], acc[q][2], acc[q][3]);
+            } else {
+#pragma unroll
+                for (int v = 0; v < TV; ++v) dp[q * inner + v * vstep] = acc[q][v];
+            }
+        }
     }
+}
+
+template <int TU>
+__device__ __forceinline__ void axis_dispatch(float *dst, const float *src, const float *T, int s, int inner, int M)
+{
+    const int outer = M / (s * inner);
+    // 4-wide tiles along i (or o) where the chunk has enough outputs to keep the CTA busy with them
+    if (M >= 16 * GEN_THREADS / 2 && (inner & 3) == 0)
+        axis_pass<TU, 4, true>(dst, src, T, s, inner, outer);
+    else if (M >= 16 * GEN_THREADS / 2 && (outer & 3) == 0)
+        axis_pass<TU, 4, false>(dst, src, T, s, inner, outer);
+    else
+        axis_pass<TU, 1, true>(dst, src, T, s, inner, outer);
 }
 
 // All axes in turn, ping-pong between `a` and `b` (src may be one of them or a third buffer, which is
@@ -99,10 +164,11 @@ __device__ __forceinline__ float *transform_chunk(float *src, float *a, float *b
         inner /= s;
         if (s == 1) continue;
         float *dst = (cur == a) ? b : a;
+        const float *T = tables + e.basis[ax] + (inverse ? 0 : s * s);  // [C | C^T] per extent
         if ((s & 3) == 0)
-            axis_pass<4>(dst, cur, tables + e.basis[ax], s, inner, e.M, inverse);
+            axis_dispatch<4>(dst, cur, T, s, inner, e.M);
         else
-            axis_pass<1>(dst, cur, tables + e.basis[ax], s, inner, e.M, inverse);
+            axis_dispatch<1>(dst, cur, T, s, inner, e.M);
         __syncthreads();
         cur = dst;
     }
@@ -111,19 +177,22 @@ __device__ __forceinline__ float *transform_chunk(float *src, float *a, float *b
 
 __global__ void __launch_bounds__(GEN_THREADS) compress_nd_kernel(DemoNdCompressArgs a)
 {
-    extern __shared__ float smem[];
+    extern __shared__ __align__(16) float smem[];
     float *Bt = smem;
     float *X1 = Bt + a.max_M;
     float *X2 = X1 + a.max_M;
     unsigned *hist = reinterpret_cast<unsigned *>(X2 + a.max_M);  // [256]
     unsigned *warp_tot = hist + 256;                              // [8]
     unsigned *s_state = warp_tot + 8;                             // [2]
+    __shared__ ChunkSlot slot;
     const int tid = threadIdx.x;
+    if (tid == 0) slot.e.chunk_begin = 1, slot.e.chunk_end = 0;  // no tensor yet
 
     for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
-        const DemoNdEntry e = a.entries[find_nd_entry(a.entries, a.n_entries, c)];
+        locate_chunk(&slot, a.entries, a.n_entries, c);
+        const DemoNdEntry &e = slot.e;
         const long long lc = c - e.chunk_begin;
-        const size_t base = chunk_base(e, lc);
+        const size_t base = slot.base;
         float *__restrict__ m = a.m_ptrs[e.tensor];
         const void *g = a.g_ptrs[e.tensor];
         const int M = e.M, k_eff = e.k_eff;
@@ -191,17 +260,20 @@ __global__ void __launch_bounds__(GEN_THREADS) compress_nd_kernel(DemoNdCompress
 
 __global__ void __launch_bounds__(GEN_THREADS) decode_nd_kernel(DemoNdDecodeArgs a)
 {
-    extern __shared__ float smem[];
+    extern __shared__ __align__(16) float smem[];
     float *St = smem;
     float *X1 = St + a.max_M;
     unsigned short *Cn = reinterpret_cast<unsigned short *>(X1 + a.max_M);  // senders per coordinate (agg == 2)
+    __shared__ ChunkSlot slot;
     const int tid = threadIdx.x;
     const bool counts = a.agg == 2;
+    if (tid == 0) slot.e.chunk_begin = 1, slot.e.chunk_end = 0;  // no tensor yet
 
     for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
-        const DemoNdEntry e = a.entries[find_nd_entry(a.entries, a.n_entries, c)];
+        locate_chunk(&slot, a.entries, a.n_entries, c);
+        const DemoNdEntry &e = slot.e;
         const long long lc = c - e.chunk_begin;
-        const size_t base = chunk_base(e, lc);
+        const size_t base = slot.base;
         float *__restrict__ x = a.x_ptrs[e.tensor];
         const int M = e.M, k_eff = e.k_eff;
         const long long rec_off = e.rec_begin + lc * (long long)k_eff;
