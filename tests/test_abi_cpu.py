@@ -112,3 +112,25 @@ def test_binding_checks_the_layout_the_abi_assumes():
         validate_tensors([torch.zeros(6, 4).t(), good[1]], shapes, torch.float32, None, "m")
     with pytest.raises(ValueError, match="expected cuda:0"):
         validate_tensors(good, shapes, torch.float32, 0, "m")
+
+
+def test_divisor_chunk_shapes():
+    """Chunk extents for dimensions that are not multiples of the target: always divisors, never above the
+    target or the library's limits, and the target itself wherever it divides."""
+    import math
+
+    from paper_2411_19870_b200 import chunking
+
+    assert chunking.largest_divisor_at_most(50304, 64) == 64
+    assert chunking.largest_divisor_at_most(50257, 64) == 29      # 50257 = 29 * 1733
+    assert chunking.largest_divisor_at_most(97, 64) == 1          # prime
+    assert chunking.divisor_chunk_shape((2048, 8192), 64) == (64, 64)
+    assert chunking.divisor_chunk_shape((50257, 768), 64) == (29, 64)
+    assert chunking.divisor_chunk_shape((512, 512, 3, 3), 64) == (32, 32, 3, 3)   # 64*64*9 elements is too many
+    assert chunking.divisor_chunk_shape((1000,), 64) == (50,)
+    for shape in ((768, 3072), (50257, 1600), (6, 10, 14), (256, 256, 7, 7), (129,), (16, 16, 16, 16)):
+        for target in (8, 32, 64, 128, 500):
+            ch = chunking.divisor_chunk_shape(shape, target)
+            assert len(ch) == len(shape)
+            assert all(n % s == 0 and 1 <= s <= min(target, chunking.MAX_EXTENT) for n, s in zip(shape, ch))
+            assert math.prod(ch) <= chunking.MAX_CHUNK_ELEMS

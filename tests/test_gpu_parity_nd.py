@@ -141,3 +141,17 @@ def test_randomized_configurations():
         for _ in range(2):
             r.step()
         r.close()
+
+
+def test_dimensions_that_are_not_multiples_of_the_target_chunk():
+    """A vocabulary-sized matrix (50257 = 29 * 1733 rows) and a 7 x 7 convolution weight: every axis gets
+    the largest divisor below the target, and the step matches the oracle on every chunk."""
+    from paper_2411_19870_b200 import chunking
+
+    shapes = [(29 * 6, 192), (16, 24, 7, 7), (1000,)]
+    chunks = [chunking.divisor_chunk_shape(s, 64) for s in shapes]
+    assert chunks == [(58, 64), (16, 12, 7, 7), (50,)]  # 16*24*49 elements would be too many
+    r = parity.NdRunner(shapes, chunks, topk=32, num_workers=2)
+    for _ in range(2):
+        r.step()
+    r.close()
