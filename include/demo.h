@@ -47,8 +47,8 @@ typedef struct demo_ctx demo_ctx; /* opaque, library-owned */
 typedef enum {
     DEMO_OK = 0,
     DEMO_ERR_INVALID_ARG = 1, /* null pointer, bad worker index, misaligned buffer, bad count     */
-    DEMO_ERR_SHAPE = 2,       /* ndim not in {1,2} or a dimension not a multiple of s              */
-    DEMO_ERR_K = 3,           /* k < 1 or k > s*s                                                  */
+    DEMO_ERR_SHAPE = 2,       /* order not supported, or a dimension not a multiple of its chunk   */
+    DEMO_ERR_K = 3,           /* k < 1 or k > s*s (demo_init_nd: k > DEMO_ND_MAX_CHUNK_ELEMS)      */
     DEMO_ERR_UNSUPPORTED = 4, /* s not in {8,16,32,64,128}, unknown dtype, too many tensors        */
     DEMO_ERR_ALLOC = 5,       /* host or device allocation failed                                  */
     DEMO_ERR_CUDA = 6,        /* a CUDA runtime call failed (no device, launch error, ...)         */
@@ -115,7 +115,8 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
  * dense contractions on the CUDA cores (no fast-DCT, tensor-core or side-stream path; demo_set_path has
  * no effect); demo_set_basis, demo_set_basis_gaussian and demo_get_basis return UNSUPPORTED (one basis
  * per chunk extent: only the DCT is built).  A descriptor with ndim <= 2 and equal chunk extents gives
- * the same payload bytes as demo_init with that chunk size.
+ * the payload layout of demo_init with that chunk size and, up to the fp32 rounding of a different
+ * summation order, the same records.
  * Errors: INVALID_ARG, SHAPE (ndim, chunk[a] < 1, shape[a] not a multiple of chunk[a]), K,
  * UNSUPPORTED (chunk extent or chunk too large, dtype, too many tensors), ALLOC, CUDA.
  */

@@ -175,8 +175,8 @@ const char *demo_status_string(demo_status status)
     switch (status) {
         case DEMO_OK: return "ok";
         case DEMO_ERR_INVALID_ARG: return "invalid argument";
-        case DEMO_ERR_SHAPE: return "tensor shape is not 1-D/2-D with dimensions divisible by the chunk size";
-        case DEMO_ERR_K: return "k out of range (1 <= k <= s*s)";
+        case DEMO_ERR_SHAPE: return "tensor order not supported or a dimension is not a multiple of its chunk extent";
+        case DEMO_ERR_K: return "k out of range (1 <= k <= largest chunk)";
         case DEMO_ERR_UNSUPPORTED: return "unsupported chunk size, dtype or tensor count";
         case DEMO_ERR_ALLOC: return "allocation failed";
         case DEMO_ERR_CUDA: return "CUDA runtime error";

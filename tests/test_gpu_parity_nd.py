@@ -58,9 +58,9 @@ def test_aggregation_phi_and_alpha(agg, phi):
     r.close()
 
 
-def test_square_chunks_give_the_bytes_of_the_square_chunk_context():
-    """ndim <= 2 with equal extents: same payload bytes, momenta and parameters as demo_init (both through
-    the dense kernels)."""
+def test_square_chunks_match_the_square_chunk_context():
+    """ndim <= 2 with equal extents: same payload layout and index sets, values / momenta / parameters equal
+    to fp32 rounding of a different summation order (demo_init through its dense kernels)."""
     dev = torch.device("cuda")
     shapes, s, k, W = [(128, 192), (256,)], 32, 17, 2
     kw = dict(topk=k, beta=0.9, lr=1e-3, weight_decay=0.1, num_workers=W, grad_dtype=demo.DEMO_F32)
