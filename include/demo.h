@@ -171,6 +171,30 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
                               float *const *params, void *cuda_stream);
 
 /*
+ * Parameter-server form of the server side (Algorithm 1: the server aggregates and reconstructs the
+ * momentum and broadcasts sgn(m_t); every worker then applies x <- x - lr (sgn + weight_decay x)).
+ *
+ * demo_decode_signs -- S and R as in demo_decode_apply (same aggregation modes), but instead of updating
+ * parameters writes sign(R) in {-1, 0, +1} as one int8 per parameter.
+ *   signs_out    host array of n_tensors DEVICE pointers (int8, each shaped and ordered like its
+ *                parameter tensor), overwritten; 16-byte aligned
+ * Needs phi = DEMO_PHI_SIGN (INVALID_ARG otherwise).  2-D tensors at chunk sizes 32 and 64 run on the fast
+ * kernels, everything else on the dense kernels.
+ *
+ * demo_apply_signs -- x <- x - lr (sign + weight_decay x) for every parameter, from such int8 tensors
+ * (the broadcast's payload), with the context's current lr.
+ *   signs        host array of n_tensors DEVICE pointers (int8), read-only
+ *   params       host array of n_tensors DEVICE pointers (fp32), updated in place
+ * The two calls together leave the parameters demo_decode_apply leaves: bit for bit where that runs on the
+ * dense kernels, within one fp32 rounding of the update where it runs on the fast kernels (which fold
+ * 1 - lr weight_decay into one factor).  The small tables of these two entry points are allocated on the
+ * first call of either.  Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+demo_status demo_decode_signs(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads,
+                              int8_t *const *signs_out, void *cuda_stream);
+demo_status demo_apply_signs(demo_ctx *ctx, const int8_t *const *signs, float *const *params, void *cuda_stream);
+
+/*
  * demo_step_host -- one whole optimizer step driven from HOST gradient buffers: for every worker
  * copy its gradients host->device into the caller's device staging tensors, compress, then decode
  * and apply, then (if host_payloads_out is not NULL) copy all W payloads device->host.  Everything

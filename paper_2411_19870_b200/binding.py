@@ -24,6 +24,7 @@ RECORD_BYTES = 8
 
 EXPORTS = [
     "demo_init", "demo_init_nd", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
+    "demo_decode_signs", "demo_apply_signs",
     "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_set_basis",
     "demo_set_basis_gaussian", "demo_get_basis", "demo_selftest_bounded_wait", "demo_set_path", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
@@ -82,6 +83,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_compress.restype = i32
     lib.demo_decode_apply.argtypes = [vp, pvp, i32, pvp, vp]
     lib.demo_decode_apply.restype = i32
+    lib.demo_decode_signs.argtypes = [vp, pvp, i32, pvp, vp]
+    lib.demo_decode_signs.restype = i32
+    lib.demo_apply_signs.argtypes = [vp, pvp, pvp, vp]
+    lib.demo_apply_signs.restype = i32
     lib.demo_step_host.argtypes = [vp, pvp, pvp, pvp, pvp, pvp, vp, vp]
     lib.demo_step_host.restype = i32
     lib.demo_decode_apply_static.argtypes = [ctypes.POINTER(DemoConfig), ctypes.POINTER(DemoTensorDesc), i32, pvp, i32,
@@ -271,6 +276,20 @@ class DemoTransform:
                                         self._array("x", params, (self.shapes, torch.float32, True)), self._stream(stream))
         if st != 0:
             raise DemoError(st, "demo_decode_apply")
+
+    def decode_signs(self, payloads, signs_out, stream=None) -> None:
+        """Parameter-server form: sign of the reconstructed momentum as int8 tensors shaped like the parameters."""
+        self._check_payloads(payloads)
+        st = self.lib.demo_decode_signs(self._ctx, self._array("p", payloads), len(payloads),
+                                        self._array("s", signs_out, (self.shapes, torch.int8, True)), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_decode_signs")
+
+    def apply_signs(self, signs, params, stream=None) -> None:
+        st = self.lib.demo_apply_signs(self._ctx, self._array("s", signs, (self.shapes, torch.int8, True)),
+                                       self._array("x", params, (self.shapes, torch.float32, True)), self._stream(stream))
+        if st != 0:
+            raise DemoError(st, "demo_apply_signs")
 
     def step_host(self, host_grads, dev_grads, momentum, payloads, params, host_payloads_out=None, stream=None) -> None:
         """host_grads / dev_grads / momentum: lists over workers of lists of tensors."""

@@ -56,6 +56,9 @@ struct DemoDecodeArgs {
     int agg;          // 0 sum, 1 mean over workers, 2 per-coordinate count-normalised mean (0/0 = 0)
     int phi;          // 0 sign, 1 identity
     float agg_scale;  // 1/W for the mean, else 1 (only the identity update sees it)
+    // Parameter-server form: when not NULL, write sign(R) in {-1, 0, +1} per element to these int8 tensors
+    // (device array indexed like x_ptrs) instead of updating the parameters.
+    signed char *const *sign_ptrs = nullptr;
 };
 
 // Launchers (defined in the kernel translation units).  `s` is the chunk size, `two_d` selects
@@ -131,7 +134,25 @@ struct DemoNdDecodeArgs {
     int *status;
     int agg, phi;
     float agg_scale;
+    signed char *const *sign_ptrs = nullptr;  // see DemoDecodeArgs
 };
+
+// x <- x - lr (sign + wd x) from int8 signs, over every tensor of a context (kernels_generic.cu).
+struct DemoFlatEntry {
+    long long quad_begin;  // index of this tensor's first group of four elements in the launch
+    long long n;           // elements
+    int tensor;            // position in the pointer arrays
+    int pad;
+};
+struct DemoApplySignsArgs {
+    const DemoFlatEntry *entries;  // device
+    int n_entries;
+    long long n_quads;
+    const signed char *const *sign_ptrs;  // device array
+    float *const *x_ptrs;                 // device array
+    float lr, wd;
+};
+cudaError_t demo_launch_apply_signs(const DemoApplySignsArgs &a, int sm_count, cudaStream_t stream);
 
 cudaError_t demo_launch_compress_nd(const DemoNdCompressArgs &a, int sm_count, cudaStream_t stream);
 cudaError_t demo_launch_decode_nd(const DemoNdDecodeArgs &a, int sm_count, cudaStream_t stream);

@@ -52,6 +52,11 @@ struct demo_ctx {
     float **d_m = nullptr;           // [W][T]
     float **d_x = nullptr;           // [T]
     const DemoRecord **d_p = nullptr;  // [W]
+    signed char **d_s = nullptr;       // [T] sign tensors of the parameter-server form
+    std::vector<signed char *> h_s;
+    bool s_valid = false;
+    DemoFlatEntry *d_flat = nullptr;   // [T] element ranges for demo_apply_signs
+    long long n_quads = 0;
     std::vector<const void *> h_g;
     std::vector<float *> h_m, h_x;
     std::vector<const DemoRecord *> h_p;
@@ -153,6 +158,8 @@ void release(demo_ctx *c)
     cudaFree((void *)c->d_m);
     cudaFree((void *)c->d_x);
     cudaFree((void *)c->d_p);
+    cudaFree((void *)c->d_s);
+    cudaFree(c->d_flat);
     cudaFree(c->d_tm_g);
     cudaFree(c->d_tm_m);
     cudaFree(c->d_tm_x);
@@ -648,31 +655,85 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
     return DEMO_OK;
 }
 
-demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads, float *const *params,
-                              void *cuda_stream)
+// Tables of the parameter-server entry points, built on first use: the device array of sign-tensor
+// pointers and the element ranges demo_apply_signs walks.
+static demo_status ensure_sign_tables(demo_ctx *ctx)
 {
-    if (!ctx || !payloads || !params) return DEMO_ERR_INVALID_ARG;
+    if (ctx->d_s && ctx->d_flat) return DEMO_OK;
+    const int T = ctx->n_tensors;
+    std::vector<DemoFlatEntry> flat;
+    try {
+        ctx->h_s.assign((size_t)T, nullptr);
+        flat.resize((size_t)T);
+    } catch (const std::bad_alloc &) {
+        return DEMO_ERR_ALLOC;
+    }
+    long long q = 0;
+    for (int t = 0; t < T; ++t) {
+        flat[t].quad_begin = q;
+        flat[t].n = ctx->n_elems[t];
+        flat[t].tensor = t;
+        flat[t].pad = 0;
+        q += (ctx->n_elems[t] + 3) / 4;
+    }
+    ctx->n_quads = q;
+    if (!ctx->d_s && cudaMalloc((void **)&ctx->d_s, (size_t)T * sizeof(void *)) != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_ALLOC;
+    }
+    if (!ctx->d_flat) {
+        if (cudaMalloc(&ctx->d_flat, (size_t)T * sizeof(DemoFlatEntry)) != cudaSuccess) {
+            cudaGetLastError();
+            return DEMO_ERR_ALLOC;
+        }
+        if (cudaMemcpy(ctx->d_flat, flat.data(), (size_t)T * sizeof(DemoFlatEntry), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(ctx->d_flat);
+            ctx->d_flat = nullptr;
+            return DEMO_ERR_CUDA;
+        }
+    }
+    return DEMO_OK;
+}
+
+// demo_decode_apply (params != NULL) and demo_decode_signs (signs != NULL) share everything but the last
+// step of the kernels.
+static demo_status decode_common(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads, float *const *params,
+                                 signed char *const *signs, void *cuda_stream)
+{
+    if (!ctx || !payloads || (!params && !signs)) return DEMO_ERR_INVALID_ARG;
     if (n_payloads != ctx->cfg.num_workers) return DEMO_ERR_INVALID_ARG;
     const int T = ctx->n_tensors, W = n_payloads;
     for (int w = 0; w < W; ++w)
         if (!payloads[w] || !aligned16(payloads[w])) return DEMO_ERR_INVALID_ARG;
-    for (int t = 0; t < T; ++t)
-        if (!params[t] || !aligned16(params[t])) return DEMO_ERR_INVALID_ARG;
+    for (int t = 0; t < T; ++t) {
+        if (params && (!params[t] || !aligned16(params[t]))) return DEMO_ERR_INVALID_ARG;
+        if (signs && (!signs[t] || !aligned16(signs[t]))) return DEMO_ERR_INVALID_ARG;
+    }
+    if (signs && ctx->phi != DEMO_PHI_SIGN) return DEMO_ERR_INVALID_ARG;  // only the sign is handed out
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DEMO_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (signs) {
+        const demo_status st = ensure_sign_tables(ctx);
+        if (st != DEMO_OK) return st;
+    }
 
     cudaError_t err = sync_table<const DemoRecord *>(ctx->d_p, ctx->h_p.data(),
                                                      reinterpret_cast<const DemoRecord *const *>(payloads), W,
                                                      &ctx->p_valid, stream);
     bool x_changed = false;
-    if (err == cudaSuccess)
+    if (err == cudaSuccess && params)
         err = sync_table<float *>(ctx->d_x, ctx->h_x.data(), const_cast<float *const *>(params), T, &ctx->x_valid,
                                   stream, &x_changed);
-    if (err == cudaSuccess && ctx->encode && x_changed && !upload_tensor_maps(ctx, ctx->d_tm_x, params, false, stream)) {
+    if (err == cudaSuccess && params && ctx->encode && x_changed &&
+        !upload_tensor_maps(ctx, ctx->d_tm_x, params, false, stream)) {
         err = cudaErrorInvalidValue;
         ctx->x_valid = false;
     }
+    if (err == cudaSuccess && signs)
+        err = sync_table<signed char *>(ctx->d_s, ctx->h_s.data(), const_cast<signed char *const *>(signs), T,
+                                        &ctx->s_valid, stream);
     if (err != cudaSuccess) {
         cudaGetLastError();
         return DEMO_ERR_CUDA;
@@ -694,6 +755,7 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
         n.agg = ctx->aggregation;
         n.phi = ctx->phi;
         n.agg_scale = (ctx->aggregation == DEMO_AGG_MEAN) ? 1.0f / (float)W : 1.0f;
+        n.sign_ptrs = signs ? ctx->d_s : nullptr;
         if (demo_launch_decode_nd(n, ctx->sm_count, stream) != cudaSuccess) {
             cudaGetLastError();
             return DEMO_ERR_CUDA;
@@ -710,10 +772,11 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     a.lr = ctx->cfg.lr;
     a.wd = ctx->cfg.weight_decay;
     a.status = ctx->d_status;
-    a.tmap_x = ctx->encode ? ctx->d_tm_x : nullptr;
+    a.tmap_x = (ctx->encode && params) ? ctx->d_tm_x : nullptr;
     a.agg = ctx->aggregation;
     a.phi = ctx->phi;
     a.agg_scale = (ctx->aggregation == DEMO_AGG_MEAN) ? 1.0f / (float)W : 1.0f;
+    a.sign_ptrs = signs ? ctx->d_s : nullptr;
     const int s = ctx->cfg.chunk;
     cudaStream_t side = stream;
     if (ctx->n1d) {
@@ -728,9 +791,10 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
-        if (use_fast_path(ctx))
+        // the signs come from the fast kernels at s in {32, 64} and from the dense kernels elsewhere
+        if (use_fast_path(ctx) && (!signs || s != 128))
             err = demo_launch_decode_fast(s, a, ctx->sm_count, stream);
-        else if (use_tc_path(ctx))
+        else if (use_tc_path(ctx) && !signs)
             err = demo_launch_decode_tc(a, ctx->sm_count, stream);
         else
             err = demo_launch_decode_generic(s, 1, a, ctx->sm_count, stream);
@@ -739,6 +803,62 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
     {
         const cudaError_t jerr = join_side(ctx, side, stream);
         if (err == cudaSuccess) err = jerr;
+    }
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return DEMO_ERR_CUDA;
+    }
+    return DEMO_OK;
+}
+
+demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads, float *const *params,
+                              void *cuda_stream)
+{
+    if (!params) return DEMO_ERR_INVALID_ARG;
+    return decode_common(ctx, payloads, n_payloads, params, nullptr, cuda_stream);
+}
+
+demo_status demo_decode_signs(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads, int8_t *const *signs_out,
+                              void *cuda_stream)
+{
+    if (!signs_out) return DEMO_ERR_INVALID_ARG;
+    return decode_common(ctx, payloads, n_payloads, nullptr, reinterpret_cast<signed char *const *>(signs_out),
+                         cuda_stream);
+}
+
+demo_status demo_apply_signs(demo_ctx *ctx, const int8_t *const *signs, float *const *params, void *cuda_stream)
+{
+    if (!ctx || !signs || !params) return DEMO_ERR_INVALID_ARG;
+    const int T = ctx->n_tensors;
+    for (int t = 0; t < T; ++t)
+        if (!signs[t] || !params[t] || !aligned16(signs[t]) || !aligned16(params[t])) return DEMO_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DEMO_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const demo_status st = ensure_sign_tables(ctx);
+    if (st != DEMO_OK) return st;
+    bool x_changed = false;
+    cudaError_t err = sync_table<float *>(ctx->d_x, ctx->h_x.data(), const_cast<float *const *>(params), T,
+                                          &ctx->x_valid, stream, &x_changed);
+    if (err == cudaSuccess && ctx->encode && x_changed && !upload_tensor_maps(ctx, ctx->d_tm_x, params, false, stream)) {
+        err = cudaErrorInvalidValue;
+        ctx->x_valid = false;
+    }
+    if (err == cudaSuccess)
+        err = sync_table<signed char *>(ctx->d_s, ctx->h_s.data(),
+                                        const_cast<signed char *const *>(reinterpret_cast<const signed char *const *>(signs)),
+                                        T, &ctx->s_valid, stream);
+    if (err == cudaSuccess) {
+        DemoApplySignsArgs a;
+        a.entries = ctx->d_flat;
+        a.n_entries = T;
+        a.n_quads = ctx->n_quads;
+        a.sign_ptrs = ctx->d_s;
+        a.x_ptrs = ctx->d_x;
+        a.lr = ctx->cfg.lr;
+        a.wd = ctx->cfg.weight_decay;
+        err = demo_launch_apply_signs(a, ctx->sm_count, stream);
+        ctx->launches += 1;
     }
     if (err != cudaSuccess) {
         cudaGetLastError();

@@ -544,7 +544,9 @@ __host__ __device__ constexpr size_t decode_slot_bytes(bool counts)
     return ((size_t)S * Cfg<S>::XS * 4 + 16 + (counts ? (size_t)S * S * 2 : 0) + 127) / 128 * 128;
 }
 
-template <int S, bool TMAP, int THREADS>
+// SIGNS: the parameter-server form -- sign(R) goes out as int8 per element, the parameters are neither read
+// nor written (a separate instantiation, so that the update kernel keeps its size).
+template <int S, bool TMAP, int THREADS, bool SIGNS = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(DemoDecodeArgs a)
 {
     using C = Cfg<S>;
@@ -598,7 +600,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
         float *__restrict__ x = x_ptr;
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + lc * (long long)k_eff;
-        if (TMAP && t == 0)
+        if (TMAP && !SIGNS && t == 0)
             tma_prefetch_2d(static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES, k1 * S, (int)k0 * S);
 
         {
@@ -661,7 +663,9 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
                 for (int u = 0; u < S; ++u) r[u] = St[u * XS + t];
                 fence_proxy_async();
                 sb.sync();  // the tile is dead: stage x into it
-                if (TMAP) {
+                if (SIGNS) {
+                    // nothing to stage
+                } else if (TMAP) {
                     if (t == 0) {
                         mbar_expect_tx(bar, S * S * sizeof(float));
                         tma_load_2d(smem_u32(Xt), static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES,
@@ -679,10 +683,17 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
                 for (int v4 = 0; v4 < S / 4; ++v4)
                     row[v4] = make_float4(r[4 * v4], r[4 * v4 + 1], r[4 * v4 + 2], r[4 * v4 + 3]);
                 sb.sync();
-            } else {
+            } else if (!SIGNS) {
                 arrived = mbar_wait_bounded(bar, phase);
                 phase ^= 1u;
             }
+        }
+        if constexpr (SIGNS) {
+            signed char *__restrict__ sg = a.sign_ptrs[te.tensor];
+#pragma unroll
+            for (int i = 0; i < S; ++i) sg[base + (size_t)i * te.n1 + t] = (signed char)((r[i] > 0.f) - (r[i] < 0.f));
+            sb.sync();  // the tile is free again
+            continue;
         }
         if (!sb.sync_and(arrived)) {
             if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
@@ -752,6 +763,8 @@ cudaError_t launch_decode(const DemoDecodeArgs &a, int sm_count, cudaStream_t st
     constexpr int TH = DECODE_THREADS;
     constexpr int NCH = TH / S;
     const size_t smem = decode_slot_bytes<S>(a.agg == 2) * NCH;
+    if (a.sign_ptrs != nullptr)
+        return launch(decode_fast_kernel<S, false, TH, true>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
     if (a.tmap_x != nullptr)
         return launch(decode_fast_kernel<S, true, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
     return launch(decode_fast_kernel<S, false, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);

@@ -226,11 +226,50 @@ __global__ void __launch_bounds__(GEN_THREADS) decode_generic_kernel(DemoDecodeA
             const int r = i / S, j = i - r * S;
             const size_t off = base + (size_t)r * te.n1 + j;
             const float rv = R[i];
+            if (a.sign_ptrs) {  // parameter-server form: hand out sign(R), the workers apply it
+                a.sign_ptrs[te.tensor][off] = (signed char)((rv > 0.f) - (rv < 0.f));
+                continue;
+            }
             const float sg = a.phi ? rv * a.agg_scale : (float)((rv > 0.f) - (rv < 0.f));
             const float xv = x[off];
             x[off] = fmaf(-a.lr, fmaf(a.wd, xv, sg), xv);
         }
         __syncthreads();
+    }
+}
+
+// x <- x - lr (sign + wd x) with the signs a parameter server handed out (Algorithm 1, last two lines).
+// One thread per group of four consecutive elements of a tensor; same arithmetic as the decode kernels.
+__global__ void __launch_bounds__(GEN_THREADS) apply_signs_kernel(DemoApplySignsArgs a)
+{
+    for (long long q = (long long)blockIdx.x * GEN_THREADS + threadIdx.x; q < a.n_quads;
+         q += (long long)gridDim.x * GEN_THREADS) {
+        int lo = 0, hi = a.n_entries - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (a.entries[mid].quad_begin <= q)
+                lo = mid;
+            else
+                hi = mid - 1;
+        }
+        const DemoFlatEntry e = a.entries[lo];
+        const long long i0 = (q - e.quad_begin) * 4;
+        float *__restrict__ x = a.x_ptrs[e.tensor];
+        const signed char *__restrict__ sg = a.sign_ptrs[e.tensor];
+        if (i0 + 4 <= e.n) {  // tensors start 16-byte aligned, so groups of four are aligned too
+            float4 xv = *reinterpret_cast<const float4 *>(x + i0);
+            const char4 s4 = *reinterpret_cast<const char4 *>(sg + i0);
+            xv.x = fmaf(-a.lr, fmaf(a.wd, xv.x, (float)s4.x), xv.x);
+            xv.y = fmaf(-a.lr, fmaf(a.wd, xv.y, (float)s4.y), xv.y);
+            xv.z = fmaf(-a.lr, fmaf(a.wd, xv.z, (float)s4.z), xv.z);
+            xv.w = fmaf(-a.lr, fmaf(a.wd, xv.w, (float)s4.w), xv.w);
+            *reinterpret_cast<float4 *>(x + i0) = xv;
+        } else {
+            for (long long i = i0; i < e.n; ++i) {
+                const float xv = x[i];
+                x[i] = fmaf(-a.lr, fmaf(a.wd, xv, (float)sg[i]), xv);
+            }
+        }
     }
 }
 
@@ -267,6 +306,16 @@ cudaError_t demo_launch_compress_generic(int s, int two_d, const DemoCompressArg
         case 128: return compress_dispatch<128>(two_d, a, sm_count, stream);
         default: return cudaErrorInvalidValue;
     }
+}
+
+cudaError_t demo_launch_apply_signs(const DemoApplySignsArgs &a, int sm_count, cudaStream_t stream)
+{
+    if (a.n_quads <= 0) return cudaSuccess;
+    long long grid = (a.n_quads + GEN_THREADS - 1) / GEN_THREADS;
+    const long long cap = (long long)sm_count * 8;
+    if (grid > cap) grid = cap;
+    apply_signs_kernel<<<(unsigned)grid, GEN_THREADS, 0, stream>>>(a);
+    return cudaGetLastError();
 }
 
 cudaError_t demo_launch_decode_generic(int s, int two_d, const DemoDecodeArgs &a, int sm_count,

@@ -353,6 +353,10 @@ __global__ void __launch_bounds__(GEN_THREADS) decode_nd_kernel(DemoNdDecodeArgs
         for (int i = tid; i < M; i += GEN_THREADS) {
             const size_t off = base + elem_offset(e, i);
             const float rv = R[i];
+            if (a.sign_ptrs) {  // parameter-server form: hand out sign(R), the workers apply it
+                a.sign_ptrs[e.tensor][off] = (signed char)((rv > 0.f) - (rv < 0.f));
+                continue;
+            }
             const float sg = a.phi ? rv * a.agg_scale : (float)((rv > 0.f) - (rv < 0.f));
             const float xv = x[off];
             x[off] = fmaf(-a.lr, fmaf(a.wd, xv, sg), xv);
