@@ -187,8 +187,11 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
  *   params       host array of n_tensors DEVICE pointers (fp32), updated in place
  * The two calls together leave the parameters demo_decode_apply leaves: bit for bit where that runs on the
  * dense kernels, within one fp32 rounding of the update where it runs on the fast kernels (which fold
- * 1 - lr weight_decay into one factor).  The small tables of these two entry points are allocated on the
- * first call of either.  Errors: INVALID_ARG, ALLOC, CUDA.
+ * 1 - lr weight_decay into one factor).  Where the two forms run on different kernel families (chunk size
+ * 128; a caller-supplied basis at chunk size 64) an element whose reconstructed momentum is zero to
+ * rounding may get another sign, as between any two of the kernel families.  The small tables of these
+ * two entry points are allocated on the first call of either (so the first call cannot be part of a
+ * stream capture).  Errors: INVALID_ARG, ALLOC, CUDA.
  */
 demo_status demo_decode_signs(demo_ctx *ctx, const void *const *payloads, int32_t n_payloads,
                               int8_t *const *signs_out, void *cuda_stream);
