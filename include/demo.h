@@ -178,8 +178,9 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
  * parameters writes sign(R) in {-1, 0, +1} as one int8 per parameter.
  *   signs_out    host array of n_tensors DEVICE pointers (int8, each shaped and ordered like its
  *                parameter tensor), overwritten; 16-byte aligned
- * Needs phi = DEMO_PHI_SIGN (INVALID_ARG otherwise).  2-D tensors at chunk sizes 32 and 64 run on the fast
- * kernels, everything else on the dense kernels.
+ * Needs phi = DEMO_PHI_SIGN (INVALID_ARG otherwise).  2-D tensors run on the fast kernels where
+ * demo_decode_apply does, everything else (and every tensor under a caller-supplied basis) on the dense
+ * kernels.
  *
  * demo_apply_signs -- x <- x - lr (sign + weight_decay x) for every parameter, from such int8 tensors
  * (the broadcast's payload), with the context's current lr.
@@ -187,9 +188,9 @@ demo_status demo_decode_apply(demo_ctx *ctx, const void *const *payloads, int32_
  *   params       host array of n_tensors DEVICE pointers (fp32), updated in place
  * The two calls together leave the parameters demo_decode_apply leaves: bit for bit where that runs on the
  * dense kernels, within one fp32 rounding of the update where it runs on the fast kernels (which fold
- * 1 - lr weight_decay into one factor).  Where the two forms run on different kernel families (chunk size
- * 128; a caller-supplied basis at chunk size 64) an element whose reconstructed momentum is zero to
- * rounding may get another sign, as between any two of the kernel families.  The small tables of these
+ * 1 - lr weight_decay into one factor).  Where the two forms run on different kernel families (a
+ * caller-supplied basis at chunk size 64: tensor cores against CUDA cores) an element whose reconstructed
+ * momentum is zero to rounding may get another sign, as between any two of the kernel families.  The small tables of these
  * two entry points are allocated on the first call of either (so the first call cannot be part of a
  * stream capture).  Errors: INVALID_ARG, ALLOC, CUDA.
  */

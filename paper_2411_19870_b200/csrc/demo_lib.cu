@@ -791,8 +791,8 @@ static demo_status decode_common(demo_ctx *ctx, const void *const *payloads, int
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
-        // the signs come from the fast kernels at s in {32, 64} and from the dense kernels elsewhere
-        if (use_fast_path(ctx) && (!signs || s != 128))
+        // (a caller-supplied basis: the signs come from the dense kernels, there is no tensor-core variant)
+        if (use_fast_path(ctx))
             err = demo_launch_decode_fast(s, a, ctx->sm_count, stream);
         else if (use_tc_path(ctx) && !signs)
             err = demo_launch_decode_tc(a, ctx->sm_count, stream);

@@ -443,6 +443,8 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
 
 constexpr size_t decode128_smem(bool counts) { return (size_t)S * XSD * 4 + 16 + (counts ? (size_t)M * 2 : 0); }
 
+// SIGNS: the parameter-server form -- sign(R) goes out as int8, the parameters are not touched.
+template <bool SIGNS>
 __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -477,7 +479,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + (long long)lc * k_eff;
         const char *tm_x = static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES;
-        if (tid == 0) tma_prefetch_2d(tm_x, k1 * S, k0 * S);
+        if (!SIGNS && tid == 0) tma_prefetch_2d(tm_x, k1 * S, k0 * S);
 
         for (int i = tid; i < S * XSD / 4; i += THREADS) reinterpret_cast<float4 *>(St)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (counts)
@@ -541,7 +543,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
 #pragma unroll
                 for (int n = 0; n < H; ++n) St[line + (h ? (S - 1 - n) : n) * step] = out[n];
                 __syncthreads();
-            } else {
+            } else if (!SIGNS) {
                 if (tid == 0) {
                     mbar_expect_tx(bar, M * sizeof(float));
                     tma_load_2d(smem_u32(Xt), tm_x, k1 * S, k0 * S, bar);
@@ -549,6 +551,16 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
                 arrived = mbar_wait_bounded(bar, phase);
                 phase ^= 1u;
             }
+        }
+        if constexpr (SIGNS) {
+            signed char *__restrict__ sg = a.sign_ptrs[te.tensor];
+#pragma unroll
+            for (int n = 0; n < H; ++n) {
+                const int row = h ? (S - 1 - n) : n;
+                sg[base + (size_t)row * te.n1 + j] = (signed char)((out[n] > 0.f) - (out[n] < 0.f));
+            }
+            __syncthreads();
+            continue;
         }
         if (!__syncthreads_and(arrived)) {
             if (tid == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
@@ -598,6 +610,7 @@ cudaError_t demo_launch_compress_fast128(const DemoCompressArgs &a, int sm_count
 
 cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream)
 {
+    if (a.sign_ptrs) return launch128(decode_fast128_kernel<true>, decode128_smem(a.agg == 2), a.n_chunks, sm_count, stream, &a);
     if (!a.tmap_x) return cudaErrorNotSupported;
-    return launch128(decode_fast128_kernel, decode128_smem(a.agg == 2), a.n_chunks, sm_count, stream, &a);
+    return launch128(decode_fast128_kernel<false>, decode128_smem(a.agg == 2), a.n_chunks, sm_count, stream, &a);
 }
