@@ -224,6 +224,10 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
 
         // ---- top-k ------------------------------------------------------------------------------
         bool use_fallback = (k_eff > S);
+        // A chunk whose coefficients are all zero (a gradient tile that was never touched, e.g. unused
+        // embedding rows, on a momentum that is still zero) needs no selection: the tie rule gives it the
+        // records 0 .. k_eff-1 with value 0.  Slot-uniform; found from the per-thread maxima.
+        bool zero_chunk = false;
         unsigned n_cw = 0, off = 0;
         unsigned mlo = 0u, mhi = 0u;
         if (!use_fallback) {
@@ -260,10 +264,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                 const unsigned both_min = min(tkey, okey), both_max = max(tkey, okey);
                 const unsigned lo_all = __reduce_min_sync(0xffffffffu, both_min);
                 const unsigned hi_all = __reduce_max_sync(0xffffffffu, both_max);
+                zero_chunk = (hi_all == 0u);
                 const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
                 unsigned prefix = lo_all & ~((2u << b0) - 1u);
 #pragma unroll 1
-                for (int b = b0; b >= 15; --b) {
+                for (int b = zero_chunk ? 14 : b0; b >= 15; --b) {
                     const unsigned cand = prefix | (1u << b);
                     const unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand)) +
                                          __popc(__ballot_sync(0xffffffffu, okey >= cand));
@@ -271,37 +276,48 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                 }
                 lmin = prefix;
             }
-            const float L = __uint_as_float(lmin);
-            // candidates: coefficients with magnitude >= L (at least k_eff of them exist).
-            // |q| >= L  <=>  |q| > Lm with Lm the float just below L; the sign bit of Lm - |q| is
-            // shifted into a bit mask (independent chains of 16).
-            const float Lm = (L > 0.f) ? __uint_as_float(lmin - 1u) : -1.f;
-            unsigned mc[S / 16];
-#pragma unroll
-            for (int ch = 0; ch < S / 16; ++ch) {
-                unsigned mm = 0u;
-#pragma unroll
-                for (int j = 15; j >= 0; --j)
-                    mm = __funnelshift_l(__float_as_uint(Lm - fabsf(q[16 * ch + j])), mm, 1);
-                mc[ch] = mm;
+            if (!zero_chunk) {
+                const float L = __uint_as_float(lmin);
+                // candidates: coefficients with magnitude >= L (at least k_eff of them exist).
+                // |q| >= L  <=>  |q| > Lm with Lm the float just below L; the sign bit of Lm - |q| is
+                // shifted into a bit mask (independent chains of 16).
+                const float Lm = (L > 0.f) ? __uint_as_float(lmin - 1u) : -1.f;
+                unsigned mc[S / 16];
+    #pragma unroll
+                for (int ch = 0; ch < S / 16; ++ch) {
+                    unsigned mm = 0u;
+    #pragma unroll
+                    for (int j = 15; j >= 0; --j)
+                        mm = __funnelshift_l(__float_as_uint(Lm - fabsf(q[16 * ch + j])), mm, 1);
+                    mc[ch] = mm;
+                }
+                mlo = mc[0] | (mc[1] << 16);
+                if (S == 64) mhi = mc[S / 16 - 2] | (mc[S / 16 - 1] << 16);
+                // each warp compacts its candidates into its own list (rows of warp 0 precede rows of
+                // warp 1, so the concatenation is in ascending index order)
+                const unsigned cnt = __popc(mlo) + __popc(mhi);
+                const unsigned inc = warp_inclusive_scan(cnt, lane);
+                off = inc - cnt;
+                n_cw = __shfl_sync(0xffffffffu, inc, 31);
+                if (lane == 0) misc[warp] = n_cw;
             }
-            mlo = mc[0] | (mc[1] << 16);
-            if (S == 64) mhi = mc[S / 16 - 2] | (mc[S / 16 - 1] << 16);
-            // each warp compacts its candidates into its own list (rows of warp 0 precede rows of
-            // warp 1, so the concatenation is in ascending index order)
-            const unsigned cnt = __popc(mlo) + __popc(mhi);
-            const unsigned inc = warp_inclusive_scan(cnt, lane);
-            off = inc - cnt;
-            n_cw = __shfl_sync(0xffffffffu, inc, 31);
-            if (lane == 0) misc[warp] = n_cw;
         }
         // stash the coefficients of row t (own row: no hazard with other threads)
-        {
+        if (!zero_chunk) {
             float4 *row = reinterpret_cast<float4 *>(X + t * XS);
 #pragma unroll
             for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(q[4 * v4], q[4 * v4 + 1], q[4 * v4 + 2], q[4 * v4 + 3]);
         }
-        if (!use_fallback) {
+        if (zero_chunk) {
+            // k_eff <= S here: record i is (idx i, value 0); the row-stage list gets the same zeros
+            if (t < k_eff) {
+                DemoRecord r;
+                r.idx = t;
+                r.val = 0.f;
+                rec[t] = r;
+            }
+            if (t < ((k_eff + 7) & ~7)) recs4[t] = make_int4(0, 0, 0, 0);
+        } else if (!use_fallback) {
             const unsigned lbase = warp * CAPWP;
             if (n_cw <= CAPW) {
                 unsigned o = lbase + off;

@@ -223,10 +223,25 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                     for (int i = 0; i < 8; ++i) cnt += __popc(__ballot_sync(0xffffffffu, k8[i] >= cand));
                     prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
                 }
-                if (lane == 0) s_state[2] = prefix;
+                if (lane == 0) {
+                    s_state[2] = prefix;
+                    s_state[3] = hi;  // largest magnitude key of the chunk (read before the scan below reuses the word)
+                }
             }
             __syncthreads();
             const unsigned lmin = s_state[2];
+            // every coefficient zero (a tile that no gradient has touched yet): no selection needed, the tie
+            // rule gives the records 0 .. k_eff-1 with value 0
+            const bool zero_chunk = s_state[3] == 0u;
+            if (zero_chunk) {
+                if (tid < k_eff) {
+                    DemoRecord r;
+                    r.idx = tid;
+                    r.val = 0.f;
+                    rec[tid] = r;
+                    if (k_eff <= 128) recs4[tid] = make_int4((tid >> 7) * XS, (tid & 127) * S, 0, 0);
+                }
+            } else {
             // candidates of this thread as a bit mask over its 64 values
             unsigned long long mask = 0ull;
 #pragma unroll
@@ -282,6 +297,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                         recs4[pos] = make_int4((r.idx >> 7) * XS, (r.idx & 127) * S, __float_as_int(a.alpha * r.val), 0);
                 }
             }
+            }  // !zero_chunk
         }
         // ---- radix select on the magnitude bits, then index-ordered compaction -----------------------
         if (use_radix) {

@@ -412,6 +412,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) compress_tc_kernel(DemoCompress
                 const unsigned okey = misc[4 + (r ^ 32)];
                 const unsigned lo_all = __reduce_min_sync(0xffffffffu, min(tkey, okey));
                 const unsigned hi_all = __reduce_max_sync(0xffffffffu, max(tkey, okey));
+                if (hi_all == 0u) {
+                    // every coefficient zero (a tile no gradient has touched yet): no selection needed, the
+                    // tie rule gives the records 0 .. k_eff-1 (all in row 0, k_eff <= 64 here) with value 0
+                    if (r < k_eff) {
+                        DemoRecord rc;
+                        rc.idx = r;
+                        rc.val = 0.f;
+                        rec[r] = rc;
+                    }
+                    keep = (r == 0) ? (k_eff >= 64 ? ~0ull : ((1ull << k_eff) - 1ull)) : 0ull;
+                } else {
                 const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
                 unsigned lmin = lo_all & ~((2u << b0) - 1u);
 #pragma unroll 1
@@ -482,6 +493,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) compress_tc_kernel(DemoCompress
                     sb.sync();
                     keep = ((unsigned long long)rowmask[2 * r + 1] << 32) | rowmask[2 * r];
                 }
+                }  // chunk not all zero
             }
             if (use_radix) {
                 sb.sync();  // the coefficient tile is complete; the candidate path (if it ran) is done with its lists

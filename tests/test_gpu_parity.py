@@ -609,3 +609,25 @@ def test_bounded_wait_expires_into_a_status_and_the_context_survives():
     assert r.tr.device_status() == 0       # ... reported once, then cleared
     r.step()                               # parity-checked step on the same context
     r.close()
+
+
+@pytest.mark.parametrize("s,basis", [(32, None), (64, None), (128, None), (64, "random")])
+def test_untouched_tiles_among_ordinary_ones(s, basis):
+    """Row blocks whose gradient is exactly zero on a zero momentum (embedding rows of tokens that did not occur):
+    their chunks take the all-zero shortcut of the fast, s = 128 and tensor-core kernels while their neighbours
+    go through the ordinary selection; every chunk is checked against the oracle, two steps."""
+    wl = inputs.Workload("zero-rows", [(6 * s, 4 * s), (3 * s, 5 * s)], chunk=s, topk=min(32, s), num_workers=2,
+                         grad_kind="normal", grad_std=1e-3)
+    kw = dict(gauss=inputs.basis_gaussian(9, s).numpy()) if basis else {}
+    r = parity.Runner(wl, max_chunks=10**9, **kw)
+    for step in range(2):
+        grads = [st.next() for st in r.streams]
+        for g in grads:
+            g[0][s:3 * s] = 0          # two chunk rows of the first tensor
+            g[1][:, 2 * s:3 * s] = 0   # one chunk column of the second
+        r.step(grads=grads)
+    # the zero chunks' records are the lowest indices with value 0
+    first, n_chunks, k_eff = r.layout[0]
+    rec = parity.gather_records(r.payloads[0], first, k_eff, np.arange(4, 12, dtype=np.int64))
+    assert np.array_equal(rec["idx"], np.tile(np.arange(k_eff, dtype=np.int32), (8, 1))) and np.all(rec["val"] == 0)
+    r.close()
