@@ -61,6 +61,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
     constexpr int CAPW = CAP / NW;        // candidate capacity of one warp's list
     constexpr int CAPWP = CAPW + 4;       // list stride (padding for 128-bit key loads)
     constexpr int ITER = CAPW / 32;
+    constexpr int WCAPW = (S == 64) ? 256 : 160;  // capacity of one warp's wide list (tiles of low rank)
+    constexpr int WCAPWP = WCAPW + 4;
+    constexpr int WITER = WCAPW / 32;
+    static_assert(compress_region_bytes<S, GT>() >= (size_t)S * XS * sizeof(float) + (size_t)NW * WCAPWP * 8,
+                  "the wide candidate lists live behind the coefficient tile");
 
     extern __shared__ __align__(128) unsigned char smem_all[];
     const int slot = threadIdx.x / S;
@@ -230,6 +235,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
         bool zero_chunk = false;
         unsigned n_cw = 0, off = 0;
         unsigned mlo = 0u, mhi = 0u;
+        unsigned lmin_w = 0u;  // the bound L as a magnitude key (every candidate's key is >= it)
         if (!use_fallback) {
             // per-thread maximum magnitude: independent chains of 16 with 3-input max.  With S = 32 the two
             // chains stay apart (two maxima per thread): 64 groups again, so that the bound is still useful
@@ -275,6 +281,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                     prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
                 }
                 lmin = prefix;
+                lmin_w = prefix;
             }
             if (!zero_chunk) {
                 const float L = __uint_as_float(lmin);
@@ -345,7 +352,139 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             // candidates themselves); with NaN coefficients the comparisons above fail, and the select on
             // the integer keys, which orders every bit pattern, takes over.
             use_fallback = use_fallback || (n_all < (unsigned)k_eff);
-            if (!use_fallback) {
+            // Tiles of low rank (one active row or column: embedding and output-layer gradients) have row
+            // maxima that bound the k-th coefficient loosely and list a few hundred candidates.  Lists of up
+            // to WCAPW entries per warp, kept in the part of the staging area that the coefficient tile does
+            // not cover, are ranked by a compact (rolled) version of the code below instead of sending the
+            // whole chunk through the radix select.
+            bool wide = false;
+            if constexpr (NW > 1) {
+                // Too many candidates: the maxima of the 64 COLUMNS bound the k_eff-th coefficient as well, and
+                // tightly where the row maxima do not (a tile with a few active columns: its rows all look
+                // alike).  Taken from the stashed tile, only on this path; the candidates are then listed
+                // again under the larger of the two bounds.
+                bool over = false;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) over = over || (n_w[w] > (unsigned)WCAPW);
+                if (over && n_all >= (unsigned)k_eff) {
+                    unsigned ck = 0u;
+#pragma unroll 8
+                    for (int u = 0; u < S; ++u) ck = max(ck, mag_key(X[u * XS + t]));
+                    unsigned *tk = reinterpret_cast<unsigned *>(tmax);
+                    tk[t] = ck;
+                    sb.sync();
+                    const unsigned ok2 = tk[t ^ 32];
+                    const unsigned lo2 = __reduce_min_sync(0xffffffffu, min(ck, ok2));
+                    const unsigned hi2 = __reduce_max_sync(0xffffffffu, max(ck, ok2));
+                    const int c0 = 31 - __clz((lo2 ^ hi2) | 0x8000u);
+                    unsigned l2 = lo2 & ~((2u << c0) - 1u);
+#pragma unroll 1
+                    for (int b = c0; b >= 15; --b) {
+                        const unsigned cand = l2 | (1u << b);
+                        const unsigned cnt = __popc(__ballot_sync(0xffffffffu, ck >= cand)) +
+                                             __popc(__ballot_sync(0xffffffffu, ok2 >= cand));
+                        l2 = (cnt >= (unsigned)k_eff) ? cand : l2;
+                    }
+                    if (l2 > lmin_w) {  // slot-uniform
+                        lmin_w = l2;
+                        unsigned long long mask = 0ull;
+#pragma unroll 4
+                        for (int v = 0; v < S; ++v) mask |= (unsigned long long)(mag_key(X[t * XS + v]) >= l2) << v;
+                        mlo = (unsigned)mask;
+                        mhi = (unsigned)(mask >> 32);
+                        const unsigned cnt = __popc(mlo) + __popc(mhi);
+                        const unsigned inc = warp_inclusive_scan(cnt, lane);
+                        off = inc - cnt;
+                        n_cw = __shfl_sync(0xffffffffu, inc, 31);
+                        if (lane == 0) misc[warp] = n_cw;
+                        sb.sync();
+                        n_all = 0;
+#pragma unroll
+                        for (int w = 0; w < NW; ++w) {
+                            n_w[w] = misc[w];
+                            n_all += n_w[w];
+                        }
+                    }
+                }
+            }
+            if (use_fallback && n_all >= (unsigned)k_eff) {
+                wide = true;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) wide = wide && (n_w[w] <= (unsigned)WCAPW);
+                use_fallback = !wide;
+            }
+            if (wide) {
+                unsigned *wkey = reinterpret_cast<unsigned *>(smem_raw + (size_t)S * XS * sizeof(float));  // [NW][WCAPWP]
+                unsigned *widx = wkey + NW * WCAPWP;
+                {
+                    unsigned o = warp * WCAPWP + off;
+                    unsigned long long mask = ((unsigned long long)mhi << 32) | mlo;
+                    while (mask) {
+                        const int v = __ffsll((long long)mask) - 1;
+                        mask &= mask - 1ull;
+                        widx[o] = t * S + v;
+                        wkey[o] = mag_key(X[t * XS + v]);
+                        ++o;
+                    }
+                }
+                sb.sync();
+                // Every warp takes all candidate keys of the chunk into registers (list order = index order:
+                // warp 0's list, then warp 1's) and finds the k_eff-th largest by the same bit-by-bit ballot
+                // search as above -- no exchange between the warps is needed.
+                constexpr int WK = NW * WITER;
+                unsigned keys[WK];
+                unsigned hi = 0u;
+#pragma unroll
+                for (int j = 0; j < WK; ++j) {
+                    const int w = j / WITER;
+                    const unsigned i = (unsigned)(j % WITER) * 32u + lane;
+                    keys[j] = (i < n_w[w]) ? wkey[w * WCAPWP + i] : 0u;  // absent entries: 0, below every candidate
+                    hi = max(hi, keys[j]);
+                }
+                hi = __reduce_max_sync(0xffffffffu, hi);
+                // all candidates are >= lmin_w (> 0 here): the bits above the first one where lmin_w and the
+                // largest key differ are settled
+                const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
+                unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+#pragma unroll 1
+                for (int b = wb0; b >= 0; --b) {
+                    const unsigned cand = thr | (1u << b);
+                    unsigned cnt = 0;
+#pragma unroll
+                    for (int j = 0; j < WK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+                    thr = (cnt >= (unsigned)k_eff) ? cand : thr;
+                }
+                unsigned n_gt = 0;
+#pragma unroll
+                for (int j = 0; j < WK; ++j) n_gt += __popc(__ballot_sync(0xffffffffu, keys[j] > thr));
+                const unsigned need_eq = (unsigned)k_eff - n_gt;  // >= 1: ties at thr go to the lowest indices
+                unsigned gt_before = 0, eq_before = 0;
+                const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+                for (int j = 0; j < WK; ++j) {
+                    const unsigned key = keys[j];
+                    const unsigned gtb = __ballot_sync(0xffffffffu, key > thr);
+                    const unsigned eqb = __ballot_sync(0xffffffffu, key == thr);
+                    if (j / WITER == warp) {  // this warp's own list: it writes these records
+                        const unsigned e = eq_before + __popc(eqb & lt);
+                        const bool s = (key > thr) || (key == thr && e < need_eq);
+                        if (s) {
+                            const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
+                            DemoRecord r;
+                            r.idx = (int)widx[warp * WCAPWP + (j % WITER) * 32 + lane];
+                            const int v = r.idx & (S - 1);
+                            const int uo = (r.idx >> LOG2S) * XS;
+                            r.val = X[uo + v];
+                            rec[pos] = r;
+                            recs4[pos] = make_int4(uo, v * S, __float_as_int(a.alpha * r.val), 0);
+                            if ((int)pos == k_eff - 1)
+                                for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(uo, 0, 0, 0);
+                        }
+                    }
+                    gt_before += __popc(gtb);
+                    eq_before += __popc(eqb);
+                }
+            } else if (!use_fallback) {
                 // rank among all candidates by magnitude only.  If exactly k_eff candidates have
                 // fewer than k_eff larger ones, no tie straddles the threshold and that set is the
                 // answer; otherwise the count is redone with the index tie-break.

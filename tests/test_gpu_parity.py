@@ -631,3 +631,30 @@ def test_untouched_tiles_among_ordinary_ones(s, basis):
     rec = parity.gather_records(r.payloads[0], first, k_eff, np.arange(4, 12, dtype=np.int64))
     assert np.array_equal(rec["idx"], np.tile(np.arange(k_eff, dtype=np.int32), (8, 1))) and np.all(rec["val"] == 0)
     r.close()
+
+
+@pytest.mark.parametrize("s", [32, 64, 128])
+@pytest.mark.parametrize("pattern", ["rows", "cols"])
+def test_tiles_of_low_rank(s, pattern):
+    """Gradient tiles with one to three active rows (embedding gradients: only the tokens of the batch have a
+    row) or columns (output layer): the row maxima bound the k-th coefficient loosely there, the candidate
+    lists run long, and the kernels' wide-list / radix paths decide.  Every chunk against the oracle."""
+    shape = (6 * s, 5 * s)
+    wl = inputs.Workload("low-rank", [shape], chunk=s, topk=min(32, s), num_workers=2, grad_kind="normal", grad_std=1e-3)
+    r = parity.Runner(wl, max_chunks=10**9)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    for step in range(2):
+        grads = []
+        for w in range(2):
+            g = torch.zeros(shape, device="cuda")
+            for b in range(shape[0] // s if pattern == "rows" else shape[1] // s):
+                n_act = 1 + (b + w + step) % 3
+                idx = torch.randperm(s, generator=gen, device="cuda")[:n_act] + b * s
+                if pattern == "rows":
+                    g[idx] = torch.randn((n_act, shape[1]), generator=gen, device="cuda") * 1e-3
+                else:
+                    g[:, idx] = torch.randn((shape[0], n_act), generator=gen, device="cuda") * 1e-3
+            grads.append([g.to(torch.bfloat16)])
+        r.step(grads=grads)
+    r.close()
