@@ -210,7 +210,10 @@ def run_ours(args, rank, world):
     P0 = wl.n_params
     params = inputs.make_params(wl, dev)
     mom = [inputs.make_momentum(wl, dev) for _ in range(W)]
-    grads = [inputs.GradStream(wl, w, dev).next() for w in range(W)]  # one seeded set per worker, reused
+    streams = [inputs.GradStream(wl, w, dev) for w in range(W)]
+    for st in streams:  # ablation: row-sparse embedding gradients
+        st.embedding_active_rows = args.embedding_active_rows or None
+    grads = [st.next() for st in streams]  # one seeded set per worker, reused
     payloads = [torch.empty(tr.payload_bytes, dtype=torch.uint8, device=dev) for _ in range(W)]
     torch.cuda.synchronize()
 
@@ -337,7 +340,8 @@ def run_ours(args, rank, world):
                        "worker_params_per_s": value * W, "l2": ("inputs (%.1f GB resident in HBM) are larger than the 126 MB L2; no flush needed" % (working_set / 1e9))
                        if flush is None else ("working set %.1f MB: L2 flushed by a 256 MB write before every timed step"
                                               % (working_set / 1e6)), "kernel_path": args.path,
-                       "basis": args.basis, "chunk_shape": args.chunk_shape or None},
+                       "basis": args.basis, "chunk_shape": args.chunk_shape or None,
+                       "embedding_active_rows": args.embedding_active_rows or None},
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
         }
         if base is not None:
@@ -456,6 +460,8 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "generic"])
     ap.add_argument("--chunk", type=int, default=0, help="override the workload's chunk size (ablation)")
     ap.add_argument("--topk", type=int, default=0, help="override the workload's k (ablation)")
+    ap.add_argument("--embedding-active-rows", type=int, default=0,
+                    help="rows per chunk-row block of the embedding that get a gradient (ablation; 0 = all)")
     ap.add_argument("--chunk-shape", default="", help="AxB: rectangular chunks through the N-D kernels (ablation)")
     ap.add_argument("--basis", default="dct", choices=["dct", "identity", "random"],
                     help="transform basis; anything but dct takes the dense-transform kernels (not the headline)")

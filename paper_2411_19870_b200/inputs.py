@@ -124,6 +124,7 @@ PARAM_SEED = 10_000
 TENSOR_SCALE_SEED = 20_000
 TIE_MASK_SEED = 30_000
 ROW_FACTOR_SEED = 1
+ROW_MASK_SEED = 40_000
 
 
 def _gen(device, seed: int) -> torch.Generator:
@@ -167,6 +168,10 @@ class GradStream:
                                 for shp in wl.shapes]
         self.tie_gen = _gen(device, TIE_MASK_SEED + worker) if wl.grad_kind == "student_t_ties" else None
         self.tie_fraction = 0.05  # share of chunks replaced by tie-makers (student_t_ties)
+        # Ablation: rows of the tensor named "embedding" that receive a gradient, per block of `chunk` rows
+        # (only the tokens of a batch have a row); None = every row, the default of all configurations.
+        self.embedding_active_rows = None
+        self.row_gen = _gen(device, ROW_MASK_SEED + worker)
 
     def _draw(self, t: int, shp: Shape) -> torch.Tensor:
         wl = self.wl
@@ -208,8 +213,23 @@ class GradStream:
             return out.permute(0, 2, 1, 3).reshape(shp)
         return out.reshape(shp)
 
+    def _mask_rows(self, g: torch.Tensor) -> torch.Tensor:
+        """Keep `embedding_active_rows` seeded random rows in every block of `chunk` rows, zero the others."""
+        s, r = self.wl.chunk, int(self.embedding_active_rows)
+        blocks = g.shape[0] // s
+        order = torch.rand((blocks, s), generator=self.row_gen, device=self.device).argsort(dim=1)
+        keep = (order < r).reshape(-1, 1)
+        return torch.where(keep, g, torch.zeros_like(g))
+
     def next(self) -> List[torch.Tensor]:
-        return [self._draw(t, shp).to(self.wl.grad_dtype) for t, shp in enumerate(self.wl.shapes)]
+        out = []
+        for t, shp in enumerate(self.wl.shapes):
+            g = self._draw(t, shp)
+            if self.embedding_active_rows is not None and t < len(self.wl.tensor_names) and \
+                    self.wl.tensor_names[t] == "embedding":
+                g = self._mask_rows(g)
+            out.append(g.to(self.wl.grad_dtype))
+        return out
 
 
 def random_tensor(shape: Shape, seed: int, std: float, dtype: torch.dtype, device) -> torch.Tensor:
