@@ -18,6 +18,8 @@
 // Every wait on an mbarrier is bounded: on expiry the CTA records DEMO_DEV_TIMEOUT and returns.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "demo_internal.h"
 #include "fast_common.cuh"
 #include "fast_dct.cuh"
@@ -61,11 +63,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
     constexpr int CAPW = CAP / NW;        // candidate capacity of one warp's list
     constexpr int CAPWP = CAPW + 4;       // list stride (padding for 128-bit key loads)
     constexpr int ITER = CAPW / 32;
-    constexpr int WCAPW = (S == 64) ? 256 : 160;  // capacity of one warp's wide list (tiles of low rank)
-    constexpr int WCAPWP = WCAPW + 4;
-    constexpr int WITER = WCAPW / 32;
-    static_assert(compress_region_bytes<S, GT>() >= (size_t)S * XS * sizeof(float) + (size_t)NW * WCAPWP * 8,
-                  "the wide candidate lists live behind the coefficient tile");
+    // wide candidate list (tiles of low rank or with a concentrated spectrum): one list per chunk in the part
+    // of the staging area that the coefficient tile does not cover, 8 bytes per entry
+    constexpr int WCAP_ROOM = (int)((compress_region_bytes<S, GT>() - (size_t)S * XS * sizeof(float)) / 8) - 4;
+    constexpr int WCAP = WCAP_ROOM < 512 ? 128 : 512;
+    static_assert(WCAP_ROOM >= 128, "the wide candidate list needs room behind the coefficient tile");
 
     extern __shared__ __align__(128) unsigned char smem_all[];
     const int slot = threadIdx.x / S;
@@ -363,10 +365,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                 // tightly where the row maxima do not (a tile with a few active columns: its rows all look
                 // alike).  Taken from the stashed tile, only on this path; the candidates are then listed
                 // again under the larger of the two bounds.
-                bool over = false;
-#pragma unroll
-                for (int w = 0; w < NW; ++w) over = over || (n_w[w] > (unsigned)WCAPW);
-                if (over && n_all >= (unsigned)k_eff) {
+                if (n_all > (unsigned)WCAP) {
                     unsigned ck = 0u;
 #pragma unroll 8
                     for (int u = 0; u < S; ++u) ck = max(ck, mag_key(X[u * XS + t]));
@@ -407,17 +406,16 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                     }
                 }
             }
-            if (use_fallback && n_all >= (unsigned)k_eff) {
+            if (use_fallback && n_all >= (unsigned)k_eff && n_all <= (unsigned)WCAP) {
                 wide = true;
-#pragma unroll
-                for (int w = 0; w < NW; ++w) wide = wide && (n_w[w] <= (unsigned)WCAPW);
-                use_fallback = !wide;
+                use_fallback = false;
             }
             if (wide) {
-                unsigned *wkey = reinterpret_cast<unsigned *>(smem_raw + (size_t)S * XS * sizeof(float));  // [NW][WCAPWP]
-                unsigned *widx = wkey + NW * WCAPWP;
+                unsigned *wkey = reinterpret_cast<unsigned *>(smem_raw + (size_t)S * XS * sizeof(float));  // [WCAP + 4]
+                unsigned *widx = wkey + WCAP + 4;
                 {
-                    unsigned o = warp * WCAPWP + off;
+                    // one list in index order: the rows of warp 0, then the rows of warp 1
+                    unsigned o = ((NW > 1 && warp == 1) ? n_w[0] : 0u) + off;
                     unsigned long long mask = ((unsigned long long)mhi << 32) | mlo;
                     while (mask) {
                         const int v = __ffsll((long long)mask) - 1;
@@ -428,62 +426,68 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                     }
                 }
                 sb.sync();
-                // Every warp takes all candidate keys of the chunk into registers (list order = index order:
-                // warp 0's list, then warp 1's) and finds the k_eff-th largest by the same bit-by-bit ballot
-                // search as above -- no exchange between the warps is needed.
-                constexpr int WK = NW * WITER;
-                unsigned keys[WK];
-                unsigned hi = 0u;
+                // Every warp takes the whole list into registers (WK keys per lane) and finds the k_eff-th
+                // largest key by the same bit-by-bit ballot search as for the bound -- no exchange between the
+                // warps.  Entries above it are kept, entries equal to it in index order until k_eff are
+                // reached; the record position of a kept entry is the number of kept entries before it.  Every
+                // warp forms the running counts over the whole list and writes the groups that are its own.
+                auto wide_select = [&](auto wk_tag) {
+                    constexpr int WK = decltype(wk_tag)::value;
+                    unsigned keys[WK];
+                    unsigned hi = 0u;
 #pragma unroll
-                for (int j = 0; j < WK; ++j) {
-                    const int w = j / WITER;
-                    const unsigned i = (unsigned)(j % WITER) * 32u + lane;
-                    keys[j] = (i < n_w[w]) ? wkey[w * WCAPWP + i] : 0u;  // absent entries: 0, below every candidate
-                    hi = max(hi, keys[j]);
-                }
-                hi = __reduce_max_sync(0xffffffffu, hi);
-                // all candidates are >= lmin_w (> 0 here): the bits above the first one where lmin_w and the
-                // largest key differ are settled
-                const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
-                unsigned thr = lmin_w & ~((2u << wb0) - 1u);
-#pragma unroll 1
-                for (int b = wb0; b >= 0; --b) {
-                    const unsigned cand = thr | (1u << b);
-                    unsigned cnt = 0;
-#pragma unroll
-                    for (int j = 0; j < WK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
-                    thr = (cnt >= (unsigned)k_eff) ? cand : thr;
-                }
-                unsigned n_gt = 0;
-#pragma unroll
-                for (int j = 0; j < WK; ++j) n_gt += __popc(__ballot_sync(0xffffffffu, keys[j] > thr));
-                const unsigned need_eq = (unsigned)k_eff - n_gt;  // >= 1: ties at thr go to the lowest indices
-                unsigned gt_before = 0, eq_before = 0;
-                const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-                for (int j = 0; j < WK; ++j) {
-                    const unsigned key = keys[j];
-                    const unsigned gtb = __ballot_sync(0xffffffffu, key > thr);
-                    const unsigned eqb = __ballot_sync(0xffffffffu, key == thr);
-                    if (j / WITER == warp) {  // this warp's own list: it writes these records
-                        const unsigned e = eq_before + __popc(eqb & lt);
-                        const bool s = (key > thr) || (key == thr && e < need_eq);
-                        if (s) {
-                            const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
-                            DemoRecord r;
-                            r.idx = (int)widx[warp * WCAPWP + (j % WITER) * 32 + lane];
-                            const int v = r.idx & (S - 1);
-                            const int uo = (r.idx >> LOG2S) * XS;
-                            r.val = X[uo + v];
-                            rec[pos] = r;
-                            recs4[pos] = make_int4(uo, v * S, __float_as_int(a.alpha * r.val), 0);
-                            if ((int)pos == k_eff - 1)
-                                for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(uo, 0, 0, 0);
-                        }
+                    for (int j = 0; j < WK; ++j) {
+                        const unsigned i = (unsigned)j * 32u + lane;
+                        keys[j] = (i < n_all) ? wkey[i] : 0u;  // absent entries: 0, below every candidate
+                        hi = max(hi, keys[j]);
                     }
-                    gt_before += __popc(gtb);
-                    eq_before += __popc(eqb);
-                }
+                    hi = __reduce_max_sync(0xffffffffu, hi);
+                    // every entry is >= lmin_w (> 0 here): the bits above the first one where lmin_w and the
+                    // largest key differ are settled
+                    const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
+                    unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+#pragma unroll 1
+                    for (int b = wb0; b >= 0; --b) {
+                        const unsigned cand = thr | (1u << b);
+                        unsigned cnt = 0;
+#pragma unroll
+                        for (int j = 0; j < WK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+                        thr = (cnt >= (unsigned)k_eff) ? cand : thr;
+                    }
+                    unsigned n_gt = 0;
+#pragma unroll
+                    for (int j = 0; j < WK; ++j) n_gt += __popc(__ballot_sync(0xffffffffu, keys[j] > thr));
+                    const unsigned need_eq = (unsigned)k_eff - n_gt;  // >= 1
+                    unsigned gt_before = 0, eq_before = 0;
+                    const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+                    for (int j = 0; j < WK; ++j) {
+                        const unsigned key = keys[j];
+                        const unsigned gtb = __ballot_sync(0xffffffffu, key > thr);
+                        const unsigned eqb = __ballot_sync(0xffffffffu, key == thr);
+                        if ((j % NW) == warp) {
+                            const unsigned e = eq_before + __popc(eqb & lt);
+                            if ((key > thr) || (key == thr && e < need_eq)) {
+                                const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
+                                DemoRecord r;
+                                r.idx = (int)widx[j * 32 + lane];
+                                const int v = r.idx & (S - 1);
+                                const int uo = (r.idx >> LOG2S) * XS;
+                                r.val = X[uo + v];
+                                rec[pos] = r;
+                                recs4[pos] = make_int4(uo, v * S, __float_as_int(a.alpha * r.val), 0);
+                                if ((int)pos == k_eff - 1)
+                                    for (int pp = k_eff; pp < ((k_eff + 7) & ~7); ++pp) recs4[pp] = make_int4(uo, 0, 0, 0);
+                            }
+                        }
+                        gt_before += __popc(gtb);
+                        eq_before += __popc(eqb);
+                    }
+                };
+                if (WCAP <= 128 || n_all <= 128u)
+                    wide_select(std::integral_constant<int, 4>{});
+                else
+                    wide_select(std::integral_constant<int, WCAP / 32>{});
             } else if (!use_fallback) {
                 // rank among all candidates by magnitude only.  If exactly k_eff candidates have
                 // fewer than k_eff larger ones, no tie straddles the threshold and that set is the
