@@ -64,15 +64,17 @@ def broadcast_signs(flat: torch.Tensor, server: int, group=None) -> None:
 
 
 class DistributedDemo:
-    """DeMo step with one worker per rank of ``group``.  ``shapes`` etc. as for ``DemoTransform``."""
+    """DeMo step with one worker per rank of ``group``.  ``shapes`` etc. as for ``DemoTransform``
+    (``chunk_shapes``: tensors of any order with rectangular chunks)."""
 
-    def __init__(self, shapes, *, chunk: int, topk: int, beta: float, lr: float, weight_decay: float,
-                 grad_dtype: int = DEMO_BF16, device: int = 0, group=None):
+    def __init__(self, shapes, *, chunk: int = 0, topk: int, beta: float, lr: float, weight_decay: float,
+                 grad_dtype: int = DEMO_BF16, device: int = 0, group=None, chunk_shapes=None):
         self.group = group
         self.rank = dist.get_rank(group)
         self.world = dist.get_world_size(group)
         self.tr = DemoTransform(shapes, chunk=chunk, topk=topk, beta=beta, lr=lr, weight_decay=weight_decay,
-                                num_workers=self.world, grad_dtype=grad_dtype, device=device)
+                                num_workers=self.world, grad_dtype=grad_dtype, device=device,
+                                chunk_shapes=chunk_shapes)
         pb = self.tr.payload_bytes
         self.buffer = torch.zeros(self.world * pb, dtype=torch.uint8, device=torch.device("cuda", device))
         self.slices = [self.buffer[w * pb:(w + 1) * pb] for w in range(self.world)]
