@@ -361,29 +361,69 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             // whole chunk through the radix select.
             bool wide = false;
             if constexpr (NW > 1) {
-                // Too many candidates: the maxima of the 64 COLUMNS bound the k_eff-th coefficient as well, and
-                // tightly where the row maxima do not (a tile with a few active columns: its rows all look
-                // alike).  Taken from the stashed tile, only on this path; the candidates are then listed
-                // again under the larger of the two bounds.
+                // Too many candidates even for the wide list: a finer partition bounds the k_eff-th coefficient
+                // more tightly -- the maxima of the 256 quarter rows and of the 256 quarter columns (a tile with
+                // a few active columns has rows that all look alike, and the other way round).  Taken from the
+                // stashed tile, only on this path; the candidates are then listed again under the largest bound.
                 if (n_all > (unsigned)WCAP) {
-                    unsigned ck = 0u;
-#pragma unroll 8
-                    for (int u = 0; u < S; ++u) ck = max(ck, mag_key(X[u * XS + t]));
-                    unsigned *tk = reinterpret_cast<unsigned *>(tmax);
-                    tk[t] = ck;
-                    sb.sync();
-                    const unsigned ok2 = tk[t ^ 32];
-                    const unsigned lo2 = __reduce_min_sync(0xffffffffu, min(ck, ok2));
-                    const unsigned hi2 = __reduce_max_sync(0xffffffffu, max(ck, ok2));
-                    const int c0 = 31 - __clz((lo2 ^ hi2) | 0x8000u);
-                    unsigned l2 = lo2 & ~((2u << c0) - 1u);
-#pragma unroll 1
-                    for (int b = c0; b >= 15; --b) {
-                        const unsigned cand = l2 | (1u << b);
-                        const unsigned cnt = __popc(__ballot_sync(0xffffffffu, ck >= cand)) +
-                                             __popc(__ballot_sync(0xffffffffu, ok2 >= cand));
-                        l2 = (cnt >= (unsigned)k_eff) ? cand : l2;
+                    unsigned rk[4], ck[4];
+                    const float4 *row4 = reinterpret_cast<const float4 *>(X + t * XS);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        unsigned m = 0u;
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            const float4 f = row4[4 * g + v4];
+                            m = max(max(m, mag_key(f.x)), max(mag_key(f.y), max(mag_key(f.z), mag_key(f.w))));
+                        }
+                        rk[g] = m;
                     }
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        unsigned m = 0u;
+#pragma unroll 4
+                        for (int u = 0; u < 16; ++u) m = max(m, mag_key(X[(16 * g + u) * XS + t]));
+                        ck[g] = m;
+                    }
+                    // every warp needs all 512 maxima: its own and, through shared memory, the partner warp's
+                    unsigned *gq = reinterpret_cast<unsigned *>(smem_raw + (size_t)S * XS * sizeof(float));  // [8][64]
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        gq[g * 64 + t] = rk[g];
+                        gq[(4 + g) * 64 + t] = ck[g];
+                    }
+                    sb.sync();
+                    unsigned prk[4], pck[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        prk[g] = gq[g * 64 + (t ^ 32)];
+                        pck[g] = gq[(4 + g) * 64 + (t ^ 32)];
+                    }
+                    // the k_eff-th largest of 256 keys (four of this thread, four of its partner), low 15 bits zero
+                    auto kth_of_256 = [&](const unsigned (&own)[4], const unsigned (&oth)[4]) -> unsigned {
+                        unsigned lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            lo = min(lo, min(own[g], oth[g]));
+                            hi = max(hi, max(own[g], oth[g]));
+                        }
+                        lo = __reduce_min_sync(0xffffffffu, lo);
+                        hi = __reduce_max_sync(0xffffffffu, hi);
+                        const int c0 = 31 - __clz((lo ^ hi) | 0x8000u);
+                        unsigned pre = lo & ~((2u << c0) - 1u);
+#pragma unroll 1
+                        for (int b = c0; b >= 15; --b) {
+                            const unsigned cand = pre | (1u << b);
+                            unsigned cnt = 0;
+#pragma unroll
+                            for (int g = 0; g < 4; ++g)
+                                cnt += __popc(__ballot_sync(0xffffffffu, own[g] >= cand)) +
+                                       __popc(__ballot_sync(0xffffffffu, oth[g] >= cand));
+                            pre = (cnt >= (unsigned)k_eff) ? cand : pre;
+                        }
+                        return pre;
+                    };
+                    const unsigned l2 = max(kth_of_256(rk, prk), kth_of_256(ck, pck));
                     if (l2 > lmin_w) {  // slot-uniform
                         lmin_w = l2;
                         unsigned long long mask = 0ull;
