@@ -71,6 +71,8 @@ cudaError_t demo_launch_decode_generic(int s, int two_d, const DemoDecodeArgs &a
 bool demo_fast_supported(int s);
 cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
 cudaError_t demo_launch_decode_fast(int s, const DemoDecodeArgs &a, int sm_count, cudaStream_t stream);
+// s = 64 with TMA tensor maps (kernels_fast64.cu; cudaErrorNotSupported without them).
+cudaError_t demo_launch_compress_fast64(const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
 // s = 128 (kernels_fast128.cu); need the TMA tensor maps (cudaErrorNotSupported without them).
 cudaError_t demo_launch_compress_fast128(const DemoCompressArgs &a, int sm_count, cudaStream_t stream);
 cudaError_t demo_launch_decode_fast128(const DemoDecodeArgs &a, int sm_count, cudaStream_t stream);

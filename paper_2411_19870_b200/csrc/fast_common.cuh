@@ -64,6 +64,23 @@ __device__ __forceinline__ void tma_prefetch_2d(const void *tmap, int x, int y)
 {
     asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
 }
+// 2-D tiled TMA store of one box from shared memory (bulk-group completion).
+__device__ __forceinline__ void tma_store_2d(const void *tmap, int x, int y, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(tmap), "r"(x), "r"(y),
+                 "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits (the issuing thread's own bulk groups; completes by itself): source read out / fully done.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// The tensor maps live in global memory and are rewritten by the host (a stream-ordered copy) when the
+// caller's buffers change: the thread that is about to use one acquires it for the tensor-map proxy first.
+__device__ __forceinline__ void tmap_acquire(const void *tmap)
+{
+    asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(tmap) : "memory");
+}
 constexpr int TMAP_BYTES = 128;  // sizeof(CUtensorMap)
 
 __device__ __forceinline__ float to_f32(float v) { return v; }

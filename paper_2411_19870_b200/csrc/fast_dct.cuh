@@ -183,4 +183,92 @@ FDCT_HD void dct3_ortho(float (&X)[N])
     static_for<0, N>([&](auto i) { X[decltype(i)::value] = x[decltype(i)::value]; });
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same two transforms split so that the forward and the inverse share ONE copy of their
+// multiplications.  DCT-II_N is a cascade of butterflies (sums go down, differences are the inputs of
+// DCT-IV_{N/2}, DCT-IV_{N/4}, ..., DCT-IV_1) and DCT-III_N is the same DCT-IV blocks followed by the
+// transposed cascade, so both are  [butterflies] o core  /  core o [butterflies]  with
+//   core:  y[0] = dc * w[0],  y[H .. 2H) = DCT-IV_H(w[H .. 2H))  for H = 1, 2, 4, ..., N/2.
+// Position p of w / y corresponds to coefficient core_index<N>(p).  A kernel that runs the core inside
+// a rolled loop over its passes keeps a single copy of the (fully unrolled) DCT-IV code.
+// ------------------------------------------------------------------------------------------------
+template <int N>
+constexpr int core_index(int p)
+{
+    if (p == 0) return 0;
+    int h = 1;
+    while (2 * h <= p) h *= 2;
+    return (N / h) * (p - h) + N / (2 * h);
+}
+// inverse map: position of coefficient v
+template <int N>
+constexpr int core_pos(int v)
+{
+    for (int p = 0; p < N; ++p)
+        if (core_index<N>(p) == v) return p;
+    return -1;
+}
+
+template <int H, int N, class SC>
+FDCT_HD void core_blocks(const float (&w)[N], float (&y)[N])
+{
+    float v[H], V[H];
+    static_for<0, H>([&](auto i) { v[decltype(i)::value] = w[H + decltype(i)::value]; });
+    dct4<H, SC>(v, V);
+    static_for<0, H>([&](auto i) { y[H + decltype(i)::value] = V[decltype(i)::value]; });
+    if constexpr (H > 1) core_blocks<H / 2, N, SC>(w, y);
+}
+template <int N>
+FDCT_HD void dct_core_ortho(const float (&w)[N], float (&y)[N])
+{
+    y[0] = w[0] * dc_scale<N>();
+    core_blocks<N / 2, N, ScaleOrtho<N>>(w, y);
+}
+
+// Forward butterflies: natural-order input x -> core input w.
+template <int L, int N>
+FDCT_HD void fwd_cascade(const float (&u)[L], float (&w)[N])
+{
+    if constexpr (L == 1) {
+        w[0] = u[0];
+    } else {
+        constexpr int H = L / 2;
+        float s[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            s[n] = u[n] + u[L - 1 - n];
+            w[H + n] = u[n] - u[L - 1 - n];
+        });
+        fwd_cascade<H, N>(s, w);
+    }
+}
+template <int N>
+FDCT_HD void dct2_pre(const float (&x)[N], float (&w)[N])
+{
+    fwd_cascade<N, N>(x, w);
+}
+
+// Inverse butterflies: core output y -> natural-order output x.
+template <int H, int N>
+FDCT_HD void inv_cascade(const float (&e)[H], const float (&y)[N], float (&x)[N])
+{
+    if constexpr (H == N) {
+        static_for<0, N>([&](auto i) { x[decltype(i)::value] = e[decltype(i)::value]; });
+    } else {
+        float f[2 * H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            f[n] = e[n] + y[H + n];
+            f[2 * H - 1 - n] = e[n] - y[H + n];
+        });
+        inv_cascade<2 * H, N>(f, y, x);
+    }
+}
+template <int N>
+FDCT_HD void dct3_post(const float (&y)[N], float (&x)[N])
+{
+    float e[1] = {y[0]};
+    inv_cascade<1, N>(e, y, x);
+}
+
 }  // namespace fdct

@@ -998,9 +998,13 @@ bool demo_fast_supported(int s) { return s == 128 || s == 64 || s == 32; }
 cudaError_t demo_launch_compress_fast(int s, const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
 {
     if (s == 128) return demo_launch_compress_fast128(a, sm_count, stream);
-    if (s == 64)
+    if (s == 64) {
+#ifndef DEMO_OLD64
+        if (a.tmap_m != nullptr && a.tmap_g != nullptr) return demo_launch_compress_fast64(a, sm_count, stream);
+#endif
         return a.grad_bf16 ? launch_compress<64, __nv_bfloat16>(a, sm_count, stream)
                            : launch_compress<64, float>(a, sm_count, stream);
+    }
     if (s == 32)
         return a.grad_bf16 ? launch_compress<32, __nv_bfloat16>(a, sm_count, stream)
                            : launch_compress<32, float>(a, sm_count, stream);

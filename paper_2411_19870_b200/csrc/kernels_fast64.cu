@@ -1,0 +1,773 @@
+// Compress kernel for 2-D tensors with chunk size 64 (the paper's main configuration): Algorithm 1 worker
+// side / CompressChunks, fused per chunk -- momentum update, 2-D DCT-II, exact top-k, momentum
+// subtraction.  64 threads (a "slot") own one 64 x 64 chunk; thread t works on column t, then row t.
+//
+// What shapes this kernel is its instruction footprint.  A register-resident 64-point transform is
+// ~10 KB of straight-line code; three copies (two forward passes, one inverse) plus fully unrolled
+// tile reads do not fit the SM's instruction cache, and warps that sit at different places of such
+// a stream starve on instruction fetch.  Here the hot loop is kept near 30 KB so that every slot can
+// run on its own, and the phases of different chunks (tile wait, transform, selection, store burst)
+// overlap on the SM's pipes instead of following one another:
+//   * the three transform passes of a chunk go through ONE copy of the multiplications (the DCT-IV blocks
+//     that DCT-II and DCT-III share, fast_dct.cuh) inside a rolled loop; only the butterfly cascades differ;
+//   * B = beta*m + g is parked in tensor memory (one tcgen05.st of the thread's column) and read back for
+//     the residual, instead of fetching and recombining the two tiles a second time;
+//   * the next chunk's tiles are requested as soon as the transpose tile is dead, so they land behind
+//     the inverse transform and the store burst of the current chunk;
+//   * everything rare (tied or degenerate chunks, tiles of low rank, k > 64) lives in one out-of-line
+//     routine that works from the coefficient tile in shared memory.
+// Every wait on an mbarrier is bounded: on expiry the slot records DEMO_DEV_TIMEOUT and stops.
+#include <cuda_bf16.h>
+
+#include <type_traits>
+
+#include "demo_internal.h"
+#include "fast_common.cuh"
+#include "fast_dct.cuh"
+
+namespace {
+
+using namespace fastk;
+
+constexpr int S = 64;
+constexpr int XS = S + 4;     // row stride of the transpose tile: conflict-free column access, 128-bit row access
+constexpr int LOG2S = 6;
+constexpr int CAP = 128;      // candidate capacity of the fast top-k (two lists of 64)
+constexpr int CAPW = CAP / 2;
+constexpr int CAPWP = CAPW + 4;
+constexpr int WCAP = 512;     // capacity of the wide candidate list (out-of-line path)
+constexpr int TMEM_COLS_PER_GROUP = 64;  // one column block per four warps (two slots)
+constexpr int PAD_ROW = 0x40000000;      // row offset of the padding entries of the row-stage list (never stored to)
+
+template <typename GT>
+constexpr size_t region_bytes()
+{
+    constexpr size_t stage = (size_t)S * S * (sizeof(float) + sizeof(GT));
+    constexpr size_t need = (size_t)S * XS * sizeof(float) + (size_t)(WCAP + 4) * 8;  // tile + wide list
+    return stage > need ? stage : need;
+}
+template <typename GT>
+constexpr size_t slot_bytes()
+{
+    constexpr size_t raw = region_bytes<GT>() + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
+    return (raw + 127) / 128 * 128;
+}
+
+// Shared memory of one slot.
+struct SlotMem {
+    unsigned char *raw;
+    float *X;            // [S*XS] transpose / coefficient / row-stage tile (aliases the staged tiles)
+    float *tmax;         // [S]
+    int *cand_idx;       // [CAP + 8]
+    float *cand_val;     // [CAP + 8]
+    unsigned *cand_key;  // [CAP + 8]
+    unsigned *hist;      // [256] aliases the candidate arrays
+    int4 *recs4;         // [64] kept records, pre-decoded for the row stage
+    unsigned *misc;      // [16]
+    unsigned *wkey;      // [WCAP + 4] wide list, behind the tile
+    unsigned *widx;      // [WCAP + 4]
+};
+
+// 64 / 32 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st64(uint32_t taddr, const float (&v)[64])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, "
+        "%33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, "
+        "%49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64};" ::"r"(taddr),
+        "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]), "f"(v[9]),
+        "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]), "f"(v[18]),
+        "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]),
+        "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31]), "f"(v[32]), "f"(v[33]), "f"(v[34]), "f"(v[35]), "f"(v[36]),
+        "f"(v[37]), "f"(v[38]), "f"(v[39]), "f"(v[40]), "f"(v[41]), "f"(v[42]), "f"(v[43]), "f"(v[44]), "f"(v[45]),
+        "f"(v[46]), "f"(v[47]), "f"(v[48]), "f"(v[49]), "f"(v[50]), "f"(v[51]), "f"(v[52]), "f"(v[53]), "f"(v[54]),
+        "f"(v[55]), "f"(v[56]), "f"(v[57]), "f"(v[58]), "f"(v[59]), "f"(v[60]), "f"(v[61]), "f"(v[62]), "f"(v[63])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]),
+          "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]),
+          "=f"(v[17]), "=f"(v[18]), "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]),
+          "=f"(v[25]), "=f"(v[26]), "=f"(v[27]), "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Out-of-line selection for the chunks the in-line path does not take: more than 64 candidates in a
+// warp's list (tiles of low rank or with a concentrated spectrum, tied or degenerate chunks), fewer
+// candidates than k (NaN coefficients) or k > 64.  Works from the coefficient tile in X (row t is
+// this thread's), writes the records to `rec` and, for k <= 64, the pre-decoded list for the row stage.
+//   1. wide list: up to WCAP candidates under the bound `lmin` (the k-th largest of the 64 row maxima),
+//      every warp takes the whole list into registers and finds the exact k-th largest key by a
+//      bit-by-bit ballot search;
+//   2. if the list overflows: a tighter bound from the 256 quarter-row and the 256 quarter-column
+//      maxima, then 1. again;
+//   3. otherwise an exact 4 x 8-bit radix select over the whole tile.
+// ------------------------------------------------------------------------------------------------
+__device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord *rec, float alpha, int t, int bar_id,
+                                         unsigned lmin_w, bool bound_valid)
+{
+    const SlotBarrier<S> sb{bar_id};
+    const int lane = t & 31, warp = t >> 5;
+    float *X = sm.X;
+    unsigned *misc = sm.misc;
+    int4 *recs4 = sm.recs4;
+    sb.sync();  // the coefficient tile is complete; the in-line path is done with its lists
+
+    bool done = false;
+    if (bound_valid && k_eff <= S) {
+        unsigned long long mask = 0ull;
+        unsigned off = 0, n_all = 0;
+        auto count_under = [&](unsigned bound) {
+            mask = 0ull;
+#pragma unroll 4
+            for (int v = 0; v < S; ++v) mask |= (unsigned long long)(mag_key(X[t * XS + v]) >= bound) << v;
+            const unsigned cnt = (unsigned)__popcll(mask);
+            const unsigned inc = warp_inclusive_scan(cnt, lane);
+            sb.sync();  // earlier readers of misc are done
+            if (lane == 31) misc[warp] = inc;
+            sb.sync();
+            const unsigned n0 = misc[0];
+            n_all = n0 + misc[1];
+            off = inc - cnt + (warp ? n0 : 0u);
+        };
+        count_under(lmin_w);
+        if (n_all > (unsigned)WCAP) {
+            // tighter bound: the k_eff-th largest of the 256 quarter-row maxima and of the 256 quarter-column maxima
+            unsigned rk[4], ck[4];
+            const float4 *row4 = reinterpret_cast<const float4 *>(X + t * XS);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                unsigned m = 0u;
+#pragma unroll
+                for (int v4 = 0; v4 < 4; ++v4) {
+                    const float4 f = row4[4 * g + v4];
+                    m = max(max(m, mag_key(f.x)), max(mag_key(f.y), max(mag_key(f.z), mag_key(f.w))));
+                }
+                rk[g] = m;
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                unsigned m = 0u;
+#pragma unroll 4
+                for (int u = 0; u < 16; ++u) m = max(m, mag_key(X[(16 * g + u) * XS + t]));
+                ck[g] = m;
+            }
+            unsigned *gq = sm.wkey;  // [8][64], behind the tile
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                gq[g * 64 + t] = rk[g];
+                gq[(4 + g) * 64 + t] = ck[g];
+            }
+            sb.sync();
+            unsigned prk[4], pck[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                prk[g] = gq[g * 64 + (t ^ 32)];
+                pck[g] = gq[(4 + g) * 64 + (t ^ 32)];
+            }
+            auto kth_of_256 = [&](const unsigned (&own)[4], const unsigned (&oth)[4]) -> unsigned {
+                unsigned lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    lo = min(lo, min(own[g], oth[g]));
+                    hi = max(hi, max(own[g], oth[g]));
+                }
+                lo = __reduce_min_sync(0xffffffffu, lo);
+                hi = __reduce_max_sync(0xffffffffu, hi);
+                const int c0 = 31 - __clz((lo ^ hi) | 0x8000u);
+                unsigned pre = lo & ~((2u << c0) - 1u);
+#pragma unroll 1
+                for (int b = c0; b >= 15; --b) {
+                    const unsigned cand = pre | (1u << b);
+                    unsigned cnt = 0;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        cnt += __popc(__ballot_sync(0xffffffffu, own[g] >= cand)) +
+                               __popc(__ballot_sync(0xffffffffu, oth[g] >= cand));
+                    pre = (cnt >= (unsigned)k_eff) ? cand : pre;
+                }
+                return pre;
+            };
+            const unsigned l2 = max(kth_of_256(rk, prk), kth_of_256(ck, pck));
+            sb.sync();  // gq is read; the wide list may overwrite it
+            if (l2 > lmin_w) {
+                lmin_w = l2;
+                count_under(lmin_w);
+            }
+        }
+        if (n_all >= (unsigned)k_eff && n_all <= (unsigned)WCAP) {
+            unsigned *wkey = sm.wkey, *widx = sm.widx;
+            {
+                unsigned o = off;
+                while (mask) {
+                    const int v = __ffsll((long long)mask) - 1;
+                    mask &= mask - 1ull;
+                    widx[o] = t * S + v;
+                    wkey[o] = mag_key(X[t * XS + v]);
+                    ++o;
+                }
+            }
+            sb.sync();
+            auto wide_select = [&](auto wk_tag) {
+                constexpr int WK = decltype(wk_tag)::value;
+                unsigned keys[WK];
+                unsigned hi = 0u;
+#pragma unroll
+                for (int j = 0; j < WK; ++j) {
+                    const unsigned i = (unsigned)j * 32u + lane;
+                    keys[j] = (i < n_all) ? wkey[i] : 0u;
+                    hi = max(hi, keys[j]);
+                }
+                hi = __reduce_max_sync(0xffffffffu, hi);
+                const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
+                unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+#pragma unroll 1
+                for (int b = wb0; b >= 0; --b) {
+                    const unsigned cand = thr | (1u << b);
+                    unsigned cnt = 0;
+#pragma unroll
+                    for (int j = 0; j < WK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+                    thr = (cnt >= (unsigned)k_eff) ? cand : thr;
+                }
+                unsigned n_gt = 0;
+#pragma unroll
+                for (int j = 0; j < WK; ++j) n_gt += __popc(__ballot_sync(0xffffffffu, keys[j] > thr));
+                const unsigned need_eq = (unsigned)k_eff - n_gt;
+                unsigned gt_before = 0, eq_before = 0;
+                const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+                for (int j = 0; j < WK; ++j) {
+                    const unsigned key = keys[j];
+                    const unsigned gtb = __ballot_sync(0xffffffffu, key > thr);
+                    const unsigned eqb = __ballot_sync(0xffffffffu, key == thr);
+                    if ((j & 1) == warp) {
+                        const unsigned e = eq_before + __popc(eqb & lt);
+                        if ((key > thr) || (key == thr && e < need_eq)) {
+                            const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
+                            DemoRecord r;
+                            r.idx = (int)widx[j * 32 + lane];
+                            const int v = r.idx & (S - 1);
+                            const int uo = (r.idx >> LOG2S) * XS;
+                            r.val = X[uo + v];
+                            rec[pos] = r;
+                            recs4[pos] = make_int4(uo, v * S, __float_as_int(alpha * r.val), 0);
+                        }
+                    }
+                    gt_before += __popc(gtb);
+                    eq_before += __popc(eqb);
+                }
+            };
+            if (n_all <= 128u)
+                wide_select(std::integral_constant<int, 4>{});
+            else
+                wide_select(std::integral_constant<int, WCAP / 32>{});
+            done = true;
+        }
+    }
+    if (!done) {
+        unsigned thr, need_eq;
+        sb.sync();
+        radix_select_tile<S, XS>(X, k_eff, sm.hist, misc, &thr, &need_eq, t, sb);
+        unsigned gt = 0, eq = 0;
+#pragma unroll 1
+        for (int v = 0; v < S; ++v) {
+            const unsigned key = mag_key(X[t * XS + v]);
+            gt += key > thr;
+            eq += key == thr;
+        }
+        const unsigned packed = gt | (eq << 16);
+        const unsigned inc = warp_inclusive_scan(packed, lane);
+        sb.sync();  // radix_select_tile's last reads of misc are done
+        if (lane == 31) misc[warp] = inc;
+        sb.sync();
+        unsigned before = inc - packed;
+        if (warp == 1) before += misc[0];
+        unsigned gb = before & 0xffffu, eb = before >> 16;
+#pragma unroll 1
+        for (int v = 0; v < S; ++v) {
+            const float val = X[t * XS + v];
+            const unsigned key = mag_key(val);
+            bool s = false;
+            unsigned pos = 0;
+            if (key > thr) {
+                pos = gb + min(eb, need_eq);
+                ++gb;
+                s = true;
+            } else if (key == thr) {
+                if (eb < need_eq) {
+                    pos = gb + eb;
+                    s = true;
+                }
+                ++eb;
+            }
+            if (s) {
+                DemoRecord r;
+                r.idx = t * S + v;
+                r.val = val;
+                rec[pos] = r;
+                if (k_eff <= 64) {
+                    recs4[pos] = make_int4(t * XS, v * S, __float_as_int(alpha * val), 0);
+                }
+            }
+        }
+    }
+}
+
+template <typename GT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(DemoCompressArgs a)
+{
+    constexpr int NCH = THREADS / S;
+    constexpr int NGROUPS = (THREADS + 127) / 128;                   // groups of four warps
+    constexpr int TMEM_COLS = NGROUPS * TMEM_COLS_PER_GROUP < 32 ? 32 : NGROUPS * TMEM_COLS_PER_GROUP;
+    static_assert((TMEM_COLS & (TMEM_COLS - 1)) == 0, "tensor-memory allocations are powers of two");
+    constexpr unsigned TILE_BYTES = S * S * sizeof(float) + S * S * sizeof(GT);
+
+    extern __shared__ __align__(128) unsigned char smem_all[];
+    const int slot = threadIdx.x / S;
+    SlotMem sm;
+    sm.raw = smem_all + (size_t)slot * slot_bytes<GT>();
+    float *Ms = reinterpret_cast<float *>(sm.raw);   // [S*S] m tile
+    GT *Gs = reinterpret_cast<GT *>(Ms + S * S);     // [S*S] g tile
+    sm.X = Ms;
+    sm.wkey = reinterpret_cast<unsigned *>(sm.raw + (size_t)S * XS * sizeof(float));
+    sm.widx = sm.wkey + WCAP + 4;
+    sm.tmax = reinterpret_cast<float *>(sm.raw + region_bytes<GT>());
+    sm.cand_idx = reinterpret_cast<int *>(sm.tmax + S);
+    sm.cand_val = reinterpret_cast<float *>(sm.cand_idx + CAP + 8);
+    sm.cand_key = reinterpret_cast<unsigned *>(sm.cand_val + CAP + 8);
+    sm.hist = reinterpret_cast<unsigned *>(sm.cand_idx);
+    sm.recs4 = reinterpret_cast<int4 *>(sm.cand_key + CAP + 8);
+    sm.misc = reinterpret_cast<unsigned *>(sm.recs4 + 64);
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(sm.misc + 16);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_all + (size_t)NCH * slot_bytes<GT>());
+    float *X = sm.X;
+    float *tmax = sm.tmax;
+    int *cand_idx = sm.cand_idx;
+    float *cand_val = sm.cand_val;
+    unsigned *cand_key = sm.cand_key;
+    int4 *recs4 = sm.recs4;
+    unsigned *misc = sm.misc;
+
+    const int t = threadIdx.x % S, lane = t & 31, warp = t >> 5;
+    const int hw_warp = threadIdx.x >> 5;
+    const SlotBarrier<S> sb{slot + 1};
+    const uint32_t bar = smem_u32(bar_mem);
+
+    if (t == 0) {
+        mbar_init(bar, 1);
+        fence_proxy_async();
+    }
+    if (hw_warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    fence_proxy_async();
+    const uint32_t tmem_base = *tmem_slot;
+    // this thread's lane of tensor memory (a warp reaches the 32 lanes of its quadrant) and its slot's columns
+    const uint32_t taddr = tmem_base + ((uint32_t)((hw_warp & 3) * 32) << 16) + (uint32_t)((hw_warp >> 2) * TMEM_COLS_PER_GROUP);
+
+    EntryCursor cur;
+    int cached_tensor = -1;
+    unsigned phase = 0;
+
+    struct TileRef {
+        const char *tm_m, *tm_g;
+        int x, y;
+    };
+    auto locate = [&](long long c) {
+        cur.seek(a.entries, a.n_entries, c);
+        const unsigned lc = (unsigned)(c - cur.te.chunk_begin);
+        const unsigned k0 = lc / (unsigned)cur.te.c1;
+        const int k1 = (int)(lc - k0 * (unsigned)cur.te.c1);
+        TileRef r;
+        r.x = k1 * S;
+        r.y = (int)k0 * S;
+        r.tm_m = static_cast<const char *>(a.tmap_m) + (size_t)cur.te.tensor * TMAP_BYTES;
+        r.tm_g = static_cast<const char *>(a.tmap_g) + (size_t)cur.te.tensor * TMAP_BYTES;
+        if (cur.te.tensor != cached_tensor) {
+            cached_tensor = cur.te.tensor;
+            if (t == 0) {
+                tmap_acquire(r.tm_m);
+                tmap_acquire(r.tm_g);
+            }
+        }
+        return r;
+    };
+    auto issue_loads = [&](const TileRef &r) {
+        if (t == 0) {
+            mbar_expect_tx(bar, TILE_BYTES);
+            tma_load_2d(smem_u32(Ms), r.tm_m, r.x, r.y, bar);
+            tma_load_2d(smem_u32(Gs), r.tm_g, r.x, r.y, bar);
+        }
+    };
+
+    const long long stride = (long long)gridDim.x * NCH;
+    long long c = (long long)blockIdx.x * NCH + slot;
+    TileRef tile_cur, tile_next;
+    if (c < a.n_chunks) {
+        tile_next = locate(c);
+        issue_loads(tile_next);
+    }
+
+    for (; c < a.n_chunks; c += stride) {
+        // the cursor points at chunk c (its loads were issued last)
+        tile_cur = tile_next;
+        const int k_eff = cur.te.k_eff;
+        DemoRecord *rec = a.payload + cur.te.rec_begin + (c - cur.te.chunk_begin) * (long long)k_eff;
+
+        const bool arrived = mbar_wait_bounded(bar, phase);
+        phase ^= 1u;
+        if (!sb.sync_and(arrived)) {
+            if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
+            mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
+            break;
+        }
+        const long long nc = c + stride;
+        if (nc < a.n_chunks) {
+            tile_next = locate(nc);
+            if (t == 0) {
+                tma_prefetch_2d(tile_next.tm_m, tile_next.x, tile_next.y);
+                tma_prefetch_2d(tile_next.tm_g, tile_next.x, tile_next.y);
+            }
+        }
+
+        // Three passes through one copy of the transform core: 0 = DCT-II down column t of B = beta*m + g,
+        // 1 = DCT-II along row t (followed by the selection and the sparse row stage of the inverse),
+        // 2 = DCT-III down column t of the row-stage tile (followed by the residual).
+#pragma unroll 1
+        for (int ph = 0; ph < 3; ++ph) {
+            float w[S], y[S];
+            if (ph < 2) {
+                float x[S];
+                if (ph == 0) {
+#pragma unroll
+                    for (int i = 0; i < S; ++i) x[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
+                    tmem_st64(taddr, x);  // B = beta*m + g, parked for the residual
+                    sb.sync();            // every thread has consumed its column of the staged tiles (X aliases them)
+                } else {
+                    const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
+#pragma unroll
+                    for (int v4 = 0; v4 < S / 4; ++v4) {
+                        const float4 f = row[v4];
+                        x[4 * v4 + 0] = f.x;
+                        x[4 * v4 + 1] = f.y;
+                        x[4 * v4 + 2] = f.z;
+                        x[4 * v4 + 3] = f.w;
+                    }
+                }
+                fdct::dct2_pre<S>(x, w);
+            } else {
+                // column t of the row-stage tile was written by this thread only: no barrier before reading it
+                fdct::static_for<0, S>([&](auto i) {
+                    constexpr int p = decltype(i)::value;
+                    w[p] = X[fdct::core_index<S>(p) * XS + t];
+                });
+            }
+
+            fdct::dct_core_ortho<S>(w, y);
+
+            if (ph == 0) {
+                fdct::static_for<0, S>([&](auto i) {
+                    constexpr int p = decltype(i)::value;
+                    X[fdct::core_index<S>(p) * XS + t] = y[p];
+                });
+                sb.sync();
+            } else if (ph == 2) {
+                // m <- B - alpha * IDCT(kept): column t of the new momentum goes into a dense tile (the m staging
+                // area; the row-stage tile it overlaps is dead for every thread only after the barrier below, so the
+                // column is formed in registers first), which one TMA store writes out; the next chunk's tiles are
+                // requested as soon as the store has read the tile.
+                float r[S];
+                fdct::dct3_post<S>(y, r);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    float b[32];
+                    tmem_ld32(taddr + 32 * h, b);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[32 * h + i] = b[i] - r[32 * h + i];
+                }
+                sb.sync();  // every thread has read its column of the row-stage tile
+#pragma unroll
+                for (int i = 0; i < S; ++i) Ms[i * S + t] = r[i];
+                fence_proxy_async();
+                sb.sync();
+                if (t == 0) {
+                    tma_store_2d(tile_cur.tm_m, tile_cur.x, tile_cur.y, smem_u32(Ms));
+                    tma_store_commit();
+                    tma_store_wait_read();
+                    if (nc < a.n_chunks) issue_loads(tile_next);
+                }
+            } else {
+                // ---- coefficients of row t: q[v] = Q[t][v] ------------------------------------------
+                float q[S];
+                fdct::static_for<0, S>([&](auto i) {
+                    constexpr int p = decltype(i)::value;
+                    q[fdct::core_index<S>(p)] = y[p];
+                });
+                // ---- exact top-k (Section 2.1 "Top-k Sparsification") -------------------------------
+                recs4[t] = make_int4(PAD_ROW, 0, 0, 0);  // list padding (ordered before the record writes by the barriers below)
+                bool slow = (k_eff > S);
+                bool bound_valid = false;
+                bool zero_chunk = false;
+                unsigned n_cw = 0, off = 0, mlo = 0u, mhi = 0u, lmin_w = 0u;
+                if (!slow) {
+                    // per-thread maximum magnitude (independent chains of 16, 3-input max)
+                    float tm = 0.f;
+#pragma unroll
+                    for (int ch = 0; ch < S / 16; ++ch) {
+                        const int b0 = 16 * ch;
+                        float cm = max3abs(q[b0], q[b0 + 1], q[b0 + 2]);
+#pragma unroll
+                        for (int j = 3; j + 1 < 16; j += 2) cm = max3f(cm, fabsf(q[b0 + j]), fabsf(q[b0 + j + 1]));
+                        tm = max3f(tm, cm, fabsf(q[b0 + 15]));
+                    }
+                    // L = the k_eff-th largest of the 64 row maxima (low 15 mantissa bits cleared): a lower bound of
+                    // the k_eff-th largest coefficient.  Every warp holds all 64 keys, two ballots per step count them.
+                    const unsigned tkey = __float_as_uint(tm);
+                    unsigned *tk = reinterpret_cast<unsigned *>(tmax);
+                    tk[t] = tkey;
+                    sb.sync();
+                    const unsigned okey = tk[t ^ 32];
+                    const unsigned lo_all = __reduce_min_sync(0xffffffffu, min(tkey, okey));
+                    const unsigned hi_all = __reduce_max_sync(0xffffffffu, max(tkey, okey));
+                    zero_chunk = (hi_all == 0u);
+                    const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
+                    unsigned prefix = lo_all & ~((2u << b0) - 1u);
+#pragma unroll 1
+                    for (int b = zero_chunk ? 14 : b0; b >= 15; --b) {
+                        const unsigned cand = prefix | (1u << b);
+                        const unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand)) +
+                                             __popc(__ballot_sync(0xffffffffu, okey >= cand));
+                        prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
+                    }
+                    lmin_w = prefix;
+                    bound_valid = true;
+                    if (!zero_chunk) {
+                        // candidates: |q| >= L  <=>  |q| > Lm (the float just below L); the sign bit of Lm - |q|
+                        // is funnel-shifted into a bit mask (independent chains of 16)
+                        const float L = __uint_as_float(lmin_w);
+                        const float Lm = (L > 0.f) ? __uint_as_float(lmin_w - 1u) : -1.f;
+                        unsigned mc[S / 16];
+#pragma unroll
+                        for (int ch = 0; ch < S / 16; ++ch) {
+                            unsigned mm = 0u;
+#pragma unroll
+                            for (int j = 15; j >= 0; --j)
+                                mm = __funnelshift_l(__float_as_uint(Lm - fabsf(q[16 * ch + j])), mm, 1);
+                            mc[ch] = mm;
+                        }
+                        mlo = mc[0] | (mc[1] << 16);
+                        mhi = mc[2] | (mc[3] << 16);
+                        const unsigned cnt = __popc(mlo) + __popc(mhi);
+                        const unsigned inc = warp_inclusive_scan(cnt, lane);
+                        off = inc - cnt;
+                        n_cw = __shfl_sync(0xffffffffu, inc, 31);
+                        if (lane == 0) misc[warp] = n_cw;
+                    }
+                }
+                if (zero_chunk) {
+                    // all coefficients zero: the tie rule gives the records 0 .. k_eff-1 with value 0
+                    if (t < k_eff) {
+                        DemoRecord r;
+                        r.idx = t;
+                        r.val = 0.f;
+                        rec[t] = r;
+                    }
+                    if (t < k_eff) recs4[t] = make_int4(0, 0, 0, 0);
+                } else {
+                    // stash the coefficients of row t (own row: no hazard with other threads)
+                    float4 *row = reinterpret_cast<float4 *>(X + t * XS);
+#pragma unroll
+                    for (int v4 = 0; v4 < S / 4; ++v4)
+                        row[v4] = make_float4(q[4 * v4], q[4 * v4 + 1], q[4 * v4 + 2], q[4 * v4 + 3]);
+                    if (!slow) {
+                        const unsigned lbase = warp * CAPWP;
+                        if (n_cw <= CAPW) {
+                            // each warp compacts its candidates into its own list (rows of warp 0 precede rows of
+                            // warp 1, so the concatenation is in ascending index order)
+                            unsigned o = lbase + off;
+                            unsigned long long mask = ((unsigned long long)mhi << 32) | mlo;
+                            while (mask) {
+                                const int v = __ffsll((long long)mask) - 1;
+                                mask &= mask - 1ull;
+                                const float val = X[t * XS + v];
+                                cand_idx[o] = t * S + v;
+                                cand_val[o] = val;
+                                cand_key[o] = mag_key(val);
+                                ++o;
+                            }
+                            if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
+                        }
+                        sb.sync();
+                        const unsigned n_w0 = misc[0], n_w1 = misc[1];
+                        // more than a list holds, or fewer candidates than k_eff (NaN coefficients fail the float
+                        // comparisons above): the out-of-line selection takes over
+                        slow = (n_w0 > (unsigned)CAPW) || (n_w1 > (unsigned)CAPW) || (n_w0 + n_w1 < (unsigned)k_eff);
+                        if (!slow) {
+                            // Every warp takes both lists into registers (two keys per lane and list) and searches,
+                            // bit by bit from the first bit where the bound and the largest key differ, for a
+                            // threshold with exactly k_eff keys at or above it; the search stops as soon as one is
+                            // found.  If it runs out of bits, equal keys straddle the k_eff-th place: keys above
+                            // the threshold are kept, keys equal to it in index order until k_eff are reached.
+                            const unsigned n_mine = warp ? n_w1 : n_w0, n_oth = warp ? n_w0 : n_w1;
+                            const unsigned obase = (warp ^ 1) * CAPWP;
+                            unsigned keys[4];  // 0, 1: this warp's list; 2, 3: the other warp's
+                            keys[0] = (lane < n_mine) ? cand_key[lbase + lane] : 0u;
+                            keys[1] = (lane + 32u < n_mine) ? cand_key[lbase + 32 + lane] : 0u;
+                            keys[2] = (lane < n_oth) ? cand_key[obase + lane] : 0u;
+                            keys[3] = (lane + 32u < n_oth) ? cand_key[obase + 32 + lane] : 0u;
+                            const unsigned hi = __reduce_max_sync(0xffffffffu, max(max(keys[0], keys[1]), max(keys[2], keys[3])));
+                            const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
+                            unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+                            unsigned n_ge = n_w0 + n_w1;  // every candidate is >= the bound >= thr
+#pragma unroll 1
+                            for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
+                                const unsigned cand = thr | (1u << b);
+                                unsigned cnt = 0;
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+                                if (cnt >= (unsigned)k_eff) {
+                                    thr = cand;
+                                    n_ge = cnt;
+                                }
+                            }
+                            // kept entries before this warp's list (index order: list 0, then list 1) and in all
+                            const unsigned g_oth = __popc(__ballot_sync(0xffffffffu, keys[2] > thr)) +
+                                                   __popc(__ballot_sync(0xffffffffu, keys[3] > thr));
+                            const unsigned e_oth = __popc(__ballot_sync(0xffffffffu, keys[2] == thr)) +
+                                                   __popc(__ballot_sync(0xffffffffu, keys[3] == thr));
+                            const unsigned gtb0 = __ballot_sync(0xffffffffu, keys[0] > thr);
+                            const unsigned gtb1 = __ballot_sync(0xffffffffu, keys[1] > thr);
+                            const unsigned eqb0 = __ballot_sync(0xffffffffu, keys[0] == thr);
+                            const unsigned eqb1 = __ballot_sync(0xffffffffu, keys[1] == thr);
+                            const unsigned need_eq = (unsigned)k_eff - (g_oth + __popc(gtb0) + __popc(gtb1));
+                            const unsigned lt = (1u << lane) - 1u;
+#pragma unroll 1
+                            for (int jj = 0; jj < 2; ++jj) {  // (rolled: one copy of the record write)
+                                const unsigned key = jj ? keys[1] : keys[0];
+                                const unsigned gtb = jj ? gtb1 : gtb0, eqb = jj ? eqb1 : eqb0;
+                                const unsigned gt_before = (warp ? g_oth : 0u) + (jj ? __popc(gtb0) : 0u);
+                                const unsigned e = (warp ? e_oth : 0u) + (jj ? __popc(eqb0) : 0u) + __popc(eqb & lt);
+                                if ((key > thr) || (key == thr && e < need_eq)) {
+                                    const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
+                                    const unsigned li = lbase + (unsigned)jj * 32u + lane;
+                                    DemoRecord r;
+                                    r.idx = cand_idx[li];
+                                    r.val = cand_val[li];
+                                    rec[pos] = r;
+                                    recs4[pos] = make_int4((r.idx >> LOG2S) * XS, (r.idx & (S - 1)) * S,
+                                                           __float_as_int(a.alpha * r.val), 0);
+                                }
+                            }
+                        }
+                    }
+                    if (slow) select_slow(sm, k_eff, rec, a.alpha, t, slot + 1, lmin_w, bound_valid);
+                }
+                sb.sync();  // records complete (shared list and global payload); X is free
+
+                // ---- residual: row stage of the inverse from the k_eff records, sparse --------------
+                {
+                    float4 *row = reinterpret_cast<float4 *>(X + t * XS);
+#pragma unroll
+                    for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                sb.sync();
+                {
+                    // T[u][t] = sum over kept (u, v) of alpha * val * C[v][t]; the basis is read through L1
+                    const float *Ct = a.C + t;
+                    float acc = 0.f;
+                    int cur_u = PAD_ROW;
+                    if (k_eff <= 64) {
+                        // the list is padded to 64 entries with zero-valued records of row PAD_ROW; four records and
+                        // their cosines are fetched ahead of the dependent accumulation
+#pragma unroll 1
+                        for (int r0 = 0; r0 < k_eff; r0 += 4) {
+                            int4 rc[4];
+                            float cv[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) rc[j] = recs4[r0 + j];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) cv[j] = __ldg(Ct + rc[j].y);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const bool chg = rc[j].x != cur_u;
+                                if (chg && cur_u != PAD_ROW) X[cur_u + t] = acc;
+                                acc = chg ? 0.f : acc;
+                                cur_u = rc[j].x;
+                                acc = fmaf(__int_as_float(rc[j].z), cv[j], acc);
+                            }
+                        }
+                    } else {
+#pragma unroll 1
+                        for (int r = 0; r < k_eff; ++r) {
+                            const DemoRecord rc = rec[r];
+                            const int u = (rc.idx >> LOG2S) * XS, v = rc.idx & (S - 1);
+                            if (u != cur_u) {
+                                if (cur_u != PAD_ROW) X[cur_u + t] = acc;
+                                acc = 0.f;
+                                cur_u = u;
+                            }
+                            acc = fmaf(a.alpha * rc.val, __ldg(Ct + v * S), acc);
+                        }
+                    }
+                    if (cur_u != PAD_ROW) X[cur_u + t] = acc;
+                }
+            }
+        }
+    }
+    // tear-down: every slot of the CTA is done with its tensor-memory columns
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (hw_warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+}
+
+template <typename GT, int THREADS>
+cudaError_t launch64(const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
+{
+    constexpr int NCH = THREADS / S;
+    auto kernel = compress64_kernel<GT, THREADS>;
+    const size_t smem = slot_bytes<GT>() * NCH + 16;
+    if (a.n_chunks <= 0) return cudaSuccess;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    // CTAs per SM: registers (launch bounds: 512 threads per SM), shared memory (227 KB, 1 KB reserved per CTA)
+    // and tensor memory (512 columns, 64 per four warps).  The occupancy calculator is not asked: it does not
+    // know about tensor memory and was seen to answer 1 for this kernel.
+    int per_sm = 512 / THREADS;
+    const int smem_limit = (int)((227u * 1024u) / (smem + 1024u));
+    const int tmem_limit = 512 / (((THREADS + 127) / 128) * TMEM_COLS_PER_GROUP);
+    if (per_sm > smem_limit) per_sm = smem_limit;
+    if (per_sm > tmem_limit) per_sm = tmem_limit;
+    if (per_sm < 1) per_sm = 1;
+    const long long groups = (a.n_chunks + NCH - 1) / NCH;
+    long long grid = (long long)sm_count * per_sm;
+    if (grid > groups) grid = groups;
+    kernel<<<(unsigned)grid, THREADS, smem, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// Needs the TMA tensor maps of both tensors.
+cudaError_t demo_launch_compress_fast64(const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
+{
+    if (a.tmap_m == nullptr || a.tmap_g == nullptr) return cudaErrorNotSupported;
+    return a.grad_bf16 ? launch64<__nv_bfloat16, 128>(a, sm_count, stream) : launch64<float, 128>(a, sm_count, stream);
+}
