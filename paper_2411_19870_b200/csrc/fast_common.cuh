@@ -95,25 +95,29 @@ __device__ __forceinline__ float max3f(float a, float b, float c)
 __device__ __forceinline__ float max3abs(float a, float b, float c) { return max3f(fabsf(a), fabsf(b), fabsf(c)); }
 __device__ __forceinline__ unsigned mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
-// Walks the tensor table as the CTA's chunk ids grow.
+// Walks the tensor table as the CTA's chunk ids grow.  The first chunk of the next tensor is kept in a
+// register, so that a chunk inside the current tensor costs one comparison and no memory access.
 struct EntryCursor {
     int e = 0;
     DemoTensorEntry te;
+    long long next_begin = 0;  // chunk_begin of entry e + 1 (or "never")
     bool loaded = false;
+    __device__ __forceinline__ void load(const DemoTensorEntry *entries, int n)
+    {
+        te = entries[e];
+        next_begin = (e + 1 < n) ? entries[e + 1].chunk_begin : 0x7fffffffffffffffLL;
+    }
     __device__ __forceinline__ void seek(const DemoTensorEntry *entries, int n, long long c)
     {
         if (!loaded) {
             e = demo_find_entry(entries, n, c);
-            te = entries[e];
+            load(entries, n);
             loaded = true;
             return;
         }
-        bool moved = false;
-        while (e + 1 < n && entries[e + 1].chunk_begin <= c) {
-            ++e;
-            moved = true;
-        }
-        if (moved) te = entries[e];
+        if (c < next_begin) return;
+        while (e + 1 < n && entries[e + 1].chunk_begin <= c) ++e;
+        load(entries, n);
     }
 };
 

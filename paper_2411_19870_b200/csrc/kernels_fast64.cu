@@ -85,8 +85,8 @@ __device__ __forceinline__ void tmem_st64(uint32_t taddr, const float (&v)[64])
         "f"(v[46]), "f"(v[47]), "f"(v[48]), "f"(v[49]), "f"(v[50]), "f"(v[51]), "f"(v[52]), "f"(v[53]), "f"(v[54]),
         "f"(v[55]), "f"(v[56]), "f"(v[57]), "f"(v[58]), "f"(v[59]), "f"(v[60]), "f"(v[61]), "f"(v[62]), "f"(v[63])
         : "memory");
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 {
     asm volatile(
@@ -383,9 +383,10 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     const uint32_t taddr = tmem_base + ((uint32_t)((hw_warp & 3) * 32) << 16) + (uint32_t)((hw_warp >> 2) * TMEM_COLS_PER_GROUP);
 
     EntryCursor cur;
-    int cached_tensor = -1;
+    const char *acquired = nullptr;  // (thread 0) the last tensor map made visible to the tensor-map proxy
     unsigned phase = 0;
 
+    // Tile of chunk c: tensor maps and box coordinates (the cursor is moved to c; chunk ids only grow).
     struct TileRef {
         const char *tm_m, *tm_g;
         int x, y;
@@ -400,34 +401,30 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
         r.y = (int)k0 * S;
         r.tm_m = static_cast<const char *>(a.tmap_m) + (size_t)cur.te.tensor * TMAP_BYTES;
         r.tm_g = static_cast<const char *>(a.tmap_g) + (size_t)cur.te.tensor * TMAP_BYTES;
-        if (cur.te.tensor != cached_tensor) {
-            cached_tensor = cur.te.tensor;
-            if (t == 0) {
-                tmap_acquire(r.tm_m);
-                tmap_acquire(r.tm_g);
-            }
-        }
         return r;
     };
+    // (thread 0) request the tiles of a chunk; a tensor map that this thread has not used yet is acquired first
     auto issue_loads = [&](const TileRef &r) {
-        if (t == 0) {
-            mbar_expect_tx(bar, TILE_BYTES);
-            tma_load_2d(smem_u32(Ms), r.tm_m, r.x, r.y, bar);
-            tma_load_2d(smem_u32(Gs), r.tm_g, r.x, r.y, bar);
+        if (r.tm_m != acquired) {
+            acquired = r.tm_m;
+            tmap_acquire(r.tm_m);
+            tmap_acquire(r.tm_g);
         }
+        mbar_expect_tx(bar, TILE_BYTES);
+        tma_load_2d(smem_u32(Ms), r.tm_m, r.x, r.y, bar);
+        tma_load_2d(smem_u32(Gs), r.tm_g, r.x, r.y, bar);
     };
 
     const long long stride = (long long)gridDim.x * NCH;
     long long c = (long long)blockIdx.x * NCH + slot;
-    TileRef tile_cur, tile_next;
+    TileRef next{};
     if (c < a.n_chunks) {
-        tile_next = locate(c);
-        issue_loads(tile_next);
+        next = locate(c);
+        if (t == 0) issue_loads(next);
     }
 
     for (; c < a.n_chunks; c += stride) {
         // the cursor points at chunk c (its loads were issued last)
-        tile_cur = tile_next;
         const int k_eff = cur.te.k_eff;
         DemoRecord *rec = a.payload + cur.te.rec_begin + (c - cur.te.chunk_begin) * (long long)k_eff;
 
@@ -438,14 +435,10 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
             mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
             break;
         }
+        // where this chunk's tile goes back to and where the next one comes from (moves the cursor on)
+        const TileRef mine = next;
         const long long nc = c + stride;
-        if (nc < a.n_chunks) {
-            tile_next = locate(nc);
-            if (t == 0) {
-                tma_prefetch_2d(tile_next.tm_m, tile_next.x, tile_next.y);
-                tma_prefetch_2d(tile_next.tm_g, tile_next.x, tile_next.y);
-            }
-        }
+        if (nc < a.n_chunks) next = locate(nc);
 
         // Three passes through one copy of the transform core: 0 = DCT-II down column t of B = beta*m + g,
         // 1 = DCT-II along row t (followed by the selection and the sparse row stage of the inverse),
@@ -495,6 +488,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 // requested as soon as the store has read the tile.
                 float r[S];
                 fdct::dct3_post<S>(y, r);
+                tmem_wait_st();  // the store of B (pass 0) has long completed
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     float b[32];
@@ -507,11 +501,14 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 for (int i = 0; i < S; ++i) Ms[i * S + t] = r[i];
                 fence_proxy_async();
                 sb.sync();
-                if (t == 0) {
-                    tma_store_2d(tile_cur.tm_m, tile_cur.x, tile_cur.y, smem_u32(Ms));
-                    tma_store_commit();
-                    tma_store_wait_read();
-                    if (nc < a.n_chunks) issue_loads(tile_next);
+                {
+                    // the store of this chunk, then -- once it has read the tile -- the loads of the next chunk
+                    if (t == 0) {
+                        tma_store_2d(mine.tm_m, mine.x, mine.y, smem_u32(Ms));
+                        tma_store_commit();
+                        tma_store_wait_read();
+                        if (nc < a.n_chunks) issue_loads(next);
+                    }
                 }
             } else {
                 // ---- coefficients of row t: q[v] = Q[t][v] ------------------------------------------
@@ -520,6 +517,12 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                     constexpr int p = decltype(i)::value;
                     q[fdct::core_index<S>(p)] = y[p];
                 });
+                // the row-stage tile starts from zero; every thread clears its own row once it is done with it
+                auto zero_row = [&]() {
+                    float4 *row = reinterpret_cast<float4 *>(X + t * XS);
+#pragma unroll
+                    for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
+                };
                 // ---- exact top-k (Section 2.1 "Top-k Sparsification") -------------------------------
                 recs4[t] = make_int4(PAD_ROW, 0, 0, 0);  // list padding (ordered before the record writes by the barriers below)
                 bool slow = (k_eff > S);
@@ -590,6 +593,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                         rec[t] = r;
                     }
                     if (t < k_eff) recs4[t] = make_int4(0, 0, 0, 0);
+                    zero_row();
                 } else {
                     // stash the coefficients of row t (own row: no hazard with other threads)
                     float4 *row = reinterpret_cast<float4 *>(X + t * XS);
@@ -620,6 +624,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                         // comparisons above): the out-of-line selection takes over
                         slow = (n_w0 > (unsigned)CAPW) || (n_w1 > (unsigned)CAPW) || (n_w0 + n_w1 < (unsigned)k_eff);
                         if (!slow) {
+                            zero_row();  // row t of the stash was read by this thread only
                             // Every warp takes both lists into registers (two keys per lane and list) and searches,
                             // bit by bit from the first bit where the bound and the largest key differ, for a
                             // threshold with exactly k_eff keys at or above it; the search stops as soon as one is
@@ -677,17 +682,15 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                             }
                         }
                     }
-                    if (slow) select_slow(sm, k_eff, rec, a.alpha, t, slot + 1, lmin_w, bound_valid);
+                    if (slow) {
+                        select_slow(sm, k_eff, rec, a.alpha, t, slot + 1, lmin_w, bound_valid);
+                        sb.sync();  // every thread is done with the coefficient tile
+                        zero_row();
+                    }
                 }
-                sb.sync();  // records complete (shared list and global payload); X is free
+                sb.sync();  // records complete (shared list and global payload), tile zeroed
 
                 // ---- residual: row stage of the inverse from the k_eff records, sparse --------------
-                {
-                    float4 *row = reinterpret_cast<float4 *>(X + t * XS);
-#pragma unroll
-                    for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                sb.sync();
                 {
                     // T[u][t] = sum over kept (u, v) of alpha * val * C[v][t]; the basis is read through L1
                     const float *Ct = a.C + t;
@@ -696,16 +699,22 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                     if (k_eff <= 64) {
                         // the list is padded to 64 entries with zero-valued records of row PAD_ROW; four records and
                         // their cosines are fetched ahead of the dependent accumulation
+#ifndef DEMO_CV
+#define DEMO_CV(p) __ldg(p)
+#endif
+#ifndef DEMO_RU
+#define DEMO_RU 4
+#endif
 #pragma unroll 1
-                        for (int r0 = 0; r0 < k_eff; r0 += 4) {
-                            int4 rc[4];
-                            float cv[4];
+                        for (int r0 = 0; r0 < k_eff; r0 += DEMO_RU) {
+                            int4 rc[DEMO_RU];
+                            float cv[DEMO_RU];
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) rc[j] = recs4[r0 + j];
+                            for (int j = 0; j < DEMO_RU; ++j) rc[j] = recs4[r0 + j];
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) cv[j] = __ldg(Ct + rc[j].y);
+                            for (int j = 0; j < DEMO_RU; ++j) cv[j] = DEMO_CV(Ct + rc[j].y);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
+                            for (int j = 0; j < DEMO_RU; ++j) {
                                 const bool chg = rc[j].x != cur_u;
                                 if (chg && cur_u != PAD_ROW) X[cur_u + t] = acc;
                                 acc = chg ? 0.f : acc;
@@ -769,5 +778,8 @@ cudaError_t launch64(const DemoCompressArgs &a, int sm_count, cudaStream_t strea
 cudaError_t demo_launch_compress_fast64(const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
 {
     if (a.tmap_m == nullptr || a.tmap_g == nullptr) return cudaErrorNotSupported;
-    return a.grad_bf16 ? launch64<__nv_bfloat16, 128>(a, sm_count, stream) : launch64<float, 128>(a, sm_count, stream);
+#ifndef DEMO_T64
+#define DEMO_T64 64
+#endif
+    return a.grad_bf16 ? launch64<__nv_bfloat16, DEMO_T64>(a, sm_count, stream) : launch64<float, DEMO_T64>(a, sm_count, stream);
 }
