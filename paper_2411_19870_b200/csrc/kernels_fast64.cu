@@ -49,7 +49,7 @@ constexpr size_t region_bytes()
 template <typename GT>
 constexpr size_t slot_bytes()
 {
-    constexpr size_t raw = region_bytes<GT>() + S * 4 + (CAP + 8) * 3 * 4 + 64 * 16 + 16 * 4 + 16;
+    constexpr size_t raw = region_bytes<GT>() + S * 4 + (CAP + 8) * 3 * 4 + 65 * 16 + 16 * 4 + 16;
     return (raw + 127) / 128 * 128;
 }
 
@@ -62,7 +62,7 @@ struct SlotMem {
     float *cand_val;     // [CAP + 8]
     unsigned *cand_key;  // [CAP + 8]
     unsigned *hist;      // [256] aliases the candidate arrays
-    int4 *recs4;         // [64] kept records, pre-decoded for the row stage
+    int4 *recs4;         // [65] kept records, pre-decoded for the row stage; entry 64 is always padding
     unsigned *misc;      // [16]
     unsigned *wkey;      // [WCAP + 4] wide list, behind the tile
     unsigned *widx;      // [WCAP + 4]
@@ -348,7 +348,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     sm.cand_key = reinterpret_cast<unsigned *>(sm.cand_val + CAP + 8);
     sm.hist = reinterpret_cast<unsigned *>(sm.cand_idx);
     sm.recs4 = reinterpret_cast<int4 *>(sm.cand_key + CAP + 8);
-    sm.misc = reinterpret_cast<unsigned *>(sm.recs4 + 64);
+    sm.misc = reinterpret_cast<unsigned *>(sm.recs4 + 65);
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(sm.misc + 16);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_all + (size_t)NCH * slot_bytes<GT>());
     float *X = sm.X;
@@ -428,13 +428,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
         const int k_eff = cur.te.k_eff;
         DemoRecord *rec = a.payload + cur.te.rec_begin + (c - cur.te.chunk_begin) * (long long)k_eff;
 
+        // every thread waits for the tiles by itself; whether the wait expired is settled for the whole slot
+        // at the first barrier of pass 0 (no barrier lies in between)
         const bool arrived = mbar_wait_bounded(bar, phase);
         phase ^= 1u;
-        if (!sb.sync_and(arrived)) {
-            if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
-            mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
-            break;
-        }
+        bool dead = false;
         // where this chunk's tile goes back to and where the next one comes from (moves the cursor on)
         const TileRef mine = next;
         const long long nc = c + stride;
@@ -452,7 +450,13 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
 #pragma unroll
                     for (int i = 0; i < S; ++i) x[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
                     tmem_st64(taddr, x);  // B = beta*m + g, parked for the residual
-                    sb.sync();            // every thread has consumed its column of the staged tiles (X aliases them)
+                    // every thread has consumed its column of the staged tiles (X aliases them)
+                    if (!sb.sync_and(arrived)) {
+                        if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
+                        mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
+                        dead = true;
+                        break;
+                    }
                 } else {
                     const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
 #pragma unroll
@@ -525,6 +529,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 };
                 // ---- exact top-k (Section 2.1 "Top-k Sparsification") -------------------------------
                 recs4[t] = make_int4(PAD_ROW, 0, 0, 0);  // list padding (ordered before the record writes by the barriers below)
+                if (t == 0) recs4[64] = make_int4(PAD_ROW, 0, 0, 0);
                 bool slow = (k_eff > S);
                 bool bound_valid = false;
                 bool zero_chunk = false;
@@ -695,50 +700,51 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                     // T[u][t] = sum over kept (u, v) of alpha * val * C[v][t]; the basis is read through L1
                     const float *Ct = a.C + t;
                     float acc = 0.f;
-                    int cur_u = PAD_ROW;
                     if (k_eff <= 64) {
-                        // the list is padded to 64 entries with zero-valued records of row PAD_ROW; four records and
-                        // their cosines are fetched ahead of the dependent accumulation
-#ifndef DEMO_CV
-#define DEMO_CV(p) __ldg(p)
-#endif
-#ifndef DEMO_RU
-#define DEMO_RU 4
-#endif
+                        // The list is padded with zero-valued entries of row PAD_ROW (entry 64 is always one).  A row's
+                        // sum is stored when the next entry belongs to another row; padding follows padding, so the
+                        // padding row itself is never stored.  Four entries and their cosines are fetched ahead of the
+                        // dependent accumulation.
+                        float *Xt = X + t;
+                        int4 nx = recs4[0];
 #pragma unroll 1
-                        for (int r0 = 0; r0 < k_eff; r0 += DEMO_RU) {
-                            int4 rc[DEMO_RU];
-                            float cv[DEMO_RU];
+                        for (int r0 = 0; r0 < k_eff; r0 += 4) {
+                            int4 rc[5];
+                            float cv[4];
+                            rc[0] = nx;
 #pragma unroll
-                            for (int j = 0; j < DEMO_RU; ++j) rc[j] = recs4[r0 + j];
+                            for (int j = 1; j < 5; ++j) rc[j] = recs4[r0 + j];
+                            nx = rc[4];
 #pragma unroll
-                            for (int j = 0; j < DEMO_RU; ++j) cv[j] = DEMO_CV(Ct + rc[j].y);
+                            for (int j = 0; j < 4; ++j) cv[j] = __ldg(Ct + rc[j].y);
 #pragma unroll
-                            for (int j = 0; j < DEMO_RU; ++j) {
-                                const bool chg = rc[j].x != cur_u;
-                                if (chg && cur_u != PAD_ROW) X[cur_u + t] = acc;
-                                acc = chg ? 0.f : acc;
-                                cur_u = rc[j].x;
+                            for (int j = 0; j < 4; ++j) {
                                 acc = fmaf(__int_as_float(rc[j].z), cv[j], acc);
+                                if (rc[j].x != rc[j + 1].x) {
+                                    Xt[rc[j].x] = acc;
+                                    acc = 0.f;
+                                }
                             }
                         }
                     } else {
+                        int cur_u = -1;
 #pragma unroll 1
                         for (int r = 0; r < k_eff; ++r) {
                             const DemoRecord rc = rec[r];
                             const int u = (rc.idx >> LOG2S) * XS, v = rc.idx & (S - 1);
                             if (u != cur_u) {
-                                if (cur_u != PAD_ROW) X[cur_u + t] = acc;
+                                if (cur_u >= 0) X[cur_u + t] = acc;
                                 acc = 0.f;
                                 cur_u = u;
                             }
                             acc = fmaf(a.alpha * rc.val, __ldg(Ct + v * S), acc);
                         }
+                        if (cur_u >= 0) X[cur_u + t] = acc;
                     }
-                    if (cur_u != PAD_ROW) X[cur_u + t] = acc;
                 }
             }
         }
+        if (dead) break;
     }
     // tear-down: every slot of the CTA is done with its tensor-memory columns
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
