@@ -247,8 +247,10 @@ demo_status demo_step_host(demo_ctx *ctx, const void *const *host_grads, void *c
  * their chunk are skipped as in demo_decode_apply, but are not reported (there is no context to query).
  *
  * The first call on a device looks up the array's device address (a one-time set-up that should
- * happen before any stream capture begins).  The 2-D and 1-D tensors run through the generic decode
- * kernels.  Errors: INVALID_ARG, SHAPE, K, UNSUPPORTED, CUDA.
+ * happen before any stream capture begins).  Every call copies its tables from host memory that is
+ * gone when the call returns, so the call must not be recorded into a CUDA graph: a stream that is
+ * capturing is refused with DEMO_ERR_INVALID_ARG before anything is enqueued.  The 2-D and 1-D
+ * tensors run through the generic decode kernels.  Errors: INVALID_ARG, SHAPE, K, UNSUPPORTED, CUDA.
  */
 #define DEMO_STATIC_MAX_TENSORS 256
 #define DEMO_STATIC_MAX_WORKERS 64

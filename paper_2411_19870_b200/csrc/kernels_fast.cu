@@ -104,6 +104,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
     const GT *g_ptr = nullptr;
     int cached_tensor = -1;
     unsigned phase = 0;
+    const char *acquired = nullptr;  // the last tensor map made visible to the tensor-map proxy (thread 0 of the slot)
 
     // Locate the tile of chunk c (advances the tensor cursor; chunk ids only grow): tensor maps and box
     // coordinates for the TMA path, row t of the tile for the row-by-row path.
@@ -133,6 +134,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
         if (TMAP) {
             r.tm_m = static_cast<const char *>(a.tmap_m) + (size_t)cached_tensor * TMAP_BYTES;
             r.tm_g = static_cast<const char *>(a.tmap_g) + (size_t)cached_tensor * TMAP_BYTES;
+            if (t == 0 && r.tm_m != acquired) {  // first use of these maps by the issuing thread
+                acquired = r.tm_m;
+                tmap_acquire(r.tm_m);
+                tmap_acquire(r.tm_g);
+            }
         } else {
             const size_t off = ((size_t)k0 * S + t) * (size_t)cur.te.n1 + (size_t)k1 * S;
             r.m_src = m_ptr + off;
@@ -777,6 +783,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
     int cached_tensor = -1;
     unsigned phase = 0;
     bool failed = false;
+    const char *acquired = nullptr;
     const unsigned lr_bits = __float_as_uint(a.lr);
     const float decay = 1.f - a.lr * a.wd;
     const float neg_lr_scale = -a.lr * a.agg_scale;
@@ -799,8 +806,14 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
         float *__restrict__ x = x_ptr;
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + lc * (long long)k_eff;
-        if (TMAP && !SIGNS && t == 0)
-            tma_prefetch_2d(static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES, k1 * S, (int)k0 * S);
+        if (TMAP && !SIGNS && t == 0) {
+            const char *tm_x = static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES;
+            if (tm_x != acquired) {  // first use of this tensor's map by the issuing thread
+                acquired = tm_x;
+                tmap_acquire(tm_x);
+            }
+            tma_prefetch_2d(tm_x, k1 * S, (int)k0 * S);
+        }
 
         {
             float4 *row = reinterpret_cast<float4 *>(St + t * XS);

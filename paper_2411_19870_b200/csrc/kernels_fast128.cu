@@ -109,14 +109,22 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
 
     EntryCursor cur;
     unsigned phase = 0;
+    const char *acquired = nullptr;
 
     auto issue_tiles = [&](const DemoTensorEntry &te, long long c) {
         const unsigned lc = (unsigned)(c - te.chunk_begin);
         const unsigned k0 = lc / (unsigned)te.c1, k1 = lc - k0 * (unsigned)te.c1;
         if (tid == 0) {
+            const char *tm_m = static_cast<const char *>(a.tmap_m) + (size_t)te.tensor * TMAP_BYTES;
+            const char *tm_g = static_cast<const char *>(a.tmap_g) + (size_t)te.tensor * TMAP_BYTES;
+            if (tm_m != acquired) {  // a tensor map this thread has not used yet: acquire it for the tensor-map proxy
+                acquired = tm_m;
+                tmap_acquire(tm_m);
+                tmap_acquire(tm_g);
+            }
             mbar_expect_tx(bar, TILE_BYTES);
-            tma_load_2d(smem_u32(Ms), static_cast<const char *>(a.tmap_m) + (size_t)te.tensor * TMAP_BYTES, k1 * S, k0 * S, bar);
-            tma_load_2d(smem_u32(Gs), static_cast<const char *>(a.tmap_g) + (size_t)te.tensor * TMAP_BYTES, k1 * S, k0 * S, bar);
+            tma_load_2d(smem_u32(Ms), tm_m, k1 * S, k0 * S, bar);
+            tma_load_2d(smem_u32(Gs), tm_g, k1 * S, k0 * S, bar);
         }
     };
 
@@ -484,6 +492,7 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
     const float decay = 1.f - a.lr * a.wd;
     const float neg_lr_scale = -a.lr * a.agg_scale;
     const bool counts = a.agg == 2;
+    const char *acquired = nullptr;
 
     for (long long c = blockIdx.x; c < a.n_chunks; c += gridDim.x) {
         cur.seek(a.entries, a.n_entries, c);
@@ -495,7 +504,13 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
         const int k_eff = te.k_eff;
         const long long rec_off = te.rec_begin + (long long)lc * k_eff;
         const char *tm_x = static_cast<const char *>(a.tmap_x) + (size_t)te.tensor * TMAP_BYTES;
-        if (!SIGNS && tid == 0) tma_prefetch_2d(tm_x, k1 * S, k0 * S);
+        if (!SIGNS && tid == 0) {
+            if (tm_x != acquired) {  // first use of this tensor's map by this thread
+                acquired = tm_x;
+                tmap_acquire(tm_x);
+            }
+            tma_prefetch_2d(tm_x, k1 * S, k0 * S);
+        }
 
         for (int i = tid; i < S * XSD / 4; i += THREADS) reinterpret_cast<float4 *>(St)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (counts)

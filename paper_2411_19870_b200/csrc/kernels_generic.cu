@@ -491,6 +491,15 @@ extern "C" demo_status demo_decode_apply_static(const demo_config *cfg, const de
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     demo_status result = DEMO_OK;
     do {
+        // The tables are copied from host memory that is gone when this call returns (a stack frame, the
+        // caller's pointer arrays).  Recorded into a CUDA graph those copies would be replayed from dead
+        // memory, so a stream that is capturing is refused before anything is enqueued.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+            cudaGetLastError();
+            result = DEMO_ERR_INVALID_ARG;
+            break;
+        }
         // one-time set-up per device, with that device current: translate the symbol into a device address
         unsigned char *base = nullptr;
         {

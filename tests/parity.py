@@ -33,6 +33,13 @@ def sample_chunk_ids(n_chunks: int, max_n: int, seed: int) -> np.ndarray:
     return np.sort(np.concatenate([[0, n_chunks - 1], mid])).astype(np.int64)
 
 
+def sample_chunk_fraction(n_chunks: int, denom: int, seed: int, min_n: int = 8) -> np.ndarray:
+    """First and last chunk plus a seeded uniform sample, at least n_chunks / denom chunks in all (every chunk
+    when the tensor has no more than min_n)."""
+    want = max(min_n, -(-n_chunks // denom))
+    return sample_chunk_ids(n_chunks, want, seed)
+
+
 def gather_tiles(t: torch.Tensor, s: int, chunk_ids: np.ndarray) -> np.ndarray:
     """Tiles of the listed chunks (row-major chunk ids) as float64 [n, M]."""
     ids = torch.as_tensor(chunk_ids, device=t.device)
@@ -240,15 +247,24 @@ class Runner:
             self.tr.set_basis(None)
             self.basis = None
 
-    def step(self, check=True, grads=None):
+    def step(self, check=True, grads=None, workers=None, invariants=False):
+        """One optimizer step.  `workers`: the workers whose compress call is compared with the oracle (default:
+        all); the decode is compared on the payloads of every worker either way.  `invariants`: also check the
+        whole-tensor properties (every chunk, no oracle) of every worker's compress call."""
         wl, s = self.wl, self.wl.chunk
         T = len(wl.shapes)
         for w in range(wl.num_workers):
             g = grads[w] if grads is not None else self.streams[w].next()
-            if check:
+            check_w = check and (workers is None or w in workers)
+            if invariants:
+                energy = [tensor_energy(self.beta, self.mom[w][t], g[t]) for t in range(T)]
+            if check_w:
                 before = [gather_tiles(self.mom[w][t], s, self.ids[t]) for t in range(T)]
             self.tr.compress(w, g, self.mom[w], self.payloads[w])
-            if check:
+            if invariants:
+                self.report.add("invariant_records", check_whole_tensor_invariants(
+                    self.payloads[w], self.layout, wl.shapes, s, energy, self.mom[w], what="worker %d" % w))
+            if check_w:
                 for t in range(T):
                     rows = s if len(wl.shapes[t]) == 2 else 1
                     first, _, k_eff = self.layout[t]
@@ -343,3 +359,55 @@ class NdRunner:
 
     def close(self):
         self.tr.close()
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Whole-tensor properties that hold at any size, evaluated on the device over EVERY chunk (no oracle call):
+#   * every record index lies in its chunk and the indices of a chunk are strictly ascending (exactly k_eff
+#     distinct coefficients per chunk, Section 2.1 "Top-k Sparsification");
+#   * energy split of an orthonormal transform: ||m_new||^2 = ||beta m + g||^2 - sum val^2 per tensor
+#     (Parseval; the residual is B minus the kept coefficients' reconstruction).
+# ---------------------------------------------------------------------------------------------------------
+def tensor_energy(beta: float, m: torch.Tensor, g: torch.Tensor) -> float:
+    """sum (beta m + g)^2 of one tensor, accumulated in fp64 slice by slice (bounded temporary memory)."""
+    tot = 0.0
+    mf, gf = m.reshape(-1), g.reshape(-1)
+    step = 1 << 26
+    for i in range(0, mf.numel(), step):
+        b = torch.add(gf[i:i + step].double(), mf[i:i + step].double(), alpha=beta)
+        tot += float(b.pow(2).sum().item())
+    return tot
+
+
+def sum_squares(t: torch.Tensor) -> float:
+    tot = 0.0
+    f = t.reshape(-1)
+    step = 1 << 26
+    for i in range(0, f.numel(), step):
+        tot += float(f[i:i + step].double().pow(2).sum().item())
+    return tot
+
+
+def check_whole_tensor_invariants(payload: torch.Tensor, layout, shapes, chunk: int, energy_before, mom_after,
+                                  what: str = "", rtol: float = 1e-5) -> int:
+    """payload: one worker's uint8 buffer; layout[t] = (first_record, n_chunks, k_eff); energy_before[t] =
+    tensor_energy(...) taken before the compress call; mom_after: that worker's momentum tensors after it.
+    Returns the number of records seen."""
+    rec = payload.view(torch.int32).view(-1, 2)
+    seen = 0
+    for t, shp in enumerate(shapes):
+        first, n_chunks, k_eff = layout[t]
+        M = chunk * chunk if len(shp) == 2 else chunk
+        rr = rec[first:first + n_chunks * k_eff].view(n_chunks, k_eff, 2)
+        idx = rr[:, :, 0]
+        assert int(idx.min().item()) >= 0 and int(idx.max().item()) < M, "%s t%d: record index out of range" % (what, t)
+        if k_eff > 1:
+            assert bool(torch.all(idx[:, 1:] > idx[:, :-1]).item()), "%s t%d: indices not strictly ascending" % (what, t)
+        val2 = float(rr[:, :, 1].contiguous().view(torch.float32).double().pow(2).sum().item())
+        lhs = sum_squares(mom_after[t])
+        rhs = energy_before[t] - val2
+        assert abs(lhs - rhs) <= rtol * max(energy_before[t], 1e-300), "%s t%d: energy identity off by %.3e of %.3e" % (
+            what, t, abs(lhs - rhs), energy_before[t])
+        seen += n_chunks * k_eff
+    assert seen == rec.shape[0], "%s: payload holds %d records, the layout accounts for %d" % (what, rec.shape[0], seen)
+    return seen

@@ -573,3 +573,86 @@ def test_explicit_dct_basis_equals_default_and_tensor_driver_takes_a_basis():
     Qs = np.zeros(s * s)
     Qs[c["idx"][0]] = c["val"][0].astype(np.float32)
     assert np.max(np.abs(R - P.T @ Qs.reshape(s, s) @ P)) < 1e-12
+
+
+# --------------------------------------------------------------------------------------------
+# Forced-index continuation of the C oracle (the comparison harness uses it where several top-k
+# sets are valid): with a given index set the residual is B - alpha * IDCT(Q restricted to the set)
+# (Section 2.1 "Momentum Subtraction as Error Feedback"), whatever the magnitudes say.
+# --------------------------------------------------------------------------------------------
+def _forced_case(seed, n, s, rows, k):
+    rng = np.random.default_rng(seed)
+    M = rows * s
+    g = rng.standard_normal((n, M))
+    m = rng.standard_normal((n, M))
+    return g, m, M, min(k, M)
+
+
+@pytest.mark.parametrize("s,rows,k", [(8, 8, 5), (16, 16, 7), (8, 1, 3)])
+def test_forced_index_with_the_oracles_own_set_changes_nothing(s, rows, k):
+    g, m, M, k_eff = _forced_case(11, 5, s, rows, k)
+    beta = 0.9
+    free = orc.compress_chunks(g, m, s, rows, k, beta)
+    forced = orc.compress_chunks(g, m, s, rows, k, beta, forced_idx=free["idx"])
+    assert np.array_equal(forced["idx"], free["idx"])
+    assert np.array_equal(forced["val"], free["val"])
+    assert np.array_equal(forced["m_new"], free["m_new"])  # bit for bit
+    assert np.array_equal(forced["Q"], free["Q"])
+
+
+@pytest.mark.parametrize("alpha", [1.0, 0.25])
+def test_forced_index_with_another_set_follows_the_definition(alpha):
+    s, rows, k, beta = 8, 8, 6, 0.75
+    g, m, M, k_eff = _forced_case(12, 4, s, rows, k)
+    rng = np.random.default_rng(13)
+    # a different, deliberately non-top set per chunk (ascending, unique), different from chunk to chunk
+    sets = np.stack([np.sort(rng.choice(M, size=k_eff, replace=False)) for _ in range(g.shape[0])]).astype(np.int32)
+    out = orc.compress_chunks(g, m, s, rows, k, beta, forced_idx=sets, alpha=alpha)
+    assert np.array_equal(out["idx"], sets)
+    for c in range(g.shape[0]):
+        B = (beta * m[c] + g[c]).reshape(rows, s)
+        Q = scipy.fft.dctn(B, type=2, norm="ortho")
+        assert np.max(np.abs(out["Q"][c].reshape(rows, s) - Q)) < 1e-12
+        keep = np.zeros(M)
+        keep[sets[c]] = Q.reshape(-1)[sets[c]]
+        want = B - alpha * scipy.fft.idctn(keep.reshape(rows, s), type=2, norm="ortho")
+        assert np.max(np.abs(out["m_new"][c].reshape(rows, s) - want)) < 1e-12
+        assert np.max(np.abs(out["val"][c] - Q.reshape(-1)[sets[c]])) < 1e-12
+    # and it is not what the free selection gives (the forced branch was really taken)
+    free = orc.compress_chunks(g, m, s, rows, k, beta, alpha=alpha)
+    assert not np.array_equal(free["idx"], sets)
+    assert np.max(np.abs(free["m_new"] - out["m_new"])) > 1e-3
+
+
+def test_forced_index_tensor_driver_walks_the_sets_chunk_by_chunk():
+    # 2 x 3 chunk grid: a stride or ordering mistake in the per-chunk forced sets would pair a chunk with
+    # its neighbour's set
+    s, k, beta = 8, 4, 0.5
+    rng = np.random.default_rng(14)
+    g = rng.standard_normal((16, 24))
+    m = rng.standard_normal((16, 24))
+    M = s * s
+    sets = np.stack([np.sort(rng.choice(M, size=k, replace=False)) for _ in range(6)]).astype(np.int32)
+    out = orc.compress_tensor(g, m, s, k, beta, forced_idx=sets)
+    assert np.array_equal(out["records"]["idx"], sets)
+    for c in range(6):
+        k0, k1 = divmod(c, 3)  # chunks row-major over the chunk grid
+        B = beta * m[8 * k0:8 * k0 + 8, 8 * k1:8 * k1 + 8] + g[8 * k0:8 * k0 + 8, 8 * k1:8 * k1 + 8]
+        Q = scipy.fft.dctn(B, type=2, norm="ortho")
+        keep = np.zeros(M)
+        keep[sets[c]] = Q.reshape(-1)[sets[c]]
+        want = B - scipy.fft.idctn(keep.reshape(8, 8), type=2, norm="ortho")
+        assert np.max(np.abs(out["m_new"][8 * k0:8 * k0 + 8, 8 * k1:8 * k1 + 8] - want)) < 1e-12
+        assert np.max(np.abs(out["val64"][c] - Q.reshape(-1)[sets[c]])) < 1e-12
+        assert np.array_equal(out["records"]["val"][c], Q.reshape(-1)[sets[c]].astype(np.float32))
+    # 1-D tensor, three segments
+    g1 = rng.standard_normal(24)
+    m1 = rng.standard_normal(24)
+    sets1 = np.stack([np.sort(rng.choice(8, size=3, replace=False)) for _ in range(3)]).astype(np.int32)
+    out1 = orc.compress_tensor(g1, m1, 8, 3, beta, forced_idx=sets1)
+    for c in range(3):
+        b = beta * m1[8 * c:8 * c + 8] + g1[8 * c:8 * c + 8]
+        q = scipy.fft.dct(b, type=2, norm="ortho")
+        keep = np.zeros(8)
+        keep[sets1[c]] = q[sets1[c]]
+        assert np.max(np.abs(out1["m_new"][8 * c:8 * c + 8] - (b - scipy.fft.idct(keep, type=2, norm="ortho")))) < 1e-12
