@@ -340,6 +340,9 @@ def run_ours(args, rank, world):
                        "worker_params_per_s": value * W, "l2": ("inputs (%.1f GB resident in HBM) are larger than the 126 MB L2; no flush needed" % (working_set / 1e9))
                        if flush is None else ("working set %.1f MB: L2 flushed by a 256 MB write before every timed step"
                                               % (working_set / 1e6)), "kernel_path": args.path,
+                       "gradients": "one seeded gradient set per worker, reused every step on purpose (a second set "
+                                    "per worker does not fit beside the %d momenta; the momentum still changes "
+                                    "every step)" % W,
                        "basis": args.basis, "chunk_shape": args.chunk_shape or None,
                        "embedding_active_rows": args.embedding_active_rows or None},
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
@@ -397,6 +400,52 @@ def max_over_ranks(ms: float, dist, device) -> float:
 def replica_throughput(units_per_rank: float, world: int, ms: float) -> float:
     """Whole-job throughput of `world` independent replicas: all units over the slowest rank's time."""
     return world * units_per_rank / (ms * 1e-3)
+
+
+def spawn_ranks(args) -> int:
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script on this node, one per GPU,
+    under torch.distributed.run (rendezvous on 127.0.0.1) and pass their output through.  The ranks stay
+    independent replicas: the process group only carries the barrier and the MAX over ranks of the device time."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def run_standin(args, rank, world):
+    """The launch, rendezvous and reporting path of the N-rank benchmark with a CPU stand-in for the timed region
+    (a gloo group, a short host loop per step): what can be checked of `--gpus N` on a machine without GPUs.
+    Prints the same JSON shape with "standin": "cpu"; never a benchmark number."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    if world > 1:
+        dist.init_process_group("gloo")
+    a = np.random.default_rng(rank).standard_normal((64, 64))
+    for _ in range(args.warmup):
+        a = a @ a.T / 64.0
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        a = a @ a.T / 64.0
+    ms_local = (time.perf_counter() - t0) * 1e3
+    ms = max_over_ranks(ms_local, dist if world > 1 else None, torch.device("cpu")) / args.steps
+    if world > 1:
+        dist.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": replica_throughput(float(a.size), world, ms), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "higher_is_better": True, "scaling": "weak", "standin": "cpu",
+                          "config": {"workload": "launcher check", "parallelism": "replicas only"}}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def run_grid(args):
@@ -470,12 +519,20 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--grid", action="store_true", help="print the stress/ablation grid instead of the benchmark line")
     ap.add_argument("--grid-set", action="store_true", help="with --grid: also run the 1B-class set")
+    ap.add_argument("--standin", default="", choices=["", "cpu"],
+                    help="cpu: run the launcher / rendezvous / reporting path with a host stand-in for the timed "
+                         "region (checks `--gpus N` without GPUs; not a benchmark)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = max(args.warmup, 1)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and "RANK" not in os.environ and not args.grid:
+        # not under a launcher: become one (N ranks, one per GPU; each rank re-enters main() with RANK set)
+        raise SystemExit(spawn_ranks(args))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.grid:
+    if args.standin == "cpu":
+        run_standin(args, rank, world)
+    elif args.grid:
         if rank == 0:
             run_grid(args)
     elif args.impl == "reference":
