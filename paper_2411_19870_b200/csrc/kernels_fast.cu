@@ -743,10 +743,12 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
 
 // Bytes of one decode slot: the tile, the mbarrier and -- for the count-normalised mean -- one
 // 16-bit sender count per coordinate.
+constexpr int STAGE_RECORDS = 512;  // records staged per batch of the scatter (sixteen workers at k <= 32)
 template <int S>
 __host__ __device__ constexpr size_t decode_slot_bytes(bool counts)
 {
-    return ((size_t)S * Cfg<S>::XS * 4 + 16 + (counts ? (size_t)S * S * 2 : 0) + 127) / 128 * 128;
+    return ((size_t)S * Cfg<S>::XS * 4 + 16 + 2 * STAGE_RECORDS * sizeof(DemoRecord) + (counts ? (size_t)S * S * 2 : 0) + 127) /
+           128 * 128;
 }
 
 // SIGNS: the parameter-server form -- sign(R) goes out as int8 per element, the parameters are neither read
@@ -767,7 +769,8 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
     float *St = reinterpret_cast<float *>(smem_raw);  // [S*XS]
     float *Xt = St;                                   // [S*S] (aliases St)
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(St + S * XS);
-    unsigned short *Cn = reinterpret_cast<unsigned short *>(bar_mem + 2);  // [S*S] senders per coordinate (agg == 2)
+    DemoRecord *stage_all = reinterpret_cast<DemoRecord *>(bar_mem + 2);    // [2][STAGE_RECORDS] records of a batch of workers
+    unsigned short *Cn = reinterpret_cast<unsigned short *>(stage_all + 2 * STAGE_RECORDS);  // [S*S] senders per coordinate (agg == 2)
 
     const int t = threadIdx.x % S;
     const uint32_t bar = smem_u32(bar_mem);
@@ -788,10 +791,34 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
     const float decay = 1.f - a.lr * a.wd;
     const float neg_lr_scale = -a.lr * a.agg_scale;
 
+    // The records of a chunk's first batch of workers (up to STAGE_RECORDS records) are copied into one of two
+    // staging buffers by asynchronous copies issued a whole chunk ahead, so that the payload reads of the W
+    // workers -- W small pieces from W buffers -- never stand in front of the scatter.  One copy group per chunk.
+    auto stage_ahead = [&](int buf, long long chunk) {
+        cur.seek(a.entries, a.n_entries, chunk);
+        const int k_n = cur.te.k_eff;
+        if (k_n <= 64) {
+            const long long off_n = cur.te.rec_begin + (chunk - cur.te.chunk_begin) * (long long)k_n;
+            const int sh = (k_n > 32) ? 6 : 5;
+            DemoRecord *dst = stage_all + buf * STAGE_RECORDS;
+#pragma unroll
+            for (int i = 0; i < STAGE_RECORDS / S; ++i) {
+                const int r = i * S + t, wl = r >> sh, j = r & ((1 << sh) - 1);
+                if (wl < a.W && j < k_n)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst + r)),
+                                 "l"(a.payloads[wl] + off_n + j)
+                                 : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
     const long long stride = (long long)gridDim.x * NCH;
     long long c = (long long)blockIdx.x * NCH + slot;
+    int buf = 0;
+    if (c < a.n_chunks) stage_ahead(0, c);
     for (long long cb = (long long)blockIdx.x * NCH; cb < a.n_chunks; cb += stride, c += stride) {
-        if (__syncthreads_or(failed)) return;  // all slots start a chunk together (shared instruction stream)
+        if (__syncthreads_or(failed)) break;  // all slots start a chunk together (shared instruction stream)
         if (c >= a.n_chunks) continue;
         cur.seek(a.entries, a.n_entries, c);
         const DemoTensorEntry te = cur.te;
@@ -822,28 +849,94 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
             if (counts)
                 for (int v = 0; v < S; ++v) Cn[t * S + v] = 0;
         }
-        sb.sync();
-        // S = sum over workers in worker order; a barrier per worker fixes the order of additions.
-        // Records are fetched eight workers ahead so that one memory latency covers eight workers.
-        for (int kb = 0; kb < k_eff; kb += S) {
-            const bool mine = kb + t < k_eff;
-            for (int w0 = 0; w0 < a.W; w0 += 8) {
-                DemoRecord r[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (mine && w0 + j < a.W) r[j] = a.payloads[w0 + j][rec_off + kb + t];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (w0 + j < a.W) {
-                        if (mine) {
-                            if ((unsigned)r[j].idx < (unsigned)M) {
-                                St[(r[j].idx >> C::LOG2S) * XS + (r[j].idx & (S - 1))] += r[j].val;
-                                if (counts) Cn[r[j].idx] += 1;
-                            } else {
-                                atomicMax(a.status, DEMO_DEV_PAYLOAD);
+        // next chunk's records on their way (the cursor moves on; this chunk's table entry is in `te`)
+        if (c + stride < a.n_chunks)
+            stage_ahead(buf ^ 1, c + stride);
+        else
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 1;" ::: "memory");  // this chunk's copies have landed
+        DemoRecord *stage = stage_all + buf * STAGE_RECORDS;
+        buf ^= 1;
+        // S = sum over workers in worker order (Decompress&Aggregate).
+        if (k_eff <= 64) {
+            // Every warp owns the 32 rows of the tile its threads cleared and will transform (rows 32 w .. 32 w + 31
+            // for warp w of the slot).  The records of up to sixteen workers (512 records) are staged in shared
+            // memory with one round of global loads; then every warp walks the staged workers in order, reads ALL
+            // records of a worker (lane j: record j, and j + 32 where k > 32) and adds those that fall into its rows.
+            // A coordinate is only ever touched by one warp, so the order of the additions -- worker after worker,
+            // hence bit-reproducible -- needs nothing but warp-level synchronisation.
+            const int lane = t & 31, warp = t >> 5;
+            const int sh = (k_eff > 32) ? 6 : 5;          // a worker's records take 32 or 64 staging entries
+            const int wb = STAGE_RECORDS >> sh;           // workers per batch: 16 or 8
+            for (int w0 = 0; w0 < a.W; w0 += wb) {
+                if (w0 > 0) {  // further batches of a large fan-in: fetched on the spot
+                    sb.sync();  // the previous batch has been consumed by both warps
+#pragma unroll 1
+                    for (int r = t; r < STAGE_RECORDS; r += S) {
+                        const int wl = r >> sh, j = r & ((1 << sh) - 1);
+                        if (w0 + wl < a.W && j < k_eff) stage[r] = a.payloads[w0 + wl][rec_off + j];
+                    }
+                }
+                sb.sync();  // staged records visible (also orders the clearing of the tile before the first additions)
+                const int nw = min(wb, a.W - w0);
+                // (the next worker's record is read before this worker's addition, so that only the addition itself
+                // lies between two warp barriers)
+                const bool two = k_eff > 32;
+                DemoRecord nx0 = stage[lane], nx1 = stage[two ? lane + 32 : lane];
+#pragma unroll 1
+                for (int wl = 0; wl < nw; ++wl) {
+                    const DemoRecord rc0 = nx0, rc1 = nx1;
+                    if (wl + 1 < nw) {
+                        nx0 = stage[((wl + 1) << sh) + lane];
+                        if (two) nx1 = stage[((wl + 1) << sh) + lane + 32];
+                    }
+                    if (lane < k_eff) {
+                        if ((unsigned)rc0.idx < (unsigned)M) {
+                            if ((rc0.idx >> (C::LOG2S + 5)) == warp) {
+                                St[(rc0.idx >> C::LOG2S) * XS + (rc0.idx & (S - 1))] += rc0.val;
+                                if (counts) Cn[rc0.idx] += 1;
                             }
+                        } else {
+                            atomicMax(a.status, DEMO_DEV_PAYLOAD);
                         }
-                        sb.sync();
+                    }
+                    if (two && lane + 32 < k_eff) {
+                        if ((unsigned)rc1.idx < (unsigned)M) {
+                            if ((rc1.idx >> (C::LOG2S + 5)) == warp) {
+                                St[(rc1.idx >> C::LOG2S) * XS + (rc1.idx & (S - 1))] += rc1.val;
+                                if (counts) Cn[rc1.idx] += 1;
+                            }
+                        } else {
+                            atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+        } else {
+            // k > 64: a thread's records may fall into any row; a barrier per worker fixes the order of additions.
+            // Records are fetched eight workers ahead so that one memory latency covers eight workers.
+            sb.sync();
+            for (int kb = 0; kb < k_eff; kb += S) {
+                const bool mine = kb + t < k_eff;
+                for (int w0 = 0; w0 < a.W; w0 += 8) {
+                    DemoRecord r[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (mine && w0 + j < a.W) r[j] = a.payloads[w0 + j][rec_off + kb + t];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (w0 + j < a.W) {
+                            if (mine) {
+                                if ((unsigned)r[j].idx < (unsigned)M) {
+                                    St[(r[j].idx >> C::LOG2S) * XS + (r[j].idx & (S - 1))] += r[j].val;
+                                    if (counts) Cn[r[j].idx] += 1;
+                                } else {
+                                    atomicMax(a.status, DEMO_DEV_PAYLOAD);
+                                }
+                            }
+                            sb.sync();
+                        }
                     }
                 }
             }
@@ -925,6 +1018,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
         }
         sb.sync();  // the tile is free again
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");  // no copy of this thread may outlive the CTA's shared memory
 }
 
 // CTA sizes: the compress kernel runs best with all eight slots of an SM in one CTA (one shared
