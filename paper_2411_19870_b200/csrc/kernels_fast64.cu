@@ -43,7 +43,7 @@ template <typename GT>
 constexpr size_t region_bytes()
 {
     constexpr size_t stage = (size_t)S * S * (sizeof(float) + sizeof(GT));
-    constexpr size_t need = (size_t)S * XS * sizeof(float) + (size_t)(WCAP + 4) * 8;  // tile + wide list
+    constexpr size_t need = (size_t)S * XS * sizeof(float) + (size_t)(WCAP + 4) * 8 + 256 * 8;  // tile + wide list + big-k list
     return stage > need ? stage : need;
 }
 template <typename GT>
@@ -66,6 +66,7 @@ struct SlotMem {
     unsigned *misc;      // [16]
     unsigned *wkey;      // [WCAP + 4] wide list, behind the tile
     unsigned *widx;      // [WCAP + 4]
+    uint2 *rbig;         // [256] kept records for 64 < k <= 256: (row << 16 | column, alpha * value), behind the wide list
 };
 
 // 64 / 32 consecutive fp32 columns of this thread's tensor-memory lane.
@@ -105,7 +106,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 // ------------------------------------------------------------------------------------------------
 // Out-of-line selection for the chunks the in-line path does not take: more than 64 candidates in a
 // warp's list (tiles of low rank or with a concentrated spectrum, tied or degenerate chunks), fewer
-// candidates than k (NaN coefficients) or k > 64.  Works from the coefficient tile in X (row t is
+// candidates than k (NaN coefficients) or k > 64 (for 64 < k <= 256 the bound comes from step 2 alone).  Works from the coefficient tile in X (row t is
 // this thread's), writes the records to `rec` and, for k <= 64, the pre-decoded list for the row stage.
 //   1. wide list: up to WCAP candidates under the bound `lmin` (the k-th largest of the 64 row maxima),
 //      every warp takes the whole list into registers and finds the exact k-th largest key by a
@@ -125,9 +126,9 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
     sb.sync();  // the coefficient tile is complete; the in-line path is done with its lists
 
     bool done = false;
-    if (bound_valid && k_eff <= S) {
+    if (k_eff <= 256) {  // (the finer bound below needs at least k groups: 256 quarter rows / quarter columns)
         unsigned long long mask = 0ull;
-        unsigned off = 0, n_all = 0;
+        unsigned off = 0, n_all = 0xffffffffu;
         auto count_under = [&](unsigned bound) {
             mask = 0ull;
 #pragma unroll 4
@@ -141,7 +142,10 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
             n_all = n0 + misc[1];
             off = inc - cnt + (warp ? n0 : 0u);
         };
-        count_under(lmin_w);
+        if (bound_valid)
+            count_under(lmin_w);
+        else
+            lmin_w = 0u;  // k > 64: the row maxima give no bound, the finer partition does
         if (n_all > (unsigned)WCAP) {
             // tighter bound: the k_eff-th largest of the 256 quarter-row maxima and of the 256 quarter-column maxima
             unsigned rk[4], ck[4];
@@ -156,11 +160,15 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                 }
                 rk[g] = m;
             }
+            // (the quarter-column maxima matter for tiles with a few active columns; with k > 64, where this is the
+            // ordinary path of every chunk, the quarter rows alone give the bound)
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 unsigned m = 0u;
+                if (bound_valid) {
 #pragma unroll 4
-                for (int u = 0; u < 16; ++u) m = max(m, mag_key(X[(16 * g + u) * XS + t]));
+                    for (int u = 0; u < 16; ++u) m = max(m, mag_key(X[(16 * g + u) * XS + t]));
+                }
                 ck[g] = m;
             }
             unsigned *gq = sm.wkey;  // [8][64], behind the tile
@@ -199,9 +207,10 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                 }
                 return pre;
             };
-            const unsigned l2 = max(kth_of_256(rk, prk), kth_of_256(ck, pck));
+            unsigned l2 = kth_of_256(rk, prk);
+            if (bound_valid) l2 = max(l2, kth_of_256(ck, pck));
             sb.sync();  // gq is read; the wide list may overwrite it
-            if (l2 > lmin_w) {
+            if (l2 > lmin_w || !bound_valid) {
                 lmin_w = l2;
                 count_under(lmin_w);
             }
@@ -232,13 +241,17 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                 hi = __reduce_max_sync(0xffffffffu, hi);
                 const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
                 unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+                unsigned n_ge = n_all;  // every entry is >= the bound >= thr; the search stops at exactly k_eff
 #pragma unroll 1
-                for (int b = wb0; b >= 0; --b) {
+                for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
                     const unsigned cand = thr | (1u << b);
                     unsigned cnt = 0;
 #pragma unroll
                     for (int j = 0; j < WK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
-                    thr = (cnt >= (unsigned)k_eff) ? cand : thr;
+                    if (cnt >= (unsigned)k_eff) {
+                        thr = cand;
+                        n_ge = cnt;
+                    }
                 }
                 unsigned n_gt = 0;
 #pragma unroll
@@ -261,7 +274,10 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                             const int uo = (r.idx >> LOG2S) * XS;
                             r.val = X[uo + v];
                             rec[pos] = r;
-                            recs4[pos] = make_int4(uo, v * S, __float_as_int(alpha * r.val), 0);
+                            if (k_eff <= 64)
+                                recs4[pos] = make_int4(uo, v * S, __float_as_int(alpha * r.val), 0);
+                            else
+                                sm.rbig[pos] = make_uint2(((unsigned)r.idx >> LOG2S) << 16 | (unsigned)v, __float_as_uint(alpha * r.val));
                         }
                     }
                     gt_before += __popc(gtb);
@@ -316,9 +332,10 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                 r.idx = t * S + v;
                 r.val = val;
                 rec[pos] = r;
-                if (k_eff <= 64) {
+                if (k_eff <= 64)
                     recs4[pos] = make_int4(t * XS, v * S, __float_as_int(alpha * val), 0);
-                }
+                else if (k_eff <= 256)
+                    sm.rbig[pos] = make_uint2((unsigned)t << 16 | (unsigned)v, __float_as_uint(alpha * val));
             }
         }
     }
@@ -342,6 +359,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     sm.X = Ms;
     sm.wkey = reinterpret_cast<unsigned *>(sm.raw + (size_t)S * XS * sizeof(float));
     sm.widx = sm.wkey + WCAP + 4;
+    sm.rbig = reinterpret_cast<uint2 *>(sm.widx + WCAP + 4);
     sm.tmax = reinterpret_cast<float *>(sm.raw + region_bytes<GT>());
     sm.cand_idx = reinterpret_cast<int *>(sm.tmax + S);
     sm.cand_val = reinterpret_cast<float *>(sm.cand_idx + CAP + 8);
@@ -727,17 +745,45 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                             }
                         }
                     } else {
+                        // k > 64: up to 256 kept records come from a compact shared list, more from the payload
+                        // itself; four cosines are fetched ahead
+                        const bool listed = k_eff <= 256;
                         int cur_u = -1;
 #pragma unroll 1
-                        for (int r = 0; r < k_eff; ++r) {
-                            const DemoRecord rc = rec[r];
-                            const int u = (rc.idx >> LOG2S) * XS, v = rc.idx & (S - 1);
-                            if (u != cur_u) {
-                                if (cur_u >= 0) X[cur_u + t] = acc;
-                                acc = 0.f;
-                                cur_u = u;
+                        for (int r0 = 0; r0 < k_eff; r0 += 4) {
+                            int u[4];
+                            float z[4], cv[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                u[j] = -1;
+                                z[j] = 0.f;
+                                int v = 0;
+                                if (r0 + j < k_eff) {
+                                    if (listed) {
+                                        const uint2 e = sm.rbig[r0 + j];
+                                        u[j] = (int)(e.x >> 16) * XS;
+                                        v = (int)(e.x & 0xffffu);
+                                        z[j] = __uint_as_float(e.y);
+                                    } else {
+                                        const DemoRecord rc = rec[r0 + j];
+                                        u[j] = (rc.idx >> LOG2S) * XS;
+                                        v = rc.idx & (S - 1);
+                                        z[j] = a.alpha * rc.val;
+                                    }
+                                }
+                                cv[j] = __ldg(Ct + v * S);
                             }
-                            acc = fmaf(a.alpha * rc.val, __ldg(Ct + v * S), acc);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                if (u[j] >= 0) {
+                                    if (u[j] != cur_u) {
+                                        if (cur_u >= 0) X[cur_u + t] = acc;
+                                        acc = 0.f;
+                                        cur_u = u[j];
+                                    }
+                                    acc = fmaf(z[j], cv[j], acc);
+                                }
+                            }
                         }
                         if (cur_u >= 0) X[cur_u + t] = acc;
                     }
