@@ -39,17 +39,23 @@ constexpr int WCAP = 512;     // capacity of the wide candidate list (out-of-lin
 constexpr int TMEM_COLS_PER_GROUP = 64;  // one column block per four warps (two slots)
 constexpr int PAD_ROW = 0x40000000;      // row offset of the padding entries of the row-stage list (never stored to)
 
+// Tile area of a slot:  [0, 64*68*4)  the padded transpose / coefficient / row-stage tile X; its first 16 KB double as
+// the landing area of the m tile and as the source of the TMA store of the new momentum;  behind it the landing
+// area of the g tile, which between its two uses holds the lists of the selection: wide candidate list, big-k list, and -- at its
+// end -- the row-stage list.
+constexpr size_t TILE_X_BYTES = (size_t)S * XS * sizeof(float);
 template <typename GT>
 constexpr size_t region_bytes()
 {
-    constexpr size_t stage = (size_t)S * S * (sizeof(float) + sizeof(GT));
-    constexpr size_t need = (size_t)S * XS * sizeof(float) + (size_t)(WCAP + 4) * 8 + 256 * 8;  // tile + wide list + big-k list
-    return stage > need ? stage : need;
+    constexpr size_t g_bytes = (size_t)S * S * sizeof(GT);
+    constexpr size_t lists = (size_t)(WCAP + 4) * 8 + 256 * 8 + 65 * 16;  // wide list + big-k list + row-stage list
+    static_assert(lists <= g_bytes, "the selection's lists live in the g landing area");
+    return TILE_X_BYTES + g_bytes;
 }
 template <typename GT>
 constexpr size_t slot_bytes()
 {
-    constexpr size_t raw = region_bytes<GT>() + S * 4 + (CAP + 8) * 3 * 4 + 65 * 16 + 16 * 4 + 16;
+    constexpr size_t raw = region_bytes<GT>() + S * 4 + (CAP + 8) * 3 * 4 + 16 * 4 + 16;
     return (raw + 127) / 128 * 128;
 }
 
@@ -354,10 +360,10 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     const int slot = threadIdx.x / S;
     SlotMem sm;
     sm.raw = smem_all + (size_t)slot * slot_bytes<GT>();
-    float *Ms = reinterpret_cast<float *>(sm.raw);   // [S*S] m tile
-    GT *Gs = reinterpret_cast<GT *>(Ms + S * S);     // [S*S] g tile
+    float *Ms = reinterpret_cast<float *>(sm.raw);             // [S*S] m tile
+    GT *Gs = reinterpret_cast<GT *>(sm.raw + TILE_X_BYTES);    // [S*S] g tile
     sm.X = Ms;
-    sm.wkey = reinterpret_cast<unsigned *>(sm.raw + (size_t)S * XS * sizeof(float));
+    sm.wkey = reinterpret_cast<unsigned *>(sm.raw + TILE_X_BYTES);
     sm.widx = sm.wkey + WCAP + 4;
     sm.rbig = reinterpret_cast<uint2 *>(sm.widx + WCAP + 4);
     sm.tmax = reinterpret_cast<float *>(sm.raw + region_bytes<GT>());
@@ -365,8 +371,8 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     sm.cand_val = reinterpret_cast<float *>(sm.cand_idx + CAP + 8);
     sm.cand_key = reinterpret_cast<unsigned *>(sm.cand_val + CAP + 8);
     sm.hist = reinterpret_cast<unsigned *>(sm.cand_idx);
-    sm.recs4 = reinterpret_cast<int4 *>(sm.cand_key + CAP + 8);
-    sm.misc = reinterpret_cast<unsigned *>(sm.recs4 + 65);
+    sm.recs4 = reinterpret_cast<int4 *>(sm.raw + region_bytes<GT>()) - 65;
+    sm.misc = reinterpret_cast<unsigned *>(sm.cand_key + CAP + 8);
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(sm.misc + 16);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_all + (size_t)NCH * slot_bytes<GT>());
     float *X = sm.X;
