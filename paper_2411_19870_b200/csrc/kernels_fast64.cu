@@ -37,7 +37,7 @@ constexpr int CAPW = CAP / 2;
 constexpr int CAPWP = CAPW + 4;
 constexpr int WCAP = 512;     // capacity of the wide candidate list (out-of-line path)
 constexpr int TMEM_COLS_PER_GROUP = 64;  // one column block per four warps (two slots)
-constexpr int PAD_ROW = 0x40000000;      // row offset of the padding entries of the row-stage list (never stored to)
+constexpr int ROW_AHEAD = 8;              // entries of the row-stage list fetched ahead
 
 // Tile area of a slot:  [0, 64*68*4)  the padded transpose / coefficient / row-stage tile X; its first 16 KB double as
 // the landing area of the m tile and as the source of the TMA store of the new momentum;  behind it the landing
@@ -383,6 +383,8 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     int4 *recs4 = sm.recs4;
     unsigned *misc = sm.misc;
 
+    // "row" of the padding entries of the row-stage list: the scratch line tmax[0..S) seen from X
+    constexpr int PAD_ROW = (int)(region_bytes<GT>() / sizeof(float));
     const int t = threadIdx.x % S, lane = t & 31, warp = t >> 5;
     const int hw_warp = threadIdx.x >> 5;
     const SlotBarrier<S> sb{slot + 1};
@@ -725,29 +727,28 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                     const float *Ct = a.C + t;
                     float acc = 0.f;
                     if (k_eff <= 64) {
-                        // The list is padded with zero-valued entries of row PAD_ROW (entry 64 is always one).  A row's
-                        // sum is stored when the next entry belongs to another row; padding follows padding, so the
-                        // padding row itself is never stored.  Four entries and their cosines are fetched ahead of the
+                        // The running sum of a row is stored after every entry (the last store of a row carries the
+                        // whole sum) and starts again from zero when the next entry belongs to another row: no branch in
+                        // the loop.  The list is padded with zero-valued entries (entry 64 is always one) whose "row" is
+                        // a scratch line outside the tile.  Entries and their cosines are fetched ahead of the
                         // dependent accumulation.
                         float *Xt = X + t;
                         int4 nx = recs4[0];
 #pragma unroll 1
-                        for (int r0 = 0; r0 < k_eff; r0 += 4) {
-                            int4 rc[5];
-                            float cv[4];
+                        for (int r0 = 0; r0 < k_eff; r0 += ROW_AHEAD) {
+                            int4 rc[ROW_AHEAD + 1];
+                            float cv[ROW_AHEAD];
                             rc[0] = nx;
 #pragma unroll
-                            for (int j = 1; j < 5; ++j) rc[j] = recs4[r0 + j];
-                            nx = rc[4];
+                            for (int j = 1; j < ROW_AHEAD + 1; ++j) rc[j] = recs4[r0 + j];
+                            nx = rc[ROW_AHEAD];
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) cv[j] = __ldg(Ct + rc[j].y);
+                            for (int j = 0; j < ROW_AHEAD; ++j) cv[j] = __ldg(Ct + rc[j].y);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
+                            for (int j = 0; j < ROW_AHEAD; ++j) {
                                 acc = fmaf(__int_as_float(rc[j].z), cv[j], acc);
-                                if (rc[j].x != rc[j + 1].x) {
-                                    Xt[rc[j].x] = acc;
-                                    acc = 0.f;
-                                }
+                                Xt[rc[j].x] = acc;
+                                acc = (rc[j].x != rc[j + 1].x) ? 0.f : acc;
                             }
                         }
                     } else {
