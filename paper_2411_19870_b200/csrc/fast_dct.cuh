@@ -271,4 +271,274 @@ FDCT_HD void dct3_post(const float (&y)[N], float (&x)[N])
     inv_cascade<1, N>(e, y, x);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Two floats per operation.  sm_100 adds packed fp32 arithmetic (add / sub on a register pair, one issue
+// slot for two results, each result rounded exactly like the scalar operation).  A kernel whose limit is
+// instruction issue gains from it wherever two values go through the same addition at the same time:
+//   * the two half-size DCT-II inside every DCT-IV work on independent vectors a and b: they run as ONE
+//     transform over pairs (a[n], b[n]); nested DCT-IV blocks rotate each half of a pair by scalar
+//     operations (the rotation constants would otherwise need register pairs of their own) and hand the
+//     four resulting vectors on as two vectors of pairs;
+//   * the butterfly cascades work on pairs of neighbouring elements, stored (x[2p], x[2p+1]) for even p
+//     and swapped for odd p: the partner pair of pair j at a level of L elements is pair L/2-1-j, whose
+//     swapped order is exactly the mirror image, and sums and differences come out in the same
+//     alternating order for the next level.
+// On the host the pair is two floats and the operations are the scalar ones (same results bit for bit).
+// ------------------------------------------------------------------------------------------------
+struct F2 {
+#if defined(__CUDA_ARCH__)
+    unsigned long long v;
+#else
+    float lo, hi;
+#endif
+};
+FDCT_HD F2 f2_make(float lo, float hi)
+{
+    F2 r;
+#if defined(__CUDA_ARCH__)
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+#else
+    r.lo = lo;
+    r.hi = hi;
+#endif
+    return r;
+}
+FDCT_HD float f2_lo(F2 a)
+{
+#if defined(__CUDA_ARCH__)
+    float lo;
+    asm("{\n\t.reg .b32 t;\n\tmov.b64 {%0, t}, %1;\n\t}" : "=f"(lo) : "l"(a.v));
+    return lo;
+#else
+    return a.lo;
+#endif
+}
+FDCT_HD float f2_hi(F2 a)
+{
+#if defined(__CUDA_ARCH__)
+    float hi;
+    asm("{\n\t.reg .b32 t;\n\tmov.b64 {t, %0}, %1;\n\t}" : "=f"(hi) : "l"(a.v));
+    return hi;
+#else
+    return a.hi;
+#endif
+}
+FDCT_HD F2 f2_add(F2 a, F2 b)
+{
+    F2 r;
+#if defined(__CUDA_ARCH__)
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+#else
+    r.lo = a.lo + b.lo;
+    r.hi = a.hi + b.hi;
+#endif
+    return r;
+}
+FDCT_HD F2 f2_sub(F2 a, F2 b)
+{
+    F2 r;
+#if defined(__CUDA_ARCH__)
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+#else
+    r.lo = a.lo - b.lo;
+    r.hi = a.hi - b.hi;
+#endif
+    return r;
+}
+
+template <int N, class SC>
+FDCT_HD void dct4v(const F2 (&v)[N], F2 (&V)[N]);
+
+// DCT-II of two independent vectors at once (one in each half of the pairs); same scaling as dct2.
+template <int N, class SC>
+FDCT_HD void dct2v(const F2 (&x)[N], F2 (&X)[N])
+{
+    if constexpr (N == 1) {
+        X[0] = x[0];
+    } else {
+        constexpr int H = N / 2;
+        F2 u[H], v[H], E[H], O[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            u[n] = f2_add(x[n], x[N - 1 - n]);
+            v[n] = f2_sub(x[n], x[N - 1 - n]);
+        });
+        dct2v<H, SC>(u, E);
+        dct4v<H, SC>(v, O);
+        static_for<0, H>([&](auto i) {
+            constexpr int j = decltype(i)::value;
+            X[2 * j] = E[j];
+            X[2 * j + 1] = O[j];
+        });
+    }
+}
+
+// DCT-IV of two independent vectors at once; same scaling as dct4.
+template <int N, class SC>
+FDCT_HD void dct4v(const F2 (&v)[N], F2 (&V)[N])
+{
+    if constexpr (N == 1) {
+        constexpr float c = (float)(SC::value * c_cos(kPi / 4.0));
+        V[0] = f2_make(f2_lo(v[0]) * c, f2_hi(v[0]) * c);
+    } else {
+        constexpr int H = N / 2;
+        F2 a[H], b[H], A[H], Bt[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            constexpr double th = (2.0 * n + 1.0) * kPi / (4.0 * N);
+            constexpr double sg = (n % 2 == 0) ? 1.0 : -1.0;
+            constexpr float c = (float)(SC::value * c_cos(th));
+            constexpr float s = (float)(SC::value * c_sin(th));
+            constexpr float cb = (float)(SC::value * sg * c_cos(th));
+            constexpr float sb = (float)(SC::value * sg * c_sin(th));
+            const float l0 = f2_lo(v[n]), h0 = f2_lo(v[N - 1 - n]);
+            const float l1 = f2_hi(v[n]), h1 = f2_hi(v[N - 1 - n]);
+            a[n] = f2_make(fmaf(h0, s, l0 * c), fmaf(h1, s, l1 * c));
+            b[n] = f2_make(fmaf(h0, cb, -(l0 * sb)), fmaf(h1, cb, -(l1 * sb)));
+        });
+        dct2v<H, ScaleOne>(a, A);
+        dct2v<H, ScaleOne>(b, Bt);
+        V[0] = A[0];
+        V[N - 1] = f2_make(-f2_lo(Bt[0]), -f2_hi(Bt[0]));
+        static_for<1, H>([&](auto i) {
+            constexpr int p = decltype(i)::value;
+            V[2 * p - 1] = f2_sub(A[p], Bt[H - p]);
+            V[2 * p] = f2_add(A[p], Bt[H - p]);
+        });
+    }
+}
+
+// dct4 with its two half-size DCT-II run as one transform over pairs (a[n], b[n]).
+template <int N, class SC>
+FDCT_HD void dct4_paired(const float (&v)[N], float (&V)[N])
+{
+    if constexpr (N <= 2) {
+        dct4<N, SC>(v, V);
+    } else {
+        constexpr int H = N / 2;
+        F2 ab[H], AB[H];
+        static_for<0, H>([&](auto i) {
+            constexpr int n = decltype(i)::value;
+            constexpr double th = (2.0 * n + 1.0) * kPi / (4.0 * N);
+            constexpr double sg = (n % 2 == 0) ? 1.0 : -1.0;
+            constexpr float c = (float)(SC::value * c_cos(th));
+            constexpr float s = (float)(SC::value * c_sin(th));
+            constexpr float cb = (float)(SC::value * sg * c_cos(th));
+            constexpr float sb = (float)(SC::value * sg * c_sin(th));
+            const float lo = v[n], hi = v[N - 1 - n];
+            ab[n] = f2_make(fmaf(hi, s, lo * c), fmaf(hi, cb, -(lo * sb)));
+        });
+        dct2v<H, ScaleOne>(ab, AB);
+        V[0] = f2_lo(AB[0]);
+        V[N - 1] = -f2_hi(AB[0]);
+        static_for<1, H>([&](auto i) {
+            constexpr int p = decltype(i)::value;
+            V[2 * p - 1] = f2_lo(AB[p]) - f2_hi(AB[H - p]);
+            V[2 * p] = f2_lo(AB[p]) + f2_hi(AB[H - p]);
+        });
+    }
+}
+
+template <int H, int N, class SC>
+FDCT_HD void core_blocks_paired(const float (&w)[N], float (&y)[N])
+{
+    float v[H], V[H];
+    static_for<0, H>([&](auto i) { v[decltype(i)::value] = w[H + decltype(i)::value]; });
+    dct4_paired<H, SC>(v, V);
+    static_for<0, H>([&](auto i) { y[H + decltype(i)::value] = V[decltype(i)::value]; });
+    if constexpr (H > 1) core_blocks_paired<H / 2, N, SC>(w, y);
+}
+// dct_core_ortho with packed arithmetic (same results).
+template <int N>
+FDCT_HD void dct_core_ortho_paired(const float (&w)[N], float (&y)[N])
+{
+    y[0] = w[0] * dc_scale<N>();
+    core_blocks_paired<N / 2, N, ScaleOrtho<N>>(w, y);
+}
+
+// Forward cascade on pairs of neighbours: a level of L elements is L/2 pairs, pair p = (e[2p], e[2p+1]) for even p and
+// (e[2p+1], e[2p]) for odd p.
+template <int L, int N>
+FDCT_HD void fwd_cascade_paired(const F2 (&e)[L / 2], float (&w)[N])
+{
+    if constexpr (L == 2) {
+        w[0] = f2_lo(e[0]) + f2_hi(e[0]);
+        w[1] = f2_lo(e[0]) - f2_hi(e[0]);
+    } else {
+        constexpr int Q = L / 4;  // pairs of the next level
+        F2 s[Q];
+        static_for<0, Q>([&](auto i) {
+            constexpr int j = decltype(i)::value;
+            s[j] = f2_add(e[j], e[L / 2 - 1 - j]);
+            const F2 d = f2_sub(e[j], e[L / 2 - 1 - j]);
+            w[L / 2 + 2 * j] = (j % 2 == 0) ? f2_lo(d) : f2_hi(d);
+            w[L / 2 + 2 * j + 1] = (j % 2 == 0) ? f2_hi(d) : f2_lo(d);
+        });
+        fwd_cascade_paired<L / 2, N>(s, w);
+    }
+}
+template <int N>
+FDCT_HD void dct2_pre_paired(const float (&x)[N], float (&w)[N])
+{
+    F2 e[N / 2];
+    static_for<0, N / 2>([&](auto i) {
+        constexpr int p = decltype(i)::value;
+        e[p] = (p % 2 == 0) ? f2_make(x[2 * p], x[2 * p + 1]) : f2_make(x[2 * p + 1], x[2 * p]);
+    });
+    fwd_cascade_paired<N, N>(e, w);
+}
+
+// Inverse cascade on pairs: e holds H elements as H/2 pairs in the alternating order.
+template <int H, int N>
+FDCT_HD void inv_cascade_paired(const F2 (&e)[H / 2], const float (&y)[N], float (&x)[N])
+{
+    if constexpr (H == N) {
+        static_for<0, N / 2>([&](auto i) {
+            constexpr int p = decltype(i)::value;
+            x[2 * p] = (p % 2 == 0) ? f2_lo(e[p]) : f2_hi(e[p]);
+            x[2 * p + 1] = (p % 2 == 0) ? f2_hi(e[p]) : f2_lo(e[p]);
+        });
+    } else {
+        F2 f[H];  // 2H elements
+        static_for<0, H / 2>([&](auto i) {
+            constexpr int j = decltype(i)::value;
+            const F2 yy = (j % 2 == 0) ? f2_make(y[H + 2 * j], y[H + 2 * j + 1]) : f2_make(y[H + 2 * j + 1], y[H + 2 * j]);
+            f[j] = f2_add(e[j], yy);
+            f[H - 1 - j] = f2_sub(e[j], yy);
+        });
+        inv_cascade_paired<2 * H, N>(f, y, x);
+    }
+}
+template <int N>
+FDCT_HD void dct3_post_paired(const float (&y)[N], float (&x)[N])
+{
+    const F2 e[1] = {f2_make(y[0] + y[1], y[0] - y[1])};
+    inv_cascade_paired<2, N>(e, y, x);
+}
+// The same with the result left in pairs: xp[p] = (x[2p], x[2p+1]) for even p, (x[2p+1], x[2p]) for odd p.
+template <int H, int N>
+FDCT_HD void inv_cascade_pairs(const F2 (&e)[H / 2], const float (&y)[N], F2 (&xp)[N / 2])
+{
+    if constexpr (H == N) {
+        static_for<0, N / 2>([&](auto i) { xp[decltype(i)::value] = e[decltype(i)::value]; });
+    } else {
+        F2 f[H];
+        static_for<0, H / 2>([&](auto i) {
+            constexpr int j = decltype(i)::value;
+            const F2 yy = (j % 2 == 0) ? f2_make(y[H + 2 * j], y[H + 2 * j + 1]) : f2_make(y[H + 2 * j + 1], y[H + 2 * j]);
+            f[j] = f2_add(e[j], yy);
+            f[H - 1 - j] = f2_sub(e[j], yy);
+        });
+        inv_cascade_pairs<2 * H, N>(f, y, xp);
+    }
+}
+template <int N>
+FDCT_HD void dct3_post_pairs(const float (&y)[N], F2 (&xp)[N / 2])
+{
+    const F2 e[1] = {f2_make(y[0] + y[1], y[0] - y[1])};
+    inv_cascade_pairs<2, N>(e, y, xp);
+}
+// Position of element v in the "pair order" (neighbours of odd pairs swapped); its own inverse.
+constexpr int pair_order(int v) { return v ^ ((v >> 1) & 1); }
+
 }  // namespace fdct

@@ -463,6 +463,10 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
         const TileRef mine = next;
         const long long nc = c + stride;
         if (nc < a.n_chunks) next = locate(nc);
+        if (nc < a.n_chunks && t == 0) {  // pull the next chunk's tiles into L2 while this chunk is processed
+            tma_prefetch_2d(next.tm_m, next.x, next.y);
+            tma_prefetch_2d(next.tm_g, next.x, next.y);
+        }
 
         // Three passes through one copy of the transform core: 0 = DCT-II down column t of B = beta*m + g,
         // 1 = DCT-II along row t (followed by the selection and the sparse row stage of the inverse),
@@ -475,7 +479,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 if (ph == 0) {
 #pragma unroll
                     for (int i = 0; i < S; ++i) x[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
-                    tmem_st64(taddr, x);  // B = beta*m + g, parked for the residual
+                    // B = beta*m + g, parked for the residual; column k of the tensor-memory lane takes element
+                    // pair_order(k), so that the registers of the store are those of the cascade's pairs
+                    float xp[S];
+                    fdct::static_for<0, S>([&](auto i) { xp[decltype(i)::value] = x[fdct::pair_order(decltype(i)::value)]; });
+                    tmem_st64(taddr, xp);
                     // every thread has consumed its column of the staged tiles (X aliases them)
                     if (!sb.sync_and(arrived)) {
                         if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
@@ -486,15 +494,15 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 } else {
                     const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
 #pragma unroll
-                    for (int v4 = 0; v4 < S / 4; ++v4) {
+                    for (int v4 = 0; v4 < S / 4; ++v4) {  // (pass 0 stored the rows in pair order)
                         const float4 f = row[v4];
                         x[4 * v4 + 0] = f.x;
                         x[4 * v4 + 1] = f.y;
-                        x[4 * v4 + 2] = f.z;
-                        x[4 * v4 + 3] = f.w;
+                        x[4 * v4 + 3] = f.z;
+                        x[4 * v4 + 2] = f.w;
                     }
                 }
-                fdct::dct2_pre<S>(x, w);
+                fdct::dct2_pre_paired<S>(x, w);
             } else {
                 // column t of the row-stage tile was written by this thread only: no barrier before reading it
                 fdct::static_for<0, S>([&](auto i) {
@@ -503,12 +511,15 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 });
             }
 
-            fdct::dct_core_ortho<S>(w, y);
+            fdct::dct_core_ortho_paired<S>(w, y);
 
             if (ph == 0) {
+                // transpose through shared memory; inside a row the elements sit in pair order, so that the 128-bit
+                // row reads of pass 1 deliver the cascade's pairs as they are
+                float *Xc = X + fdct::pair_order(t);
                 fdct::static_for<0, S>([&](auto i) {
                     constexpr int p = decltype(i)::value;
-                    X[fdct::core_index<S>(p) * XS + t] = y[p];
+                    Xc[fdct::core_index<S>(p) * XS] = y[p];
                 });
                 sb.sync();
             } else if (ph == 2) {
@@ -516,19 +527,22 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                 // area; the row-stage tile it overlaps is dead for every thread only after the barrier below, so the
                 // column is formed in registers first), which one TMA store writes out; the next chunk's tiles are
                 // requested as soon as the store has read the tile.
-                float r[S];
-                fdct::dct3_post<S>(y, r);
+                fdct::F2 rp[S / 2];  // pair p: rows (2p, 2p+1), swapped for odd p
+                fdct::dct3_post_pairs<S>(y, rp);
                 tmem_wait_st();  // the store of B (pass 0) has long completed
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    float b[32];
+                    float b[32];  // columns 32h .. 32h+31 of the lane: B in pair order, i.e. the pairs' own order
                     tmem_ld32(taddr + 32 * h, b);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[32 * h + i] = b[i] - r[32 * h + i];
+                    for (int q = 0; q < 16; ++q) rp[16 * h + q] = fdct::f2_sub(fdct::f2_make(b[2 * q], b[2 * q + 1]), rp[16 * h + q]);
                 }
                 sb.sync();  // every thread has read its column of the row-stage tile
-#pragma unroll
-                for (int i = 0; i < S; ++i) Ms[i * S + t] = r[i];
+                fdct::static_for<0, S / 2>([&](auto i) {
+                    constexpr int p = decltype(i)::value;
+                    Ms[(2 * p + (p & 1)) * S + t] = fdct::f2_lo(rp[p]);
+                    Ms[(2 * p + 1 - (p & 1)) * S + t] = fdct::f2_hi(rp[p]);
+                });
                 fence_proxy_async();
                 sb.sync();
                 {
