@@ -981,7 +981,14 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
                     bulk_g2s(smem_u32(Xt + t * S), x + base + (size_t)t * te.n1, S * sizeof(float), bar);
                 }
             }
-            fdct::dct3_ortho<S>(r);
+            {
+                // inverse transform: the DCT-IV blocks and the butterfly cascade with two sums per instruction
+                // (same results as the scalar form)
+                float w[S], y[S];
+                fdct::static_for<0, S>([&](auto i) { w[decltype(i)::value] = r[fdct::core_index<S>(decltype(i)::value)]; });
+                fdct::dct_core_ortho_paired<S>(w, y);
+                fdct::dct3_post_paired<S>(y, r);
+            }
             if (pass == 0) {
                 float4 *row = reinterpret_cast<float4 *>(St + t * XS);
 #pragma unroll
