@@ -515,6 +515,27 @@ FDCT_HD void dct3_post_paired(const float (&y)[N], float (&x)[N])
     const F2 e[1] = {f2_make(y[0] + y[1], y[0] - y[1])};
     inv_cascade_paired<2, N>(e, y, x);
 }
+// dct2<N, SC> / dct3<N, SC> (any output scale SC, DC term unscaled) through the packed cascades and blocks: same
+// results, about a third fewer instructions.
+template <int N, class SC>
+FDCT_HD void dct2_packed(const float (&x)[N], float (&X)[N])
+{
+    float w[N], y[N];
+    dct2_pre_paired<N>(x, w);
+    y[0] = w[0];
+    core_blocks_paired<N / 2, N, SC>(w, y);
+    static_for<0, N>([&](auto i) { X[core_index<N>(decltype(i)::value)] = y[decltype(i)::value]; });
+}
+template <int N, class SC>
+FDCT_HD void dct3_packed(const float (&X)[N], float (&x)[N])
+{
+    float w[N], y[N];
+    static_for<0, N>([&](auto i) { w[decltype(i)::value] = X[core_index<N>(decltype(i)::value)]; });
+    y[0] = w[0];
+    core_blocks_paired<N / 2, N, SC>(w, y);
+    dct3_post_paired<N>(y, x);
+}
+
 // The same with the result left in pairs: xp[p] = (x[2p], x[2p+1]) for even p, (x[2p+1], x[2p]) for odd p.
 template <int H, int N>
 FDCT_HD void inv_cascade_pairs(const F2 (&e)[H / 2], const float (&y)[N], F2 (&xp)[N / 2])

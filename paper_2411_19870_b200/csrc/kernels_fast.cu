@@ -227,7 +227,13 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
                     q[4 * v4 + 3] = f.w;
                 }
             }
-            fdct::dct2_ortho<S>(q);
+            {
+                float qi[S];
+#pragma unroll
+                for (int i = 0; i < S; ++i) qi[i] = q[i];
+                fdct::dct2_packed<S, fdct::ScaleOrtho<S>>(qi, q);
+                q[0] *= fdct::dc_scale<S>();
+            }
             if (pass == 0) {
 #pragma unroll
                 for (int u = 0; u < S; ++u) X[u * XS + t] = q[u];
@@ -719,7 +725,13 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress_fast_kernel(D
             fence_proxy_async();
             sb.sync();
             issue_loads(tile_cur);
-            fdct::dct3_ortho<S>(r);
+            {
+                float ri[S];
+                r[0] *= fdct::dc_scale<S>();
+#pragma unroll
+                for (int i = 0; i < S; ++i) ri[i] = r[i];
+                fdct::dct3_packed<S, fdct::ScaleOrtho<S>>(ri, r);
+            }
             const bool again = mbar_wait_bounded(bar, phase);
             phase ^= 1u;
             if (!sb.sync_and(again)) {

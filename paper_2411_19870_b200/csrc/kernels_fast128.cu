@@ -52,10 +52,10 @@ __device__ __forceinline__ unsigned block_exclusive_scan(unsigned v, unsigned *w
 __device__ __forceinline__ void forward_half(int h, float (&in)[H], float (&out)[H])
 {
     if (h == 0) {
-        fdct::dct2<H, SC>(in, out);
+        fdct::dct2_packed<H, SC>(in, out);
         out[0] *= fdct::dc_scale<S>();
     } else {
-        fdct::dct4<H, SC>(in, out);
+        fdct::dct4_paired<H, SC>(in, out);
     }
 }
 // Inverse half-transform: in[p] = coefficient 2p (h = 0) or 2p+1 (h = 1); out = e (h = 0) or o (h = 1).
@@ -63,9 +63,9 @@ __device__ __forceinline__ void inverse_half(int h, float (&in)[H], float (&out)
 {
     if (h == 0) {
         in[0] *= fdct::dc_scale<S>();
-        fdct::dct3<H, SC>(in, out);
+        fdct::dct3_packed<H, SC>(in, out);
     } else {
-        fdct::dct4<H, SC>(in, out);
+        fdct::dct4_paired<H, SC>(in, out);
     }
 }
 
