@@ -203,6 +203,8 @@ def run_ours(args, rank, world):
                             chunk_shapes=chunk_shapes)
     if args.path == "generic":
         tr.set_path(demo.DEMO_PATH_GENERIC)
+    if args.momentum_domain == "dct":  # experiment, not the headline: momentum of 2-D tensors kept as DCT tiles
+        tr.set_momentum_domain(demo.DEMO_MOMENTUM_DCT)
     if args.basis == "identity":
         tr.set_basis(torch.eye(wl.chunk))
     elif args.basis == "random":  # Gaussian draws seeded by a step number, orthonormalised on the device
@@ -343,6 +345,7 @@ def run_ours(args, rank, world):
                        "gradients": "one seeded gradient set per worker, reused every step on purpose (a second set "
                                     "per worker does not fit beside the %d momenta; the momentum still changes "
                                     "every step)" % W,
+                       "momentum_domain": args.momentum_domain,
                        "basis": args.basis, "chunk_shape": args.chunk_shape or None,
                        "embedding_active_rows": args.embedding_active_rows or None},
             "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
@@ -514,6 +517,8 @@ def main():
     ap.add_argument("--chunk-shape", default="", help="AxB: rectangular chunks through the N-D kernels (ablation)")
     ap.add_argument("--basis", default="dct", choices=["dct", "identity", "random"],
                     help="transform basis; anything but dct takes the dense-transform kernels (not the headline)")
+    ap.add_argument("--momentum-domain", default="spatial", choices=["spatial", "dct"],
+                    help="dct: the opt-in representation of demo_set_momentum_domain (a second, non-headline line)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -317,6 +317,25 @@ demo_status demo_selftest_bounded_wait(demo_ctx *ctx, int64_t limit_cycles, void
 /* Select the kernel family (see demo_path).  Errors: INVALID_ARG. */
 demo_status demo_set_path(demo_ctx *ctx, int32_t path);
 
+/* Representation of the momentum tensors of 2-D parameters (opt-in; the paper keeps the momentum itself and
+ * has no counterpart of this switch).  The chunk transform is linear and orthonormal, so the step of
+ * Algorithm 1 can be carried out on the transformed momentum Qm = DCT(m) chunk by chunk:
+ *     Q = beta * Qm + DCT(g);   records = top-k(Q);   Qm <- Q - alpha * Q_kept,
+ * which yields the records of demo_compress up to fp32 rounding and needs one forward transform of the
+ * gradient and no inverse transform.
+ *   DEMO_MOMENTUM_SPATIAL (default): the buffers passed to demo_compress hold m.
+ *   DEMO_MOMENTUM_DCT: for every 2-D tensor they hold, tile by tile, the TRANSPOSED coefficient tile of
+ *     the chunk: element (64*k0 + r, 64*k1 + c) of the buffer is coefficient (c, r) of chunk (k0, k1) of
+ *     DCT(m).  An all-zero buffer means m = 0 in both representations.  The momentum is recovered as
+ *     m = IDCT(tile transposed) per chunk; 1-D tensors always hold m itself.
+ * Only the s = 64 tile kernel with TMA tensor maps implements the second form: UNSUPPORTED for contexts
+ * of demo_init_nd, for chunk != 64, or when the driver offers no tensor-map encoder; while it is on,
+ * demo_compress (and demo_step_host, which calls it) returns UNSUPPORTED if a caller-supplied basis or
+ * DEMO_PATH_GENERIC is active.  The caller converts or clears the buffers when switching; the library
+ * never does.  Errors: INVALID_ARG, UNSUPPORTED. */
+typedef enum demo_momentum_domain { DEMO_MOMENTUM_SPATIAL = 0, DEMO_MOMENTUM_DCT = 1 } demo_momentum_domain;
+demo_status demo_set_momentum_domain(demo_ctx *ctx, int32_t domain);
+
 /* Number of kernel launches this context has enqueued since demo_init (for accounting). */
 int64_t demo_launch_count(const demo_ctx *ctx);
 

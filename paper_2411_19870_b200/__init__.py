@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     DEMO_AGG_COUNT_MEAN,
     DEMO_AGG_MEAN,
     DEMO_AGG_SUM,
+    DEMO_MOMENTUM_DCT,
+    DEMO_MOMENTUM_SPATIAL,
     DEMO_PATH_AUTO,
     DEMO_PHI_IDENTITY,
     DEMO_PHI_SIGN,

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(HERE, "libdemo_b200.so")
 
 DEMO_F32, DEMO_BF16 = 0, 1
 DEMO_PATH_AUTO, DEMO_PATH_GENERIC = 0, 1
+DEMO_MOMENTUM_SPATIAL, DEMO_MOMENTUM_DCT = 0, 1
 DEMO_AGG_SUM, DEMO_AGG_MEAN, DEMO_AGG_COUNT_MEAN = 0, 1, 2
 DEMO_PHI_SIGN, DEMO_PHI_IDENTITY = 0, 1
 RECORD_BYTES = 8
@@ -26,7 +27,7 @@ EXPORTS = [
     "demo_init", "demo_init_nd", "demo_payload_bytes", "demo_payload_layout", "demo_compress", "demo_decode_apply",
     "demo_decode_signs", "demo_apply_signs",
     "demo_step_host", "demo_decode_apply_static", "demo_set_lr", "demo_set_alpha", "demo_set_decode_mode", "demo_set_basis",
-    "demo_set_basis_gaussian", "demo_get_basis", "demo_selftest_bounded_wait", "demo_set_path", "demo_launch_count", "demo_device_status",
+    "demo_set_basis_gaussian", "demo_get_basis", "demo_selftest_bounded_wait", "demo_set_path", "demo_set_momentum_domain", "demo_launch_count", "demo_device_status",
     "demo_status_string", "demo_free",
 ]
 
@@ -108,6 +109,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.demo_selftest_bounded_wait.restype = i32
     lib.demo_set_path.argtypes = [vp, i32]
     lib.demo_set_path.restype = i32
+    lib.demo_set_momentum_domain.argtypes = [vp, i32]
+    lib.demo_set_momentum_domain.restype = i32
     lib.demo_launch_count.argtypes = [vp]
     lib.demo_launch_count.restype = i64
     lib.demo_device_status.argtypes = [vp, vp]
@@ -354,6 +357,11 @@ class DemoTransform:
         st = self.lib.demo_set_path(self._ctx, path)
         if st != 0:
             raise DemoError(st, "demo_set_path")
+
+    def set_momentum_domain(self, domain: int) -> None:
+        st = self.lib.demo_set_momentum_domain(self._ctx, domain)
+        if st != 0:
+            raise DemoError(st, "demo_set_momentum_domain")
 
     def device_status(self, stream=None) -> int:
         return int(self.lib.demo_device_status(self._ctx, self._stream(stream)))

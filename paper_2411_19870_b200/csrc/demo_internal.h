@@ -39,6 +39,9 @@ struct DemoCompressArgs {
     // pointer arrays; box = one s x s tile).  NULL: tiles are staged row by row with 1-D bulk copies.
     const void *tmap_m;
     const void *tmap_g;
+    // 1: the momentum tensors hold the chunk-wise DCT of the momentum (tiles transposed); only the s = 64 tile
+    // kernel with tensor maps implements it
+    int momentum_dct = 0;
 };
 
 struct DemoDecodeArgs {

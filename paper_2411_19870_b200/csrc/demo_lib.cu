@@ -46,6 +46,7 @@ struct demo_ctx {
     float *d_P = nullptr, *d_P_stage = nullptr;  // [s*s], [2*s*s]
     int *d_basis_flag = nullptr;
     bool custom_basis = false;
+    bool momentum_dct = false;  // demo_set_momentum_domain(DEMO_MOMENTUM_DCT)
 
     // device pointer tables and their host mirrors (uploaded only when the caller's pointers change)
     const void **d_g = nullptr;      // [W][T]
@@ -589,6 +590,9 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
         return DEMO_ERR_CUDA;
     }
 
+    if (ctx->momentum_dct && !(use_fast_path(ctx) && ctx->encode && ctx->cfg.chunk == 64 && !ctx->nd))
+        return DEMO_ERR_UNSUPPORTED;  // only the s = 64 tile kernel keeps the momentum in the transform domain
+
     if (ctx->nd) {
         DemoNdCompressArgs n;
         n.entries = ctx->d_entries_nd;
@@ -626,6 +630,7 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
     cudaStream_t side = stream;
     if (ctx->n1d) {
         side = fork_side(ctx, stream);
+        a.momentum_dct = 0;  // 1-D tensors keep the momentum itself
         a.entries = ctx->d_entries1d;
         a.n_entries = ctx->n1d;
         a.n_chunks = ctx->chunks1d;
@@ -636,6 +641,7 @@ demo_status demo_compress(demo_ctx *ctx, int32_t worker, const void *const *grad
         a.entries = ctx->d_entries2d;
         a.n_entries = ctx->n2d;
         a.n_chunks = ctx->chunks2d;
+        a.momentum_dct = ctx->momentum_dct ? 1 : 0;
         if (use_fast_path(ctx))
             err = demo_launch_compress_fast(s, a, ctx->sm_count, stream);
         else if (use_tc_path(ctx))
@@ -1042,6 +1048,14 @@ demo_status demo_get_basis(demo_ctx *ctx, float *basis_host_out, void *cuda_stre
         cudaGetLastError();
         return DEMO_ERR_CUDA;
     }
+    return DEMO_OK;
+}
+
+demo_status demo_set_momentum_domain(demo_ctx *ctx, int32_t domain)
+{
+    if (!ctx || (domain != DEMO_MOMENTUM_SPATIAL && domain != DEMO_MOMENTUM_DCT)) return DEMO_ERR_INVALID_ARG;
+    if (domain == DEMO_MOMENTUM_DCT && (ctx->nd || ctx->cfg.chunk != 64 || !ctx->encode)) return DEMO_ERR_UNSUPPORTED;
+    ctx->momentum_dct = (domain == DEMO_MOMENTUM_DCT);
     return DEMO_OK;
 }
 

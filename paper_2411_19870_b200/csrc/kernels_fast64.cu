@@ -122,7 +122,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 //   3. otherwise an exact 4 x 8-bit radix select over the whole tile.
 // ------------------------------------------------------------------------------------------------
 __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord *rec, float alpha, int t, int bar_id,
-                                         unsigned lmin_w, bool bound_valid)
+                                         unsigned lmin_w, bool bound_valid, bool qdom)
 {
     const SlotBarrier<S> sb{bar_id};
     const int lane = t & 31, warp = t >> 5;
@@ -280,7 +280,9 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                             const int uo = (r.idx >> LOG2S) * XS;
                             r.val = X[uo + v];
                             rec[pos] = r;
-                            if (k_eff <= 64)
+                            if (qdom)  // transform-domain momentum: what stays of a transmitted coefficient
+                                X[uo + v] = fmaf(-alpha, r.val, r.val);
+                            else if (k_eff <= 64)
                                 recs4[pos] = make_int4(uo, v * S, __float_as_int(alpha * r.val), 0);
                             else
                                 sm.rbig[pos] = make_uint2(((unsigned)r.idx >> LOG2S) << 16 | (unsigned)v, __float_as_uint(alpha * r.val));
@@ -338,7 +340,9 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
                 r.idx = t * S + v;
                 r.val = val;
                 rec[pos] = r;
-                if (k_eff <= 64)
+                if (qdom)
+                    X[t * XS + v] = fmaf(-alpha, val, val);
+                else if (k_eff <= 64)
                     recs4[pos] = make_int4(t * XS, v * S, __float_as_int(alpha * val), 0);
                 else if (k_eff <= 256)
                     sm.rbig[pos] = make_uint2((unsigned)t << 16 | (unsigned)v, __float_as_uint(alpha * val));
@@ -347,7 +351,213 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
     }
 }
 
-template <typename GT, int THREADS>
+// ------------------------------------------------------------------------------------------------
+// Exact top-k of one chunk (Section 2.1 "Top-k Sparsification"): thread t holds the coefficients q[v] = Q[t][v] of
+// row t.  Writes the k_eff records in ascending index order to `rec`; ends before the barrier that makes them
+// visible.  QDOM = false (momentum kept in the spatial domain): also leaves the pre-decoded row-stage list and the
+// tile X cleared for the row stage.  QDOM = true (momentum kept in the transform domain): leaves in X the
+// coefficient tile with every transmitted coefficient q replaced by q - alpha q.
+// ------------------------------------------------------------------------------------------------
+template <bool QDOM>
+__device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], int k_eff, DemoRecord *rec, float alpha,
+                                             int t, const SlotBarrier<S> &sb, int bar_id, int pad_row)
+{
+    float *X = sm.X;
+    float *tmax = sm.tmax;
+    int *cand_idx = sm.cand_idx;
+    float *cand_val = sm.cand_val;
+    unsigned *cand_key = sm.cand_key;
+    int4 *recs4 = sm.recs4;
+    unsigned *misc = sm.misc;
+    const int lane = t & 31, warp = t >> 5;
+    // the row-stage tile starts from zero; every thread clears its own row once it is done with it
+    auto zero_row = [&]() {
+        if (QDOM) return;  // (the transform-domain kernel keeps the coefficient tile: it is its output)
+        float4 *row = reinterpret_cast<float4 *>(X + t * XS);
+#pragma unroll
+        for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    auto stash_row = [&]() {
+        float4 *row = reinterpret_cast<float4 *>(X + t * XS);
+#pragma unroll
+        for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(q[4 * v4], q[4 * v4 + 1], q[4 * v4 + 2], q[4 * v4 + 3]);
+    };
+    // ---- exact top-k (Section 2.1 "Top-k Sparsification") -------------------------------
+    if (!QDOM) {
+        recs4[t] = make_int4(pad_row, 0, 0, 0);  // list padding (ordered before the record writes by the barriers below)
+        if (t == 0) recs4[64] = make_int4(pad_row, 0, 0, 0);
+    }
+    bool slow = (k_eff > S);
+    bool bound_valid = false;
+    bool zero_chunk = false;
+    unsigned n_cw = 0, off = 0, mlo = 0u, mhi = 0u, lmin_w = 0u;
+    if (!slow) {
+        // per-thread maximum magnitude (independent chains of 16, 3-input max)
+        float tm = 0.f;
+#pragma unroll
+        for (int ch = 0; ch < S / 16; ++ch) {
+            const int b0 = 16 * ch;
+            float cm = max3abs(q[b0], q[b0 + 1], q[b0 + 2]);
+#pragma unroll
+            for (int j = 3; j + 1 < 16; j += 2) cm = max3f(cm, fabsf(q[b0 + j]), fabsf(q[b0 + j + 1]));
+            tm = max3f(tm, cm, fabsf(q[b0 + 15]));
+        }
+        // L = the k_eff-th largest of the 64 row maxima (low 15 mantissa bits cleared): a lower bound of
+        // the k_eff-th largest coefficient.  Every warp holds all 64 keys, two ballots per step count them.
+        const unsigned tkey = __float_as_uint(tm);
+        unsigned *tk = reinterpret_cast<unsigned *>(tmax);
+        tk[t] = tkey;
+        sb.sync();
+        const unsigned okey = tk[t ^ 32];
+        const unsigned lo_all = __reduce_min_sync(0xffffffffu, min(tkey, okey));
+        const unsigned hi_all = __reduce_max_sync(0xffffffffu, max(tkey, okey));
+        zero_chunk = (hi_all == 0u);
+        const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
+        unsigned prefix = lo_all & ~((2u << b0) - 1u);
+#pragma unroll 1
+        for (int b = zero_chunk ? 14 : b0; b >= 15; --b) {
+            const unsigned cand = prefix | (1u << b);
+            const unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand)) +
+                                 __popc(__ballot_sync(0xffffffffu, okey >= cand));
+            prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
+        }
+        lmin_w = prefix;
+        bound_valid = true;
+        if (!zero_chunk) {
+            // candidates: |q| >= L  <=>  |q| > Lm (the float just below L); the sign bit of Lm - |q|
+            // is funnel-shifted into a bit mask (independent chains of 16)
+            const float L = __uint_as_float(lmin_w);
+            const float Lm = (L > 0.f) ? __uint_as_float(lmin_w - 1u) : -1.f;
+            unsigned mc[S / 16];
+#pragma unroll
+            for (int ch = 0; ch < S / 16; ++ch) {
+                unsigned mm = 0u;
+#pragma unroll
+                for (int j = 15; j >= 0; --j)
+                    mm = __funnelshift_l(__float_as_uint(Lm - fabsf(q[16 * ch + j])), mm, 1);
+                mc[ch] = mm;
+            }
+            mlo = mc[0] | (mc[1] << 16);
+            mhi = mc[2] | (mc[3] << 16);
+            const unsigned cnt = __popc(mlo) + __popc(mhi);
+            const unsigned inc = warp_inclusive_scan(cnt, lane);
+            off = inc - cnt;
+            n_cw = __shfl_sync(0xffffffffu, inc, 31);
+            if (lane == 0) misc[warp] = n_cw;
+        }
+    }
+    if (zero_chunk) {
+        // all coefficients zero: the tie rule gives the records 0 .. k_eff-1 with value 0
+        if (t < k_eff) {
+            DemoRecord r;
+            r.idx = t;
+            r.val = 0.f;
+            rec[t] = r;
+        }
+        if (!QDOM && t < k_eff) recs4[t] = make_int4(0, 0, 0, 0);
+        zero_row();
+        if (QDOM) stash_row();  // (all zero; the tile is the kernel's output)
+    } else {
+        // stash the coefficients of row t (own row: no hazard with other threads)
+        stash_row();
+        if (!slow) {
+            const unsigned lbase = warp * CAPWP;
+            if (n_cw <= CAPW) {
+                // each warp compacts its candidates into its own list (rows of warp 0 precede rows of
+                // warp 1, so the concatenation is in ascending index order)
+                unsigned o = lbase + off;
+                unsigned long long mask = ((unsigned long long)mhi << 32) | mlo;
+                while (mask) {
+                    const int v = __ffsll((long long)mask) - 1;
+                    mask &= mask - 1ull;
+                    const float val = X[t * XS + v];
+                    cand_idx[o] = t * S + v;
+                    cand_val[o] = val;
+                    cand_key[o] = mag_key(val);
+                    ++o;
+                }
+                if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
+            }
+            sb.sync();
+            const unsigned n_w0 = misc[0], n_w1 = misc[1];
+            // more than a list holds, or fewer candidates than k_eff (NaN coefficients fail the float
+            // comparisons above): the out-of-line selection takes over
+            slow = (n_w0 > (unsigned)CAPW) || (n_w1 > (unsigned)CAPW) || (n_w0 + n_w1 < (unsigned)k_eff);
+            if (!slow) {
+                zero_row();  // row t of the stash was read by this thread only
+                // Every warp takes both lists into registers (two keys per lane and list) and searches,
+                // bit by bit from the first bit where the bound and the largest key differ, for a
+                // threshold with exactly k_eff keys at or above it; the search stops as soon as one is
+                // found.  If it runs out of bits, equal keys straddle the k_eff-th place: keys above
+                // the threshold are kept, keys equal to it in index order until k_eff are reached.
+                const unsigned n_mine = warp ? n_w1 : n_w0, n_oth = warp ? n_w0 : n_w1;
+                const unsigned obase = (warp ^ 1) * CAPWP;
+                unsigned keys[4];  // 0, 1: this warp's list; 2, 3: the other warp's
+                keys[0] = (lane < n_mine) ? cand_key[lbase + lane] : 0u;
+                keys[1] = (lane + 32u < n_mine) ? cand_key[lbase + 32 + lane] : 0u;
+                keys[2] = (lane < n_oth) ? cand_key[obase + lane] : 0u;
+                keys[3] = (lane + 32u < n_oth) ? cand_key[obase + 32 + lane] : 0u;
+                const unsigned hi = __reduce_max_sync(0xffffffffu, max(max(keys[0], keys[1]), max(keys[2], keys[3])));
+                const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
+                unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+                unsigned n_ge = n_w0 + n_w1;  // every candidate is >= the bound >= thr
+#pragma unroll 1
+                for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
+                    const unsigned cand = thr | (1u << b);
+                    unsigned cnt = 0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+                    if (cnt >= (unsigned)k_eff) {
+                        thr = cand;
+                        n_ge = cnt;
+                    }
+                }
+                // kept entries before this warp's list (index order: list 0, then list 1) and in all
+                const unsigned g_oth = __popc(__ballot_sync(0xffffffffu, keys[2] > thr)) +
+                                       __popc(__ballot_sync(0xffffffffu, keys[3] > thr));
+                const unsigned e_oth = __popc(__ballot_sync(0xffffffffu, keys[2] == thr)) +
+                                       __popc(__ballot_sync(0xffffffffu, keys[3] == thr));
+                const unsigned gtb0 = __ballot_sync(0xffffffffu, keys[0] > thr);
+                const unsigned gtb1 = __ballot_sync(0xffffffffu, keys[1] > thr);
+                const unsigned eqb0 = __ballot_sync(0xffffffffu, keys[0] == thr);
+                const unsigned eqb1 = __ballot_sync(0xffffffffu, keys[1] == thr);
+                const unsigned need_eq = (unsigned)k_eff - (g_oth + __popc(gtb0) + __popc(gtb1));
+                const unsigned lt = (1u << lane) - 1u;
+#pragma unroll 1
+                for (int jj = 0; jj < 2; ++jj) {  // (rolled: one copy of the record write)
+                    const unsigned key = jj ? keys[1] : keys[0];
+                    const unsigned gtb = jj ? gtb1 : gtb0, eqb = jj ? eqb1 : eqb0;
+                    const unsigned gt_before = (warp ? g_oth : 0u) + (jj ? __popc(gtb0) : 0u);
+                    const unsigned e = (warp ? e_oth : 0u) + (jj ? __popc(eqb0) : 0u) + __popc(eqb & lt);
+                    if ((key > thr) || (key == thr && e < need_eq)) {
+                        const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
+                        const unsigned li = lbase + (unsigned)jj * 32u + lane;
+                        DemoRecord r;
+                        r.idx = cand_idx[li];
+                        r.val = cand_val[li];
+                        rec[pos] = r;
+                        if (QDOM)  // what stays of a transmitted coefficient: q - alpha q
+                            X[(r.idx >> LOG2S) * XS + (r.idx & (S - 1))] = fmaf(-alpha, r.val, r.val);
+                        else
+                            recs4[pos] = make_int4((r.idx >> LOG2S) * XS, (r.idx & (S - 1)) * S,
+                                                   __float_as_int(alpha * r.val), 0);
+                    }
+                }
+            }
+        }
+        if (slow) {
+            select_slow(sm, k_eff, rec, alpha, t, bar_id, lmin_w, bound_valid, QDOM);
+            sb.sync();  // every thread is done with the coefficient tile
+            zero_row();
+        }
+    }
+}
+
+// QDOM = false: the momentum buffers hold the momentum itself (the contract of demo_compress).  QDOM = true (opt-in,
+// demo_set_momentum_domain): they hold its chunk-wise DCT, tile by tile and transposed (element (r, c) of a tile
+// is coefficient (c, r)): the step is then Q = beta*Qm + DCT(g), top-k, Qm <- Q - alpha*Q_kept -- one forward
+// transform of the gradient, no inverse transform, no row stage.
+template <typename GT, int THREADS, bool QDOM>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(DemoCompressArgs a)
 {
     constexpr int NCH = THREADS / S;
@@ -376,12 +586,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(sm.misc + 16);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_all + (size_t)NCH * slot_bytes<GT>());
     float *X = sm.X;
-    float *tmax = sm.tmax;
-    int *cand_idx = sm.cand_idx;
-    float *cand_val = sm.cand_val;
-    unsigned *cand_key = sm.cand_key;
     int4 *recs4 = sm.recs4;
-    unsigned *misc = sm.misc;
 
     // "row" of the padding entries of the row-stage list: the scratch line tmax[0..S) seen from X
     constexpr int PAD_ROW = (int)(region_bytes<GT>() / sizeof(float));
@@ -472,18 +677,29 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
         // 1 = DCT-II along row t (followed by the selection and the sparse row stage of the inverse),
         // 2 = DCT-III down column t of the row-stage tile (followed by the residual).
 #pragma unroll 1
-        for (int ph = 0; ph < 3; ++ph) {
+        for (int ph = 0; ph < (QDOM ? 2 : 3); ++ph) {
             float w[S], y[S];
             if (ph < 2) {
                 float x[S];
                 if (ph == 0) {
+                    if constexpr (QDOM) {
+                        // row t of the stored coefficients (column t of the transposed tile) is parked for pass 1;
+                        // the forward transform runs on the gradient alone
+                        float mq[S];
 #pragma unroll
-                    for (int i = 0; i < S; ++i) x[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
-                    // B = beta*m + g, parked for the residual; column k of the tensor-memory lane takes element
-                    // pair_order(k), so that the registers of the store are those of the cascade's pairs
-                    float xp[S];
-                    fdct::static_for<0, S>([&](auto i) { xp[decltype(i)::value] = x[fdct::pair_order(decltype(i)::value)]; });
-                    tmem_st64(taddr, xp);
+                        for (int i = 0; i < S; ++i) mq[i] = Ms[i * S + t];
+                        tmem_st64(taddr, mq);
+#pragma unroll
+                        for (int i = 0; i < S; ++i) x[i] = to_f32(Gs[i * S + t]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < S; ++i) x[i] = fmaf(a.beta, Ms[i * S + t], to_f32(Gs[i * S + t]));
+                        // B = beta*m + g, parked for the residual; column k of the tensor-memory lane takes element
+                        // pair_order(k), so that the registers of the store are those of the cascade's pairs
+                        float xp[S];
+                        fdct::static_for<0, S>([&](auto i) { xp[decltype(i)::value] = x[fdct::pair_order(decltype(i)::value)]; });
+                        tmem_st64(taddr, xp);
+                    }
                     // every thread has consumed its column of the staged tiles (X aliases them)
                     if (!sb.sync_and(arrived)) {
                         if (t == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
@@ -561,178 +777,43 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                     constexpr int p = decltype(i)::value;
                     q[fdct::core_index<S>(p)] = y[p];
                 });
-                // the row-stage tile starts from zero; every thread clears its own row once it is done with it
-                auto zero_row = [&]() {
-                    float4 *row = reinterpret_cast<float4 *>(X + t * XS);
+                if constexpr (QDOM) {
+                    // Q = beta * Qm + DCT(g); the stored row comes back from tensor memory
+                    tmem_wait_st();
 #pragma unroll
-                    for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
-                };
-                // ---- exact top-k (Section 2.1 "Top-k Sparsification") -------------------------------
-                recs4[t] = make_int4(PAD_ROW, 0, 0, 0);  // list padding (ordered before the record writes by the barriers below)
-                if (t == 0) recs4[64] = make_int4(PAD_ROW, 0, 0, 0);
-                bool slow = (k_eff > S);
-                bool bound_valid = false;
-                bool zero_chunk = false;
-                unsigned n_cw = 0, off = 0, mlo = 0u, mhi = 0u, lmin_w = 0u;
-                if (!slow) {
-                    // per-thread maximum magnitude (independent chains of 16, 3-input max)
-                    float tm = 0.f;
+                    for (int h = 0; h < 2; ++h) {
+                        float mq[32];
+                        tmem_ld32(taddr + 32 * h, mq);
 #pragma unroll
-                    for (int ch = 0; ch < S / 16; ++ch) {
-                        const int b0 = 16 * ch;
-                        float cm = max3abs(q[b0], q[b0 + 1], q[b0 + 2]);
-#pragma unroll
-                        for (int j = 3; j + 1 < 16; j += 2) cm = max3f(cm, fabsf(q[b0 + j]), fabsf(q[b0 + j + 1]));
-                        tm = max3f(tm, cm, fabsf(q[b0 + 15]));
+                        for (int j = 0; j < 32; ++j) q[32 * h + j] = fmaf(a.beta, mq[j], q[32 * h + j]);
                     }
-                    // L = the k_eff-th largest of the 64 row maxima (low 15 mantissa bits cleared): a lower bound of
-                    // the k_eff-th largest coefficient.  Every warp holds all 64 keys, two ballots per step count them.
-                    const unsigned tkey = __float_as_uint(tm);
-                    unsigned *tk = reinterpret_cast<unsigned *>(tmax);
-                    tk[t] = tkey;
+                    select_chunk<true>(sm, q, k_eff, rec, a.alpha, t, sb, slot + 1, PAD_ROW);
+                    sb.sync();  // the tile holds Q - alpha * Q_kept (kept entries were patched by the record writers)
+                    float4 rowv[S / 4];
+                    {
+                        const float4 *row = reinterpret_cast<const float4 *>(X + t * XS);
+#pragma unroll
+                        for (int v4 = 0; v4 < S / 4; ++v4) rowv[v4] = row[v4];
+                    }
+                    sb.sync();  // the dense tile below overlaps the coefficient tile
+#pragma unroll
+                    for (int v4 = 0; v4 < S / 4; ++v4) {
+                        Ms[(4 * v4 + 0) * S + t] = rowv[v4].x;
+                        Ms[(4 * v4 + 1) * S + t] = rowv[v4].y;
+                        Ms[(4 * v4 + 2) * S + t] = rowv[v4].z;
+                        Ms[(4 * v4 + 3) * S + t] = rowv[v4].w;
+                    }
+                    fence_proxy_async();
                     sb.sync();
-                    const unsigned okey = tk[t ^ 32];
-                    const unsigned lo_all = __reduce_min_sync(0xffffffffu, min(tkey, okey));
-                    const unsigned hi_all = __reduce_max_sync(0xffffffffu, max(tkey, okey));
-                    zero_chunk = (hi_all == 0u);
-                    const int b0 = 31 - __clz((lo_all ^ hi_all) | 0x8000u);  // >= 15
-                    unsigned prefix = lo_all & ~((2u << b0) - 1u);
-#pragma unroll 1
-                    for (int b = zero_chunk ? 14 : b0; b >= 15; --b) {
-                        const unsigned cand = prefix | (1u << b);
-                        const unsigned cnt = __popc(__ballot_sync(0xffffffffu, tkey >= cand)) +
-                                             __popc(__ballot_sync(0xffffffffu, okey >= cand));
-                        prefix = (cnt >= (unsigned)k_eff) ? cand : prefix;
+                    if (t == 0) {
+                        tma_store_2d(mine.tm_m, mine.x, mine.y, smem_u32(Ms));
+                        tma_store_commit();
+                        tma_store_wait_read();
+                        if (nc < a.n_chunks) issue_loads(next);
                     }
-                    lmin_w = prefix;
-                    bound_valid = true;
-                    if (!zero_chunk) {
-                        // candidates: |q| >= L  <=>  |q| > Lm (the float just below L); the sign bit of Lm - |q|
-                        // is funnel-shifted into a bit mask (independent chains of 16)
-                        const float L = __uint_as_float(lmin_w);
-                        const float Lm = (L > 0.f) ? __uint_as_float(lmin_w - 1u) : -1.f;
-                        unsigned mc[S / 16];
-#pragma unroll
-                        for (int ch = 0; ch < S / 16; ++ch) {
-                            unsigned mm = 0u;
-#pragma unroll
-                            for (int j = 15; j >= 0; --j)
-                                mm = __funnelshift_l(__float_as_uint(Lm - fabsf(q[16 * ch + j])), mm, 1);
-                            mc[ch] = mm;
-                        }
-                        mlo = mc[0] | (mc[1] << 16);
-                        mhi = mc[2] | (mc[3] << 16);
-                        const unsigned cnt = __popc(mlo) + __popc(mhi);
-                        const unsigned inc = warp_inclusive_scan(cnt, lane);
-                        off = inc - cnt;
-                        n_cw = __shfl_sync(0xffffffffu, inc, 31);
-                        if (lane == 0) misc[warp] = n_cw;
-                    }
+                    continue;
                 }
-                if (zero_chunk) {
-                    // all coefficients zero: the tie rule gives the records 0 .. k_eff-1 with value 0
-                    if (t < k_eff) {
-                        DemoRecord r;
-                        r.idx = t;
-                        r.val = 0.f;
-                        rec[t] = r;
-                    }
-                    if (t < k_eff) recs4[t] = make_int4(0, 0, 0, 0);
-                    zero_row();
-                } else {
-                    // stash the coefficients of row t (own row: no hazard with other threads)
-                    float4 *row = reinterpret_cast<float4 *>(X + t * XS);
-#pragma unroll
-                    for (int v4 = 0; v4 < S / 4; ++v4)
-                        row[v4] = make_float4(q[4 * v4], q[4 * v4 + 1], q[4 * v4 + 2], q[4 * v4 + 3]);
-                    if (!slow) {
-                        const unsigned lbase = warp * CAPWP;
-                        if (n_cw <= CAPW) {
-                            // each warp compacts its candidates into its own list (rows of warp 0 precede rows of
-                            // warp 1, so the concatenation is in ascending index order)
-                            unsigned o = lbase + off;
-                            unsigned long long mask = ((unsigned long long)mhi << 32) | mlo;
-                            while (mask) {
-                                const int v = __ffsll((long long)mask) - 1;
-                                mask &= mask - 1ull;
-                                const float val = X[t * XS + v];
-                                cand_idx[o] = t * S + v;
-                                cand_val[o] = val;
-                                cand_key[o] = mag_key(val);
-                                ++o;
-                            }
-                            if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
-                        }
-                        sb.sync();
-                        const unsigned n_w0 = misc[0], n_w1 = misc[1];
-                        // more than a list holds, or fewer candidates than k_eff (NaN coefficients fail the float
-                        // comparisons above): the out-of-line selection takes over
-                        slow = (n_w0 > (unsigned)CAPW) || (n_w1 > (unsigned)CAPW) || (n_w0 + n_w1 < (unsigned)k_eff);
-                        if (!slow) {
-                            zero_row();  // row t of the stash was read by this thread only
-                            // Every warp takes both lists into registers (two keys per lane and list) and searches,
-                            // bit by bit from the first bit where the bound and the largest key differ, for a
-                            // threshold with exactly k_eff keys at or above it; the search stops as soon as one is
-                            // found.  If it runs out of bits, equal keys straddle the k_eff-th place: keys above
-                            // the threshold are kept, keys equal to it in index order until k_eff are reached.
-                            const unsigned n_mine = warp ? n_w1 : n_w0, n_oth = warp ? n_w0 : n_w1;
-                            const unsigned obase = (warp ^ 1) * CAPWP;
-                            unsigned keys[4];  // 0, 1: this warp's list; 2, 3: the other warp's
-                            keys[0] = (lane < n_mine) ? cand_key[lbase + lane] : 0u;
-                            keys[1] = (lane + 32u < n_mine) ? cand_key[lbase + 32 + lane] : 0u;
-                            keys[2] = (lane < n_oth) ? cand_key[obase + lane] : 0u;
-                            keys[3] = (lane + 32u < n_oth) ? cand_key[obase + 32 + lane] : 0u;
-                            const unsigned hi = __reduce_max_sync(0xffffffffu, max(max(keys[0], keys[1]), max(keys[2], keys[3])));
-                            const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
-                            unsigned thr = lmin_w & ~((2u << wb0) - 1u);
-                            unsigned n_ge = n_w0 + n_w1;  // every candidate is >= the bound >= thr
-#pragma unroll 1
-                            for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
-                                const unsigned cand = thr | (1u << b);
-                                unsigned cnt = 0;
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
-                                if (cnt >= (unsigned)k_eff) {
-                                    thr = cand;
-                                    n_ge = cnt;
-                                }
-                            }
-                            // kept entries before this warp's list (index order: list 0, then list 1) and in all
-                            const unsigned g_oth = __popc(__ballot_sync(0xffffffffu, keys[2] > thr)) +
-                                                   __popc(__ballot_sync(0xffffffffu, keys[3] > thr));
-                            const unsigned e_oth = __popc(__ballot_sync(0xffffffffu, keys[2] == thr)) +
-                                                   __popc(__ballot_sync(0xffffffffu, keys[3] == thr));
-                            const unsigned gtb0 = __ballot_sync(0xffffffffu, keys[0] > thr);
-                            const unsigned gtb1 = __ballot_sync(0xffffffffu, keys[1] > thr);
-                            const unsigned eqb0 = __ballot_sync(0xffffffffu, keys[0] == thr);
-                            const unsigned eqb1 = __ballot_sync(0xffffffffu, keys[1] == thr);
-                            const unsigned need_eq = (unsigned)k_eff - (g_oth + __popc(gtb0) + __popc(gtb1));
-                            const unsigned lt = (1u << lane) - 1u;
-#pragma unroll 1
-                            for (int jj = 0; jj < 2; ++jj) {  // (rolled: one copy of the record write)
-                                const unsigned key = jj ? keys[1] : keys[0];
-                                const unsigned gtb = jj ? gtb1 : gtb0, eqb = jj ? eqb1 : eqb0;
-                                const unsigned gt_before = (warp ? g_oth : 0u) + (jj ? __popc(gtb0) : 0u);
-                                const unsigned e = (warp ? e_oth : 0u) + (jj ? __popc(eqb0) : 0u) + __popc(eqb & lt);
-                                if ((key > thr) || (key == thr && e < need_eq)) {
-                                    const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
-                                    const unsigned li = lbase + (unsigned)jj * 32u + lane;
-                                    DemoRecord r;
-                                    r.idx = cand_idx[li];
-                                    r.val = cand_val[li];
-                                    rec[pos] = r;
-                                    recs4[pos] = make_int4((r.idx >> LOG2S) * XS, (r.idx & (S - 1)) * S,
-                                                           __float_as_int(a.alpha * r.val), 0);
-                                }
-                            }
-                        }
-                    }
-                    if (slow) {
-                        select_slow(sm, k_eff, rec, a.alpha, t, slot + 1, lmin_w, bound_valid);
-                        sb.sync();  // every thread is done with the coefficient tile
-                        zero_row();
-                    }
-                }
+                select_chunk<false>(sm, q, k_eff, rec, a.alpha, t, sb, slot + 1, PAD_ROW);
                 sb.sync();  // records complete (shared list and global payload), tile zeroed
 
                 // ---- residual: row stage of the inverse from the k_eff records, sparse --------------
@@ -820,11 +901,11 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
 }
 
-template <typename GT, int THREADS>
+template <typename GT, int THREADS, bool QDOM>
 cudaError_t launch64(const DemoCompressArgs &a, int sm_count, cudaStream_t stream)
 {
     constexpr int NCH = THREADS / S;
-    auto kernel = compress64_kernel<GT, THREADS>;
+    auto kernel = compress64_kernel<GT, THREADS, QDOM>;
     const size_t smem = slot_bytes<GT>() * NCH + 16;
     if (a.n_chunks <= 0) return cudaSuccess;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -854,5 +935,9 @@ cudaError_t demo_launch_compress_fast64(const DemoCompressArgs &a, int sm_count,
 #ifndef DEMO_T64
 #define DEMO_T64 64
 #endif
-    return a.grad_bf16 ? launch64<__nv_bfloat16, DEMO_T64>(a, sm_count, stream) : launch64<float, DEMO_T64>(a, sm_count, stream);
+    if (a.momentum_dct)
+        return a.grad_bf16 ? launch64<__nv_bfloat16, DEMO_T64, true>(a, sm_count, stream)
+                           : launch64<float, DEMO_T64, true>(a, sm_count, stream);
+    return a.grad_bf16 ? launch64<__nv_bfloat16, DEMO_T64, false>(a, sm_count, stream)
+                       : launch64<float, DEMO_T64, false>(a, sm_count, stream);
 }

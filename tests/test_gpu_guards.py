@@ -15,8 +15,11 @@ pytestmark = pytest.mark.gpu
 
 SHAPES = [(256, 384), (128, 256), (128,), (384,)]
 
-# name, chunk, topk, gradient dtype, forced path, caller-supplied basis, chunk shapes (N-D context)
+# name, chunk, topk, gradient dtype, forced path ("dct": momentum kept in the transform domain), caller-supplied
+# basis, chunk shapes (N-D context)
 FAMILIES = [
+    ("fast_s64_momentum_dct", 64, 32, torch.bfloat16, "dct", False, None),
+    ("fast_s64_momentum_dct_k_above_s", 64, 128, torch.float32, "dct", False, None),
     ("fast_s32_bf16", 32, 8, torch.bfloat16, None, False, None),
     ("fast_s32_k_above_s", 32, 100, torch.bfloat16, None, False, None),
     ("fast_s64_bf16", 64, 32, torch.bfloat16, None, False, None),
@@ -39,6 +42,8 @@ def test_no_kernel_family_writes_outside_its_buffers(name, chunk, topk, gdtype, 
                             grad_dtype=gd, chunk_shapes=chunk_shapes)
     if path == "generic":
         tr.set_path(demo.DEMO_PATH_GENERIC)
+    if path == "dct":
+        tr.set_momentum_domain(demo.DEMO_MOMENTUM_DCT)
     if custom_basis:
         q, _ = np.linalg.qr(np.random.default_rng(5).standard_normal((chunk, chunk)))
         tr.set_basis(torch.from_numpy(np.ascontiguousarray(q, dtype=np.float32)))
