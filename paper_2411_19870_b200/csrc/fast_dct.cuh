@@ -346,6 +346,29 @@ FDCT_HD F2 f2_sub(F2 a, F2 b)
     return r;
 }
 
+FDCT_HD F2 f2_mul(F2 a, F2 b)
+{
+    F2 r;
+#if defined(__CUDA_ARCH__)
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+#else
+    r.lo = a.lo * b.lo;
+    r.hi = a.hi * b.hi;
+#endif
+    return r;
+}
+FDCT_HD F2 f2_fma(F2 a, F2 b, F2 c)
+{
+    F2 r;
+#if defined(__CUDA_ARCH__)
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+#else
+    r.lo = fmaf(a.lo, b.lo, c.lo);
+    r.hi = fmaf(a.hi, b.hi, c.hi);
+#endif
+    return r;
+}
+
 template <int N, class SC>
 FDCT_HD void dct4v(const F2 (&v)[N], F2 (&V)[N]);
 
@@ -391,10 +414,9 @@ FDCT_HD void dct4v(const F2 (&v)[N], F2 (&V)[N])
             constexpr float s = (float)(SC::value * c_sin(th));
             constexpr float cb = (float)(SC::value * sg * c_cos(th));
             constexpr float sb = (float)(SC::value * sg * c_sin(th));
-            const float l0 = f2_lo(v[n]), h0 = f2_lo(v[N - 1 - n]);
-            const float l1 = f2_hi(v[n]), h1 = f2_hi(v[N - 1 - n]);
-            a[n] = f2_make(fmaf(h0, s, l0 * c), fmaf(h1, s, l1 * c));
-            b[n] = f2_make(fmaf(h0, cb, -(l0 * sb)), fmaf(h1, cb, -(l1 * sb)));
+            // both vectors turn by the same angle: packed multiply and multiply-add (rounded like the scalar forms)
+            a[n] = f2_fma(v[N - 1 - n], f2_make(s, s), f2_mul(v[n], f2_make(c, c)));
+            b[n] = f2_fma(v[N - 1 - n], f2_make(cb, cb), f2_mul(v[n], f2_make(-sb, -sb)));
         });
         dct2v<H, ScaleOne>(a, A);
         dct2v<H, ScaleOne>(b, Bt);

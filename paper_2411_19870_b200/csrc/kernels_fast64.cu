@@ -590,7 +590,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
 
     // "row" of the padding entries of the row-stage list: the scratch line tmax[0..S) seen from X
     constexpr int PAD_ROW = (int)(region_bytes<GT>() / sizeof(float));
-    const int t = threadIdx.x % S, lane = t & 31, warp = t >> 5;
+    const int t = threadIdx.x % S;
     const int hw_warp = threadIdx.x >> 5;
     const SlotBarrier<S> sb{slot + 1};
     const uint32_t bar = smem_u32(bar_mem);
