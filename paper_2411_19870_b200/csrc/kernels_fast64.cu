@@ -352,6 +352,83 @@ __device__ __noinline__ void select_slow(const SlotMem sm, int k_eff, DemoRecord
 }
 
 // ------------------------------------------------------------------------------------------------
+// Last step of the in-line selection: the k_eff largest of the n_all candidates (all >= the bound `lmin_w`, at most
+// 32 * NK of them; list 0 holds the first n_w0 in ascending index order, list 1 the rest).  Every warp takes all
+// candidates into registers, NK keys per lane in list order, and searches bit by bit, from the first bit where the
+// bound and the largest key differ, for a threshold with exactly k_eff keys at or above it; the search stops as
+// soon as one is found.  If it runs out of bits, equal keys straddle the k_eff-th place: keys above the threshold
+// are kept, keys equal to it in index order until k_eff are reached.  A kept candidate's place among the records
+// is the number of kept candidates before it; warp w writes the records of the key groups w, w + 2, ...
+// ------------------------------------------------------------------------------------------------
+template <int NK, bool QDOM>
+__device__ __forceinline__ void ballot_select(const SlotMem &sm, unsigned n_w0, unsigned n_all, unsigned lmin_w, int k_eff,
+                                              DemoRecord *rec, float alpha, int lane, int warp)
+{
+    static_assert(NK == 2 || NK == 4, "two or four keys per lane");
+    auto list_pos = [&](unsigned i) { return i < n_w0 ? i : i - n_w0 + (unsigned)CAPWP; };
+    unsigned keys[NK];
+    unsigned hi = 0u;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        const unsigned i = (unsigned)j * 32u + lane;
+        keys[j] = (i < n_all) ? sm.cand_key[list_pos(i)] : 0u;
+        hi = max(hi, keys[j]);
+    }
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
+    unsigned thr = lmin_w & ~((2u << wb0) - 1u);
+    unsigned n_ge = n_all;  // every candidate is >= the bound >= thr
+#pragma unroll 1
+    for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
+        const unsigned cand = thr | (1u << b);
+        unsigned cnt = 0;
+#pragma unroll
+        for (int j = 0; j < NK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+        if (cnt >= (unsigned)k_eff) {
+            thr = cand;
+            n_ge = cnt;
+        }
+    }
+    unsigned gtb[NK], eqb[NK];
+    unsigned n_gt = 0;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        gtb[j] = __ballot_sync(0xffffffffu, keys[j] > thr);
+        eqb[j] = __ballot_sync(0xffffffffu, keys[j] == thr);
+        n_gt += __popc(gtb[j]);
+    }
+    const unsigned need_eq = (unsigned)k_eff - n_gt;
+    const unsigned lt = (1u << lane) - 1u;
+#pragma unroll 1
+    for (int jj = 0; jj < NK / 2; ++jj) {  // (rolled: one copy of the record write)
+        const bool second = (jj != 0);     // key groups 2, 3 (NK = 4 only)
+        const unsigned key = second ? (warp ? keys[NK - 1] : keys[NK - 2]) : (warp ? keys[1] : keys[0]);
+        const unsigned gb = second ? (warp ? gtb[NK - 1] : gtb[NK - 2]) : (warp ? gtb[1] : gtb[0]);
+        const unsigned eb = second ? (warp ? eqb[NK - 1] : eqb[NK - 2]) : (warp ? eqb[1] : eqb[0]);
+        // kept / equal candidates in the key groups before this one
+        unsigned gt_before = warp ? __popc(second ? gtb[NK - 2] : gtb[0]) : 0u;
+        unsigned eq_before = warp ? __popc(second ? eqb[NK - 2] : eqb[0]) : 0u;
+        if (second) {
+            gt_before += __popc(gtb[0]) + __popc(gtb[1]);
+            eq_before += __popc(eqb[0]) + __popc(eqb[1]);
+        }
+        const unsigned e = eq_before + __popc(eb & lt);
+        if ((key > thr) || (key == thr && e < need_eq)) {
+            const unsigned pos = gt_before + __popc(gb & lt) + min(e, need_eq);
+            const unsigned li = list_pos((unsigned)(2 * jj + warp) * 32u + lane);
+            DemoRecord r;
+            r.idx = sm.cand_idx[li];
+            r.val = sm.cand_val[li];
+            rec[pos] = r;
+            if (QDOM)  // what stays of a transmitted coefficient: q - alpha q
+                sm.X[(r.idx >> LOG2S) * XS + (r.idx & (S - 1))] = fmaf(-alpha, r.val, r.val);
+            else
+                sm.recs4[pos] = make_int4((r.idx >> LOG2S) * XS, (r.idx & (S - 1)) * S, __float_as_int(alpha * r.val), 0);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Exact top-k of one chunk (Section 2.1 "Top-k Sparsification"): thread t holds the coefficients q[v] = Q[t][v] of
 // row t.  Writes the k_eff records in ascending index order to `rec`; ends before the barrier that makes them
 // visible.  QDOM = false (momentum kept in the spatial domain): also leaves the pre-decoded row-stage list and the
@@ -476,7 +553,6 @@ __device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], i
                     cand_key[o] = mag_key(val);
                     ++o;
                 }
-                if (lane < 4) cand_key[lbase + n_cw + lane] = 0u;  // pad for the vector loads
             }
             sb.sync();
             const unsigned n_w0 = misc[0], n_w1 = misc[1];
@@ -485,64 +561,11 @@ __device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], i
             slow = (n_w0 > (unsigned)CAPW) || (n_w1 > (unsigned)CAPW) || (n_w0 + n_w1 < (unsigned)k_eff);
             if (!slow) {
                 zero_row();  // row t of the stash was read by this thread only
-                // Every warp takes both lists into registers (two keys per lane and list) and searches,
-                // bit by bit from the first bit where the bound and the largest key differ, for a
-                // threshold with exactly k_eff keys at or above it; the search stops as soon as one is
-                // found.  If it runs out of bits, equal keys straddle the k_eff-th place: keys above
-                // the threshold are kept, keys equal to it in index order until k_eff are reached.
-                const unsigned n_mine = warp ? n_w1 : n_w0, n_oth = warp ? n_w0 : n_w1;
-                const unsigned obase = (warp ^ 1) * CAPWP;
-                unsigned keys[4];  // 0, 1: this warp's list; 2, 3: the other warp's
-                keys[0] = (lane < n_mine) ? cand_key[lbase + lane] : 0u;
-                keys[1] = (lane + 32u < n_mine) ? cand_key[lbase + 32 + lane] : 0u;
-                keys[2] = (lane < n_oth) ? cand_key[obase + lane] : 0u;
-                keys[3] = (lane + 32u < n_oth) ? cand_key[obase + 32 + lane] : 0u;
-                const unsigned hi = __reduce_max_sync(0xffffffffu, max(max(keys[0], keys[1]), max(keys[2], keys[3])));
-                const int wb0 = 31 - __clz((lmin_w ^ hi) | 1u);
-                unsigned thr = lmin_w & ~((2u << wb0) - 1u);
-                unsigned n_ge = n_w0 + n_w1;  // every candidate is >= the bound >= thr
-#pragma unroll 1
-                for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
-                    const unsigned cand = thr | (1u << b);
-                    unsigned cnt = 0;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
-                    if (cnt >= (unsigned)k_eff) {
-                        thr = cand;
-                        n_ge = cnt;
-                    }
-                }
-                // kept entries before this warp's list (index order: list 0, then list 1) and in all
-                const unsigned g_oth = __popc(__ballot_sync(0xffffffffu, keys[2] > thr)) +
-                                       __popc(__ballot_sync(0xffffffffu, keys[3] > thr));
-                const unsigned e_oth = __popc(__ballot_sync(0xffffffffu, keys[2] == thr)) +
-                                       __popc(__ballot_sync(0xffffffffu, keys[3] == thr));
-                const unsigned gtb0 = __ballot_sync(0xffffffffu, keys[0] > thr);
-                const unsigned gtb1 = __ballot_sync(0xffffffffu, keys[1] > thr);
-                const unsigned eqb0 = __ballot_sync(0xffffffffu, keys[0] == thr);
-                const unsigned eqb1 = __ballot_sync(0xffffffffu, keys[1] == thr);
-                const unsigned need_eq = (unsigned)k_eff - (g_oth + __popc(gtb0) + __popc(gtb1));
-                const unsigned lt = (1u << lane) - 1u;
-#pragma unroll 1
-                for (int jj = 0; jj < 2; ++jj) {  // (rolled: one copy of the record write)
-                    const unsigned key = jj ? keys[1] : keys[0];
-                    const unsigned gtb = jj ? gtb1 : gtb0, eqb = jj ? eqb1 : eqb0;
-                    const unsigned gt_before = (warp ? g_oth : 0u) + (jj ? __popc(gtb0) : 0u);
-                    const unsigned e = (warp ? e_oth : 0u) + (jj ? __popc(eqb0) : 0u) + __popc(eqb & lt);
-                    if ((key > thr) || (key == thr && e < need_eq)) {
-                        const unsigned pos = gt_before + __popc(gtb & lt) + min(e, need_eq);
-                        const unsigned li = lbase + (unsigned)jj * 32u + lane;
-                        DemoRecord r;
-                        r.idx = cand_idx[li];
-                        r.val = cand_val[li];
-                        rec[pos] = r;
-                        if (QDOM)  // what stays of a transmitted coefficient: q - alpha q
-                            X[(r.idx >> LOG2S) * XS + (r.idx & (S - 1))] = fmaf(-alpha, r.val, r.val);
-                        else
-                            recs4[pos] = make_int4((r.idx >> LOG2S) * XS, (r.idx & (S - 1)) * S,
-                                                   __float_as_int(alpha * r.val), 0);
-                    }
-                }
+                // the two lists, read one behind the other, are in ascending index order
+                if (n_w0 + n_w1 <= 64u)
+                    ballot_select<2, QDOM>(sm, n_w0, n_w0 + n_w1, lmin_w, k_eff, rec, alpha, lane, warp);
+                else
+                    ballot_select<4, QDOM>(sm, n_w0, n_w0 + n_w1, lmin_w, k_eff, rec, alpha, lane, warp);
             }
         }
         if (slow) {
