@@ -454,10 +454,25 @@ __device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], i
 #pragma unroll
         for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(0.f, 0.f, 0.f, 0.f);
     };
-    auto stash_row = [&]() {
+    // The stash of row t.  With the momentum in the spatial domain it is written in the transform core's own order
+    // (position p holds coefficient core_index(p)): the registers of a 128-bit store are then neighbours in the
+    // core's output, as the pairs of the inverse cascade are, and no register moves are needed to satisfy both.
+    constexpr bool CORE_STASH = !QDOM;
+    auto stash_row = [&](auto core_order) {
         float4 *row = reinterpret_cast<float4 *>(X + t * XS);
-#pragma unroll
-        for (int v4 = 0; v4 < S / 4; ++v4) row[v4] = make_float4(q[4 * v4], q[4 * v4 + 1], q[4 * v4 + 2], q[4 * v4 + 3]);
+        fdct::static_for<0, S / 4>([&](auto i) {
+            constexpr int v4 = decltype(i)::value;
+            constexpr bool CO = decltype(core_order)::value;
+            constexpr int i0 = CO ? fdct::core_index<S>(4 * v4) : 4 * v4, i1 = CO ? fdct::core_index<S>(4 * v4 + 1) : 4 * v4 + 1;
+            constexpr int i2 = CO ? fdct::core_index<S>(4 * v4 + 2) : 4 * v4 + 2, i3 = CO ? fdct::core_index<S>(4 * v4 + 3) : 4 * v4 + 3;
+            row[v4] = make_float4(q[i0], q[i1], q[i2], q[i3]);
+        });
+    };
+    // position of coefficient v in a stash kept in core order: v = (2j + 1) << s sits at (32 >> s) + j, v = 0 at 0
+    auto stash_pos = [](int v) {
+        if (!CORE_STASH) return v;
+        const int sft = __ffs(v | S) - 1;
+        return ((S / 2) >> sft) + (v >> (sft + 1));
     };
     // ---- exact top-k (Section 2.1 "Top-k Sparsification") -------------------------------
     if (!QDOM) {
@@ -533,10 +548,10 @@ __device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], i
         }
         if (!QDOM && t < k_eff) recs4[t] = make_int4(0, 0, 0, 0);
         zero_row();
-        if (QDOM) stash_row();  // (all zero; the tile is the kernel's output)
+        if (QDOM) stash_row(std::false_type{});  // (all zero; the tile is the kernel's output)
     } else {
         // stash the coefficients of row t (own row: no hazard with other threads)
-        stash_row();
+        stash_row(std::integral_constant<bool, CORE_STASH>{});
         if (!slow) {
             const unsigned lbase = warp * CAPWP;
             if (n_cw <= CAPW) {
@@ -547,7 +562,7 @@ __device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], i
                 while (mask) {
                     const int v = __ffsll((long long)mask) - 1;
                     mask &= mask - 1ull;
-                    const float val = X[t * XS + v];
+                    const float val = X[t * XS + stash_pos(v)];
                     cand_idx[o] = t * S + v;
                     cand_val[o] = val;
                     cand_key[o] = mag_key(val);
@@ -569,6 +584,7 @@ __device__ __forceinline__ void select_chunk(const SlotMem &sm, float (&q)[S], i
             }
         }
         if (slow) {
+            if (CORE_STASH) stash_row(std::false_type{});  // the out-of-line selection reads the tile in index order
             select_slow(sm, k_eff, rec, alpha, t, bar_id, lmin_w, bound_valid, QDOM);
             sb.sync();  // every thread is done with the coefficient tile
             zero_row();
