@@ -877,7 +877,7 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) compress64_kernel(Demo
                             for (int j = 1; j < ROW_AHEAD + 1; ++j) rc[j] = recs4[r0 + j];
                             nx = rc[ROW_AHEAD];
 #pragma unroll
-                            for (int j = 0; j < ROW_AHEAD; ++j) cv[j] = __ldg(Ct + rc[j].y);
+                            for (int j = 0; j < ROW_AHEAD; ++j) cv[j] = __ldg(a.C + (unsigned)(rc[j].y + t));
 #pragma unroll
                             for (int j = 0; j < ROW_AHEAD; ++j) {
                                 acc = fmaf(__int_as_float(rc[j].z), cv[j], acc);
