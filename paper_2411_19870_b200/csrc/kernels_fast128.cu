@@ -10,10 +10,11 @@
 //     e = DCT-III_64(X[even]),  o = DCT-IV_64(X[odd]),  x[n] = e[n] + o[n],  x[127-n] = e[n] - o[n]
 // with e and o exchanged between the two threads of a line through shared memory.
 //
-// compress: TMA-staged m and g tiles -> B = beta*m + g -> column pass -> row pass -> coefficients in
-// shared memory -> exact radix select (4 x 8 bits on the magnitude) + index-ordered compaction ->
-// records; sparse row stage of the inverse from the records, fast column stage, m and g fetched again
-// (L2) for the residual m <- B - IDCT(kept).  decode: scatter-add of the W payloads in worker order,
+// compress: TMA-staged m and g tiles -> B = beta*m + g (each thread parks the half column it will write back in
+// tensor memory) -> column pass -> row pass -> coefficients in shared memory -> exact top-k (bound from the 256
+// half-row maxima, candidate list, exact ranking; radix select for degenerate chunks) -> records; sparse row
+// stage of the inverse from the records, fast column stage, residual m <- B - alpha * IDCT(kept) against the
+// parked B, one TMA store of the new momentum tile.  decode: scatter-add of the W payloads in worker order,
 // two inverse passes, sign, update; the x tile is staged into the (then dead) coefficient tile.
 // Tiles need the TMA tensor maps; without them the host uses the generic kernels for s = 128.
 #include <cuda_bf16.h>
@@ -31,6 +32,9 @@ constexpr int S = 128, H = 64, XS = S + 4, M = S * S, THREADS = 256;
 // different rows (the row pass) on 32 different banks; S + 4 (compress: 128-bit row accesses) gives 4-way
 // conflicts there.
 constexpr int XSD = S + 1;
+constexpr int RECS128 = 128 + 16;     // row-stage list: up to 128 kept records + padding for the look-ahead
+constexpr int ROW_AHEAD128 = 8;       // entries of the row-stage list fetched ahead of the accumulation
+constexpr int TMEM_COLS128 = 128;     // tensor-memory columns of a compress CTA (two CTAs per SM)
 constexpr int CAP128 = 256;           // candidate capacity of the fast top-k (one per thread)
 constexpr int CAP128P = CAP128 + 4;   // padded for 128-bit key loads
 using SC = fdct::ScaleOrtho<S>;
@@ -78,7 +82,7 @@ constexpr size_t compress128_tile_bytes()
 template <typename GT>
 constexpr size_t compress128_smem()
 {
-    return compress128_tile_bytes<GT>() + (256 + 8 + 4) * 4 + 128 * 16 + 3 * CAP128P * 4 + 16;
+    return compress128_tile_bytes<GT>() + (256 + 8 + 4) * 4 + RECS128 * 16 + 3 * CAP128P * 4 + 16 + 16;
 }
 
 template <typename GT>
@@ -92,11 +96,12 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
     unsigned *hist = reinterpret_cast<unsigned *>(smem_raw + compress128_tile_bytes<GT>());  // [256]
     unsigned *warp_tot = hist + 256;                                                         // [8]
     unsigned *s_state = warp_tot + 8;                                                        // [4]
-    int4 *recs4 = reinterpret_cast<int4 *>(s_state + 4);                                     // [128]
-    unsigned *cand_key = reinterpret_cast<unsigned *>(recs4 + 128);                          // [CAP128P]
+    int4 *recs4 = reinterpret_cast<int4 *>(s_state + 4);                                     // [RECS128]
+    unsigned *cand_key = reinterpret_cast<unsigned *>(recs4 + RECS128);                      // [CAP128P]
     float *cand_val = reinterpret_cast<float *>(cand_key + CAP128P);                         // [CAP128P]
     int *cand_idx = reinterpret_cast<int *>(cand_val + CAP128P);                             // [CAP128P]
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(cand_idx + CAP128P);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_mem + 2);
 
     const int tid = threadIdx.x, h = tid >> 7, j = tid & 127;
     const uint32_t bar = smem_u32(bar_mem);
@@ -104,8 +109,11 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
         mbar_init(bar, 1);
         fence_proxy_async();
     }
-    __syncthreads();
+    // Tensor memory as storage: thread (h, j) parks its 64 elements of column j of B = beta*m + g (rows 0..63 for
+    // h = 0, rows 127..64 for h = 1) in lane j, columns 64h .. 64h+63, between the forward pass and the residual.
+    const uint32_t tmem_base = tmem_alloc_cta(tmem_slot, TMEM_COLS128);
     fence_proxy_async();
+    const uint32_t taddr = tmem_base + ((uint32_t)(j & ~31) << 16) + (uint32_t)(h * H);
 
     EntryCursor cur;
     unsigned phase = 0;
@@ -142,12 +150,12 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
         const int k_eff = te.k_eff;
         DemoRecord *rec = a.payload + te.rec_begin + (long long)lc * k_eff;
 
-        bool arrived = mbar_wait_bounded(bar, phase);
+        const bool arrived = mbar_wait_bounded(bar, phase);
         phase ^= 1u;
         if (!__syncthreads_and(arrived)) {
             if (tid == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
-            mbar_wait_bounded(bar, phase ^ 1u);
-            return;
+            mbar_wait_bounded(bar, phase ^ 1u);  // give copies in flight one more bounded chance to land
+            break;
         }
 
         // ---- two forward passes through one rolled copy of the half-transforms ---------------------
@@ -155,12 +163,21 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
             if (pass == 0) {
-                // column j of B = beta*m + g, folded: in[n] = B[n][j] +/- B[127-n][j]
+                // column j of B = beta*m + g, folded: in[n] = B[n][j] +/- B[127-n][j]; the half of the column that
+                // this thread will write back is parked in tensor memory (two stores of 32 columns)
+                const float sg = h ? -1.f : 1.f;
 #pragma unroll
-                for (int n = 0; n < H; ++n) {
-                    const float lo = fmaf(a.beta, Ms[n * S + j], to_f32(Gs[n * S + j]));
-                    const float hi = fmaf(a.beta, Ms[(S - 1 - n) * S + j], to_f32(Gs[(S - 1 - n) * S + j]));
-                    in[n] = h ? lo - hi : lo + hi;
+                for (int half = 0; half < 2; ++half) {
+                    float park[32];
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) {
+                        const int n = 32 * half + q;
+                        const float lo = fmaf(a.beta, Ms[n * S + j], to_f32(Gs[n * S + j]));
+                        const float hi = fmaf(a.beta, Ms[(S - 1 - n) * S + j], to_f32(Gs[(S - 1 - n) * S + j]));
+                        in[n] = fmaf(sg, hi, lo);
+                        park[q] = h ? hi : lo;
+                    }
+                    tmem_st32(taddr + 32 * half, park);
                 }
                 __syncthreads();  // the staged tiles are consumed (X aliases them)
             } else {
@@ -195,6 +212,9 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
         // candidates are listed in index order and ranked exactly, ties to the lowest index.  Everything
         // compares integer magnitude keys, so NaN and Inf are ordered like any other bit pattern.  More
         // than CAP128 candidates (tied or degenerate chunks) or k_eff > 256: radix select below.
+        // the row-stage list is padded with zero-valued entries whose "row" is a scratch line behind the tile
+        // (ordered before the record writes by the barriers below)
+        if (tid < RECS128) recs4[tid] = make_int4(S * XS, 0, 0, 0);
         bool use_radix = k_eff > 256;
         if (!use_radix) {
             const float4 *mine4 = reinterpret_cast<const float4 *>(X + (tid >> 1) * XS + 64 * (tid & 1));
@@ -394,30 +414,44 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
         // ---- residual: sparse row stage T[u][j] = sum over kept (u, v) of val * C[v][j] ------------
         for (int i = tid; i < S * XS / 4; i += THREADS) reinterpret_cast<float4 *>(X)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         __syncthreads();
-        if (h == 0) {
+        if (h == 0 && k_eff <= 128) {
+            // The running sum of a row is stored after every entry (the last store of a row carries the whole sum)
+            // and starts again from zero when the next entry belongs to another row: no branch in the loop.
+            // Entries and their cosines are fetched ahead of the dependent accumulation.
+            float *Xj = X + j;
+            float acc = 0.f;
+            int4 nx = recs4[0];
+#pragma unroll 1
+            for (int r0 = 0; r0 < k_eff; r0 += ROW_AHEAD128) {
+                int4 rc[ROW_AHEAD128 + 1];
+                float cv[ROW_AHEAD128];
+                rc[0] = nx;
+#pragma unroll
+                for (int q = 1; q < ROW_AHEAD128 + 1; ++q) rc[q] = recs4[r0 + q];
+                nx = rc[ROW_AHEAD128];
+#pragma unroll
+                for (int q = 0; q < ROW_AHEAD128; ++q) cv[q] = __ldg(a.C + (unsigned)(rc[q].y + j));
+#pragma unroll
+                for (int q = 0; q < ROW_AHEAD128; ++q) {
+                    acc = fmaf(__int_as_float(rc[q].z), cv[q], acc);
+                    Xj[rc[q].x] = acc;
+                    acc = (rc[q].x != rc[q + 1].x) ? 0.f : acc;
+                }
+            }
+        } else if (h == 0) {
+            // k > 128: the records come from the payload itself
             const float *Cj = a.C + j;
             float acc = 0.f;
             int cur_u = -1;
             for (int r = 0; r < k_eff; ++r) {
-                int uo, vo;
-                float val;
-                if (k_eff <= 128) {
-                    const int4 rc = recs4[r];
-                    uo = rc.x;
-                    vo = rc.y;
-                    val = __int_as_float(rc.z);
-                } else {
-                    const DemoRecord rc = rec[r];
-                    uo = (rc.idx >> 7) * XS;
-                    vo = (rc.idx & 127) * S;
-                    val = a.alpha * rc.val;
-                }
+                const DemoRecord rc = rec[r];
+                const int uo = (rc.idx >> 7) * XS;
                 if (uo != cur_u) {
                     if (cur_u >= 0) X[cur_u + j] = acc;
                     acc = 0.f;
                     cur_u = uo;
                 }
-                acc = fmaf(val, __ldg(Cj + vo), acc);
+                acc = fmaf(a.alpha * rc.val, __ldg(Cj + (rc.idx & 127) * S), acc);
             }
             if (cur_u >= 0) X[cur_u + j] = acc;
         }
@@ -429,8 +463,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
         fence_proxy_async();
         __syncthreads();  // T is in registers: the tile area is free
         inverse_half(h, in, out);
-        // exchange e and o through the tile area (the staged tiles would overlap it, so they are
-        // fetched again only after the exchange)
+        // exchange e and o through the tile area
         float *Ex = X;  // [2][64][128]
 #pragma unroll
         for (int n = 0; n < H; ++n) Ex[(h * H + n) * S + j] = out[n];
@@ -440,29 +473,34 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
             const float other = Ex[((h ^ 1) * H + n) * S + j];
             out[n] = h ? other - out[n] : out[n] + other;  // h=0: x[n] = e+o;  h=1: x[127-n] = e-o
         }
-        fence_proxy_async();
-        __syncthreads();
-        issue_tiles(te, c);
-        arrived = mbar_wait_bounded(bar, phase);
-        phase ^= 1u;
-        if (!__syncthreads_and(arrived)) {
-            if (tid == 0) atomicMax(a.status, DEMO_DEV_TIMEOUT);
-            mbar_wait_bounded(bar, phase ^ 1u);
-            return;
-        }
+        __syncthreads();  // the exchange area is read: the new momentum tile takes its place
+        // m <- B - alpha * IDCT(kept): B comes back from tensor memory; the dense tile goes out in one TMA store
+        tmem_wait_st();
 #pragma unroll
-        for (int n = 0; n < H; ++n) {
-            const int row = h ? (S - 1 - n) : n;
-            m[base + (size_t)row * te.n1 + j] = fmaf(a.beta, Ms[row * S + j], to_f32(Gs[row * S + j])) - out[n];
+        for (int half = 0; half < 2; ++half) {
+            float b[32];
+            tmem_ld32(taddr + 32 * half, b);
+            if (h) {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) Ms[(S - 1 - (32 * half + q)) * S + j] = b[q] - out[32 * half + q];
+            } else {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) Ms[(32 * half + q) * S + j] = b[q] - out[32 * half + q];
+            }
         }
         fence_proxy_async();
         __syncthreads();
         const long long nc = c + gridDim.x;
-        if (nc < a.n_chunks) {
-            cur.seek(a.entries, a.n_entries, nc);
-            issue_tiles(cur.te, nc);
+        if (nc < a.n_chunks) cur.seek(a.entries, a.n_entries, nc);
+        if (tid == 0) {
+            tma_store_2d(static_cast<const char *>(a.tmap_m) + (size_t)te.tensor * TMAP_BYTES, (int)(k1 * S), (int)(k0 * S),
+                         smem_u32(Ms));
+            tma_store_commit();
+            tma_store_wait_read();  // the store has read the tile: the next chunk's tiles may land
         }
+        if (nc < a.n_chunks) issue_tiles(cur.te, nc);
     }
+    tmem_free_cta(tmem_base, TMEM_COLS128);
 }
 
 constexpr size_t decode128_smem(bool counts) { return (size_t)S * XSD * 4 + 16 + (counts ? (size_t)M * 2 : 0); }
@@ -618,9 +656,10 @@ cudaError_t launch128(K kernel, size_t smem, long long n_chunks, int sm_count, c
     if (n_chunks <= 0) return cudaSuccess;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    int per_sm = 0;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, THREADS, smem);
-    if (err != cudaSuccess) return err;
+    // CTAs per SM: two by the launch bounds (registers), fewer if shared memory (227 KB, 1 KB reserved per CTA) says
+    // so.  The occupancy calculator is not asked: it answers 1 for a kernel that allocates tensor memory.
+    int per_sm = (int)((227u * 1024u) / (smem + 1024u));
+    if (per_sm > 2) per_sm = 2;
     if (per_sm < 1) per_sm = 1;
     long long grid = (long long)sm_count * per_sm;
     if (grid > n_chunks) grid = n_chunks;
