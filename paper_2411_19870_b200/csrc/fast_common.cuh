@@ -287,4 +287,60 @@ __device__ __forceinline__ void tmem_free_cta(uint32_t base, uint32_t cols)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
 }
 
+// ------------------------------------------------------------------------------------------------
+// One warp picks the k_eff largest of n_all candidate keys (all >= the bound `lmin`, n_all <= 32 * NK; list order
+// is index order).  NK keys per lane, in list order.  Bit by bit, from the first bit where the bound and the
+// largest key differ, it looks for a threshold with exactly k_eff keys at or above it and stops as soon as one is
+// found; if the bits run out, equal keys straddle the k_eff-th place: keys above the threshold are kept, keys equal
+// to it in list order until k_eff are reached.  emit(pos, li) is called for every kept candidate: li its list
+// position, pos its place among the kept ones (ascending list order).
+// ------------------------------------------------------------------------------------------------
+template <int NK, class Emit>
+__device__ __forceinline__ void warp_ballot_select(const unsigned *cand_key, unsigned n_all, unsigned lmin, int k_eff,
+                                                   int lane, Emit emit)
+{
+    unsigned keys[NK];
+    unsigned hi = 0u;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        const unsigned i = (unsigned)j * 32u + lane;
+        keys[j] = (i < n_all) ? cand_key[i] : 0u;
+        hi = max(hi, keys[j]);
+    }
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    const int wb0 = 31 - __clz((lmin ^ hi) | 1u);
+    unsigned thr = lmin & ~((2u << wb0) - 1u);
+    unsigned n_ge = n_all;  // every candidate is >= the bound >= thr
+#pragma unroll 1
+    for (int b = wb0; b >= 0 && n_ge != (unsigned)k_eff; --b) {
+        const unsigned cand = thr | (1u << b);
+        unsigned cnt = 0;
+#pragma unroll
+        for (int j = 0; j < NK; ++j) cnt += __popc(__ballot_sync(0xffffffffu, keys[j] >= cand));
+        if (cnt >= (unsigned)k_eff) {
+            thr = cand;
+            n_ge = cnt;
+        }
+    }
+    unsigned gtb[NK], eqb[NK];
+    unsigned n_gt = 0;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        gtb[j] = __ballot_sync(0xffffffffu, keys[j] > thr);
+        eqb[j] = __ballot_sync(0xffffffffu, keys[j] == thr);
+        n_gt += __popc(gtb[j]);
+    }
+    const unsigned need_eq = (unsigned)k_eff - n_gt;
+    const unsigned lt = (1u << lane) - 1u;
+    unsigned gt_before = 0, eq_before = 0;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        const unsigned e = eq_before + __popc(eqb[j] & lt);
+        if ((keys[j] > thr) || (keys[j] == thr && e < need_eq))
+            emit(gt_before + __popc(gtb[j] & lt) + min(e, need_eq), (unsigned)j * 32u + lane);
+        gt_before += __popc(gtb[j]);
+        eq_before += __popc(eqb[j]);
+    }
+}
+
 }  // namespace fastk

@@ -221,12 +221,20 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
             const int lane = tid & 31, warp = tid >> 5;
             // the two halves of a row sit 256 bytes apart (same banks): the odd one starts 4 pieces later
             const int rot = 4 * (tid & 1);
-            unsigned tkey = 0u;
+            // the 64 values stay in registers for the candidate mask (group i4 holds piece (i4 + rot) mod 16)
+            float v[64];
+            float tm = 0.f;
 #pragma unroll
             for (int i4 = 0; i4 < 16; ++i4) {
                 const float4 f = mine4[(i4 + rot) & 15];
-                tkey = max(max(tkey, mag_key(f.x)), max(mag_key(f.y), max(mag_key(f.z), mag_key(f.w))));
+                v[4 * i4 + 0] = f.x;
+                v[4 * i4 + 1] = f.y;
+                v[4 * i4 + 2] = f.z;
+                v[4 * i4 + 3] = f.w;
+                tm = max3f(tm, fabsf(f.x), fabsf(f.y));
+                tm = max3f(tm, fabsf(f.z), fabsf(f.w));
             }
+            const unsigned tkey = __float_as_uint(tm);
             hist[tid] = tkey;
             __syncthreads();
             if (warp == 0) {
@@ -270,14 +278,23 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                     if (k_eff <= 128) recs4[tid] = make_int4((tid >> 7) * XS, (tid & 127) * S, 0, 0);
                 }
             } else {
-            // candidates of this thread as a bit mask over its 64 values
-            unsigned long long mask = 0ull;
+            // candidates of this thread as a bit mask over its 64 values: |q| >= L  <=>  |q| > Lm (the float just
+            // below L); the sign bit of Lm - |q| is funnel-shifted into the mask (independent chains of 16), which is
+            // then turned from register order into index order
+            unsigned long long mask;
+            {
+                const float Lm = (lmin > 0u) ? __uint_as_float(lmin - 1u) : -1.f;
+                unsigned mc[4];
 #pragma unroll
-            for (int i4 = 0; i4 < 16; ++i4) {
-                const float4 f = mine4[i4];
-                const unsigned nib = (unsigned)(mag_key(f.x) >= lmin) | ((unsigned)(mag_key(f.y) >= lmin) << 1) |
-                                     ((unsigned)(mag_key(f.z) >= lmin) << 2) | ((unsigned)(mag_key(f.w) >= lmin) << 3);
-                mask |= (unsigned long long)nib << (4 * i4);
+                for (int ch = 0; ch < 4; ++ch) {
+                    unsigned mm = 0u;
+#pragma unroll
+                    for (int q = 15; q >= 0; --q) mm = __funnelshift_l(__float_as_uint(Lm - fabsf(v[16 * ch + q])), mm, 1);
+                    mc[ch] = mm;
+                }
+                const unsigned long long mreg =
+                    ((unsigned long long)(mc[2] | (mc[3] << 16)) << 32) | (unsigned long long)(mc[0] | (mc[1] << 16));
+                mask = (tid & 1) ? ((mreg << 16) | (mreg >> 48)) : mreg;
             }
             const unsigned cnt = (unsigned)__popcll(mask);
             unsigned o = block_exclusive_scan(cnt, warp_tot);
@@ -296,33 +313,21 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                     cand_idx[o] = 64 * tid + e;
                     ++o;
                 }
-                if (tid < 4) cand_key[n_cand + tid] = 0u;  // pad for the vector loads
                 __syncthreads();
-                // exact rank of candidate tid among all candidates (list order = index order)
-                bool sel = false;
-                if ((unsigned)tid < n_cand) {
-                    const unsigned key = cand_key[tid];
-                    unsigned rank = 0;
-                    const uint4 *keys4 = reinterpret_cast<const uint4 *>(cand_key);
-                    const unsigned n4 = (n_cand + 3u) >> 2;
-                    for (unsigned c4 = 0; c4 < n4; ++c4) {
-                        const uint4 k4 = keys4[c4];
-                        const unsigned j0 = 4u * c4;
-                        rank += (k4.x > key) || (k4.x == key && j0 < (unsigned)tid);
-                        rank += (k4.y > key) || (k4.y == key && j0 + 1u < (unsigned)tid);
-                        rank += (k4.z > key) || (k4.z == key && j0 + 2u < (unsigned)tid);
-                        rank += (k4.w > key) || (k4.w == key && j0 + 3u < (unsigned)tid);
-                    }
-                    sel = rank < (unsigned)k_eff;
-                }
-                const unsigned pos = block_exclusive_scan(sel ? 1u : 0u, warp_tot);
-                if (sel) {
-                    DemoRecord r;
-                    r.idx = cand_idx[tid];
-                    r.val = cand_val[tid];
-                    rec[pos] = r;
-                    if (k_eff <= 128)
-                        recs4[pos] = make_int4((r.idx >> 7) * XS, (r.idx & 127) * S, __float_as_int(a.alpha * r.val), 0);
+                // the first warp picks the k_eff largest candidates (list order = index order) and writes the records
+                if (warp == 0) {
+                    auto emit = [&](unsigned pos, unsigned li) {
+                        DemoRecord r;
+                        r.idx = cand_idx[li];
+                        r.val = cand_val[li];
+                        rec[pos] = r;
+                        if (k_eff <= 128)
+                            recs4[pos] = make_int4((r.idx >> 7) * XS, (r.idx & 127) * S, __float_as_int(a.alpha * r.val), 0);
+                    };
+                    if (n_cand <= 64u)
+                        warp_ballot_select<2>(cand_key, n_cand, lmin, k_eff, lane, emit);
+                    else
+                        warp_ballot_select<8>(cand_key, n_cand, lmin, k_eff, lane, emit);
                 }
             }
             }  // !zero_chunk
