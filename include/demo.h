@@ -114,9 +114,15 @@ demo_status demo_init(demo_ctx **out, const demo_config *cfg, const demo_tensor_
  * (k_0, ..., k_{d-1}); all tensors run on one family of kernels that apply the transform axis by axis as
  * dense contractions on the CUDA cores (no fast-DCT, tensor-core or side-stream path; demo_set_path has
  * no effect); demo_set_basis, demo_set_basis_gaussian and demo_get_basis return UNSUPPORTED (one basis
- * per chunk extent: only the DCT is built).  A descriptor with ndim <= 2 and equal chunk extents gives
- * the payload layout of demo_init with that chunk size and, up to the fp32 rounding of a different
- * summation order, the same records.
+ * per chunk extent: only the DCT is built).  A descriptor whose chunk is an s x s tile of its last two axes
+ * or a length-s segment of its last axis (all other chunk extents 1) gives the payload layout of demo_init
+ * with chunk size s on the tensor flattened to its last two axes / last axis and, up to the fp32 rounding of a
+ * different summation order, the same records.
+ *
+ * When EVERY descriptor is of that form with one common s in {8, 16, 32, 64, 128}, the context is that of
+ * demo_init: it is built by demo_init on the flattened tensors (topk above s * s is lowered to s * s, which
+ * leaves every k_eff unchanged) and is in every respect such a context -- fast-DCT and tensor-map kernels,
+ * demo_set_path, caller-supplied bases, demo_set_momentum_domain.
  * Errors: INVALID_ARG, SHAPE (ndim, chunk[a] < 1, shape[a] not a multiple of chunk[a]), K,
  * UNSUPPORTED (chunk extent or chunk too large, dtype, too many tensors), ALLOC, CUDA.
  */

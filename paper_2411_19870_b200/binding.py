@@ -321,10 +321,28 @@ class DemoTransform:
 
     def _host_matrix(self, a):
         a = a.detach().to("cpu", torch.float32).contiguous() if isinstance(a, torch.Tensor) else torch.tensor(a, dtype=torch.float32)
-        s = self.cfg.chunk
-        if tuple(a.shape) != (s, s):
+        s = self.basis_dim
+        if a.dim() != 2 or a.shape[0] != a.shape[1] or (s and a.shape[0] != s):
             raise ValueError("expected an s x s matrix")
         return a
+
+    @property
+    def basis_dim(self) -> int:
+        """The s of the s x s basis: the chunk size, also for a ``chunk_shapes`` context whose chunks are all s x s
+        tiles / length-s segments behind leading extents of 1 (the library builds that one with ``demo_init``);
+        0 for other ``chunk_shapes`` contexts, which have no caller-supplied basis."""
+        if self.chunk_shapes is None:
+            return self.cfg.chunk
+        sizes = set()
+        for c in self.chunk_shapes:
+            lead = 0
+            while lead < len(c) - 1 and c[lead] == 1:
+                lead += 1
+            if len(c) - lead > 2:
+                return 0
+            sizes.update(c[lead:])
+        s = sizes.pop() if len(sizes) == 1 else 0
+        return s if s in (8, 16, 32, 64, 128) else 0
 
     def set_basis(self, basis=None, stream=None) -> None:
         """s x s matrix whose rows are the basis vectors (host or device tensor); None restores the DCT."""
@@ -341,8 +359,8 @@ class DemoTransform:
             raise DemoError(st, "demo_set_basis_gaussian")
 
     def get_basis(self, stream=None) -> torch.Tensor:
-        s = self.cfg.chunk
-        out = torch.empty((s, s), dtype=torch.float32)
+        s = self.basis_dim
+        out = torch.empty((max(s, 1), max(s, 1)), dtype=torch.float32)
         st = self.lib.demo_get_basis(self._ctx, out.data_ptr(), self._stream(stream))
         if st != 0:
             raise DemoError(st, "demo_get_basis")

@@ -383,6 +383,47 @@ demo_status demo_init_nd(demo_ctx **out, const demo_config *cfg, const demo_nd_t
         }
     }
 
+    // Square chunks of one size: when every tensor is cut into s x s tiles of its last two axes or into length-s
+    // segments of its last axis (all leading chunk extents 1, so the leading axes merely stack rows), for one s
+    // that demo_init knows, the layout of chunks and records is that of demo_init on the flattened tensors -- the
+    // context is built by it and runs its kernels (fast DCT, tensor maps, side stream).
+    {
+        int s_common = 0;
+        bool regular = true;
+        std::vector<demo_tensor_desc> flat;
+        try {
+            flat.resize((size_t)n_tensors);
+        } catch (const std::bad_alloc &) {
+            return DEMO_ERR_ALLOC;
+        }
+        for (int t = 0; t < n_tensors && regular; ++t) {
+            const demo_nd_tensor_desc &d = tensors[t];
+            int lead = 0;
+            while (lead < d.ndim - 1 && d.chunk[lead] == 1) ++lead;
+            const int rest = d.ndim - lead;  // axes that are really cut: 1 or 2
+            if (rest > 2) {
+                regular = false;
+                break;
+            }
+            long long rows = 1;
+            for (int a = 0; a < lead; ++a) rows *= d.shape[a];
+            for (int a = lead; a < d.ndim; ++a) {
+                if (s_common == 0) s_common = d.chunk[a];
+                if (d.chunk[a] != s_common) regular = false;
+            }
+            flat[t].ndim = rest;
+            flat[t].shape[0] = rows * d.shape[lead];
+            flat[t].shape[1] = rest == 2 ? d.shape[lead + 1] : 0;
+            if (flat[t].shape[0] > (1LL << 31) - 1) regular = false;
+        }
+        if (regular && (s_common == 8 || s_common == 16 || s_common == 32 || s_common == 64 || s_common == 128)) {
+            demo_config sq = *cfg;
+            sq.chunk = s_common;
+            if ((long long)sq.topk > (long long)s_common * s_common) sq.topk = s_common * s_common;  // same k_eff
+            return demo_init(out, &sq, flat.data(), n_tensors, cuda_device);
+        }
+    }
+
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cuda_device >= n_dev) {
         cudaGetLastError();

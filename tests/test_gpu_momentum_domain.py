@@ -90,8 +90,8 @@ def test_refused_where_no_kernel_implements_it():
     with pytest.raises(demo.DemoError):
         r.tr.set_momentum_domain(DCT)
     r.close()
-    tr = demo.DemoTransform([(64, 64)], topk=8, beta=0.9, lr=1e-3, weight_decay=0.0, num_workers=1,
-                            chunk_shapes=[(64, 64)])
+    tr = demo.DemoTransform([(64, 128)], topk=8, beta=0.9, lr=1e-3, weight_decay=0.0, num_workers=1,
+                            chunk_shapes=[(32, 64)])
     with pytest.raises(demo.DemoError):
         tr.set_momentum_domain(DCT)
     tr.close()

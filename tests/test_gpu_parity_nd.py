@@ -25,7 +25,8 @@ def test_blocking_example_of_the_paper_128x512_in_16x32():
     ([(8, 12, 20), (64,)], [(4, 3, 5), (16,)], 7),                 # order 3 with odd extents + a vector
     ([(4, 6, 8, 16)], [(2, 3, 4, 8)], 20),                         # order 4
     ([(96, 40), (6, 64, 64)], [(32, 8), (1, 64, 64)], 32),         # rectangular + a stack of 64 x 64 tiles
-    ([(256, 128)], [(128, 128)], 64),                              # the largest chunk (16384 elements)
+    ([(256, 128), (64, 48)], [(128, 128), (32, 16)], 64),              # the largest chunk (16384 elements); the small
+                                                                   # rectangular tensor keeps the context on the N-D kernels
     ([(5, 7, 3)], [(1, 1, 1)], 1),                                 # every extent 1: the identity transform
     ([(128, 6)], [(128, 1)], 9),                                   # a column chunk
 ])
@@ -59,37 +60,81 @@ def test_aggregation_phi_and_alpha(agg, phi):
 
 
 def test_square_chunks_match_the_square_chunk_context():
-    """ndim <= 2 with equal extents: same payload layout and index sets, values / momenta / parameters equal
-    to fp32 rounding of a different summation order (demo_init through its dense kernels)."""
+    """Tensors with equal chunk extents inside an N-D context (a rectangular third tensor keeps it on the dense
+    per-axis kernels): same records per tensor as demo_init through its dense kernels -- index sets bit for bit,
+    values / momenta / parameters equal to fp32 rounding of a different summation order."""
     dev = torch.device("cuda")
     shapes, s, k, W = [(128, 192), (256,)], 32, 17, 2
     kw = dict(topk=k, beta=0.9, lr=1e-3, weight_decay=0.1, num_workers=W, grad_dtype=demo.DEMO_F32)
     a = demo.DemoTransform(shapes, chunk=s, **kw)
     a.set_path(demo.DEMO_PATH_GENERIC)
-    b = demo.DemoTransform(shapes, chunk_shapes=[(s, s), (s,)], **kw)
-    assert a.payload_bytes == b.payload_bytes
+    shapes_b = shapes + [(64, 48)]
+    b = demo.DemoTransform(shapes_b, chunk_shapes=[(s, s), (s,), (16, 8)], **kw)
+    with pytest.raises(demo.DemoError):
+        b.set_basis(torch.eye(s))              # an N-D context: one basis per chunk extent, only the DCT
+    assert [a.payload_layout(t) for t in range(2)] == [b.payload_layout(t) for t in range(2)]
+    n_rec = a.payload_bytes // 8
     state = []
-    for tr in (a, b):
-        x = [inputs.random_tensor(sh, 5 + t, 0.02, torch.float32, dev) for t, sh in enumerate(shapes)]
-        mom = [[torch.zeros(sh, device=dev) for sh in shapes] for _ in range(W)]
+    for tr, shp in ((a, shapes), (b, shapes_b)):
+        x = [inputs.random_tensor(sh, 5 + t, 0.02, torch.float32, dev) for t, sh in enumerate(shp)]
+        mom = [[torch.zeros(sh, device=dev) for sh in shp] for _ in range(W)]
         pay = [torch.zeros(tr.payload_bytes, dtype=torch.uint8, device=dev) for _ in range(W)]
         for step in range(3):
             for w in range(W):
-                g = [inputs.random_tensor(sh, 100 * step + 10 * w + t, 1.0, torch.float32, dev) for t, sh in enumerate(shapes)]
+                g = [inputs.random_tensor(sh, 100 * step + 10 * w + t, 1.0, torch.float32, dev) for t, sh in enumerate(shp)]
                 tr.compress(w, g, mom[w], pay[w])
             tr.decode_apply(pay, x)
         assert tr.device_status() == 0
         state.append((pay, mom, x))
     for w in range(W):
-        ia = state[0][0][w].view(torch.int32).view(-1, 2)
-        ib = state[1][0][w].view(torch.int32).view(-1, 2)
+        ia = state[0][0][w].view(torch.int32).view(-1, 2)[:n_rec]
+        ib = state[1][0][w].view(torch.int32).view(-1, 2)[:n_rec]
         assert torch.equal(ia[:, 0], ib[:, 0])  # index sets bit for bit
-        va, vb = state[0][0][w].view(torch.float32).view(-1, 2)[:, 1], state[1][0][w].view(torch.float32).view(-1, 2)[:, 1]
+        va = state[0][0][w].view(torch.float32).view(-1, 2)[:n_rec, 1]
+        vb = state[1][0][w].view(torch.float32).view(-1, 2)[:n_rec, 1]
         assert torch.allclose(va, vb, rtol=1e-5, atol=1e-6)  # summation orders differ
         for t in range(len(shapes)):
             assert torch.allclose(state[0][1][w][t], state[1][1][w][t], rtol=1e-5, atol=1e-6)
     for t in range(len(shapes)):
         assert torch.allclose(state[0][2][t], state[1][2][t], rtol=1e-5, atol=1e-6)
+    a.close()
+    b.close()
+
+
+@pytest.mark.parametrize("s,k", [(64, 32), (128, 40), (32, 2000)])
+def test_square_chunk_descriptors_take_the_square_chunk_kernels(s, k):
+    """demo_init_nd with s x s tiles of the last two axes / length-s segments of the last axis everywhere (leading
+    chunk extents 1) is demo_init on the flattened tensors: same kernels, so every output is bit for bit the same,
+    and what only that kind of context offers (a caller-supplied basis) is accepted."""
+    dev = torch.device("cuda")
+    nd_shapes = [(2 * s, 3 * s), (3, 2 * s, 2 * s), (4 * s,), (5, 2 * s)]
+    nd_chunks = [(s, s), (1, s, s), (s,), (1, s)]
+    flat_shapes = [(2 * s, 3 * s), (6 * s, 2 * s), (4 * s,), (10 * s,)]
+    W = 2
+    kw = dict(beta=0.999, lr=1e-3, weight_decay=0.1, num_workers=W)
+    a = demo.DemoTransform(flat_shapes, chunk=s, topk=min(k, s * s), **kw)
+    b = demo.DemoTransform(nd_shapes, chunk_shapes=nd_chunks, topk=k, **kw)
+    assert a.payload_bytes == b.payload_bytes
+    assert [a.payload_layout(t) for t in range(4)] == [b.payload_layout(t) for t in range(4)]
+    out = []
+    for tr, shp in ((a, flat_shapes), (b, nd_shapes)):
+        x = [inputs.random_tensor(sh, 5 + t, 0.02, torch.float32, dev) for t, sh in enumerate(flat_shapes)]
+        x = [v.view(sh) for v, sh in zip(x, shp)]
+        mom = [[torch.zeros(sh, device=dev) for sh in shp] for _ in range(W)]
+        pay = [torch.zeros(tr.payload_bytes, dtype=torch.uint8, device=dev) for _ in range(W)]
+        for step in range(2):
+            for w in range(W):
+                g = [inputs.random_tensor(sh, 100 * step + 10 * w + t, 1e-3, torch.bfloat16, dev).view(shn)
+                     for t, (sh, shn) in enumerate(zip(flat_shapes, shp))]
+                tr.compress(w, g, mom[w], pay[w])
+            tr.decode_apply(pay, x)
+        assert tr.device_status() == 0
+        out.append((pay, mom, x))
+    for w in range(W):
+        assert torch.equal(out[0][0][w], out[1][0][w])
+        assert all(torch.equal(p.reshape(-1), q.reshape(-1)) for p, q in zip(out[0][1][w], out[1][1][w]))
+    assert all(torch.equal(p.reshape(-1), q.reshape(-1)) for p, q in zip(out[0][2], out[1][2]))
+    b.set_basis(torch.eye(s))
     a.close()
     b.close()
 
