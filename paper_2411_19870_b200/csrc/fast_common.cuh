@@ -292,19 +292,20 @@ __device__ __forceinline__ void tmem_free_cta(uint32_t base, uint32_t cols)
 // is index order).  NK keys per lane, in list order.  Bit by bit, from the first bit where the bound and the
 // largest key differ, it looks for a threshold with exactly k_eff keys at or above it and stops as soon as one is
 // found; if the bits run out, equal keys straddle the k_eff-th place: keys above the threshold are kept, keys equal
-// to it in list order until k_eff are reached.  emit(pos, li) is called for every kept candidate: li its list
+// to it in list order until k_eff are reached.  emit(pos, i) is called for every kept candidate: i its list
 // position, pos its place among the kept ones (ascending list order).
 // ------------------------------------------------------------------------------------------------
-template <int NK, class Emit>
+template <int NK, class Where, class Emit>
 __device__ __forceinline__ void warp_ballot_select(const unsigned *cand_key, unsigned n_all, unsigned lmin, int k_eff,
-                                                   int lane, Emit emit)
+                                                   int lane, Where where, Emit emit)
 {
+    // where(i): storage position of list entry i (the list may sit in several pieces)
     unsigned keys[NK];
     unsigned hi = 0u;
 #pragma unroll
     for (int j = 0; j < NK; ++j) {
         const unsigned i = (unsigned)j * 32u + lane;
-        keys[j] = (i < n_all) ? cand_key[i] : 0u;
+        keys[j] = (i < n_all) ? cand_key[where(i)] : 0u;
         hi = max(hi, keys[j]);
     }
     hi = __reduce_max_sync(0xffffffffu, hi);

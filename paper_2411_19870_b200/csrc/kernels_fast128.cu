@@ -324,10 +324,11 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                         if (k_eff <= 128)
                             recs4[pos] = make_int4((r.idx >> 7) * XS, (r.idx & 127) * S, __float_as_int(a.alpha * r.val), 0);
                     };
+                    auto where = [](unsigned i) { return i; };
                     if (n_cand <= 64u)
-                        warp_ballot_select<2>(cand_key, n_cand, lmin, k_eff, lane, emit);
+                        warp_ballot_select<2>(cand_key, n_cand, lmin, k_eff, lane, where, emit);
                     else
-                        warp_ballot_select<8>(cand_key, n_cand, lmin, k_eff, lane, emit);
+                        warp_ballot_select<8>(cand_key, n_cand, lmin, k_eff, lane, where, emit);
                 }
             }
             }  // !zero_chunk
