@@ -496,7 +496,7 @@ def run_grid(args):
                     print(json.dumps({"workload": wl.name, "n_params": wl.n_params, "chunk": s, "topk": k,
                                       "num_workers": W, "ms_per_step": ms, "params_per_s": wl.n_params / (ms * 1e-3),
                                       "algorithmic_GBps": core / (ms * 1e-3) / 1e9,
-                                      "kernels": "fast" if s in (32, 64) else "generic"}), flush=True)
+                                      "kernels": "fast"}), flush=True)
                     tr.close()
                     del params, mom, grads, payloads
                     torch.cuda.empty_cache()
