@@ -32,7 +32,7 @@ constexpr int S = 128, H = 64, XS = S + 4, M = S * S, THREADS = 256;
 // different rows (the row pass) on 32 different banks; S + 4 (compress: 128-bit row accesses) gives 4-way
 // conflicts there.
 constexpr int XSD = S + 1;
-constexpr int RECS128 = 128 + 16;     // row-stage list: up to 128 kept records + padding for the look-ahead
+constexpr int RECS128 = 128 + 40;     // row-stage list: up to 128 kept records + padding for the look-ahead
 constexpr int ROW_AHEAD128 = 8;       // entries of the row-stage list fetched ahead of the accumulation
 constexpr int TMEM_COLS128 = 128;     // tensor-memory columns of a compress CTA (two CTAs per SM)
 constexpr int CAP128 = 256;           // candidate capacity of the fast top-k (one per thread)
@@ -423,27 +423,33 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
         if (h == 0 && k_eff <= 128) {
             // The running sum of a row is stored after every entry (the last store of a row carries the whole sum)
             // and starts again from zero when the next entry belongs to another row: no branch in the loop.
-            // Entries and their cosines are fetched ahead of the dependent accumulation.
+            // The cosines of a whole batch of entries are requested before the dependent accumulation starts: the
+            // 64 KB basis does not stay in what the two CTAs' shared memory leaves of the L1, so most of these
+            // loads go to L2 and a batch should pay that latency once.
             float *Xj = X + j;
             float acc = 0.f;
-            int4 nx = recs4[0];
+            auto row_stage = [&](auto batch_tag) {
+                constexpr int BATCH = decltype(batch_tag)::value;
 #pragma unroll 1
-            for (int r0 = 0; r0 < k_eff; r0 += ROW_AHEAD128) {
-                int4 rc[ROW_AHEAD128 + 1];
-                float cv[ROW_AHEAD128];
-                rc[0] = nx;
+                for (int r0 = 0; r0 < k_eff; r0 += BATCH) {
+                    float cv[BATCH];
 #pragma unroll
-                for (int q = 1; q < ROW_AHEAD128 + 1; ++q) rc[q] = recs4[r0 + q];
-                nx = rc[ROW_AHEAD128];
+                    for (int q = 0; q < BATCH; ++q) cv[q] = __ldg(a.C + (unsigned)(recs4[r0 + q].y + j));
+                    int4 nx = recs4[r0];
 #pragma unroll
-                for (int q = 0; q < ROW_AHEAD128; ++q) cv[q] = __ldg(a.C + (unsigned)(rc[q].y + j));
-#pragma unroll
-                for (int q = 0; q < ROW_AHEAD128; ++q) {
-                    acc = fmaf(__int_as_float(rc[q].z), cv[q], acc);
-                    Xj[rc[q].x] = acc;
-                    acc = (rc[q].x != rc[q + 1].x) ? 0.f : acc;
+                    for (int q = 0; q < BATCH; ++q) {
+                        const int4 rc = nx;
+                        nx = recs4[r0 + q + 1];
+                        acc = fmaf(__int_as_float(rc.z), cv[q], acc);
+                        Xj[rc.x] = acc;
+                        acc = (rc.x != nx.x) ? 0.f : acc;
+                    }
                 }
-            }
+            };
+            if (k_eff <= ROW_AHEAD128)
+                row_stage(std::integral_constant<int, ROW_AHEAD128>{});
+            else
+                row_stage(std::integral_constant<int, 4 * ROW_AHEAD128>{});
         } else if (h == 0) {
             // k > 128: the records come from the payload itself
             const float *Cj = a.C + j;
