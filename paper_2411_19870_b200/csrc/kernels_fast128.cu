@@ -199,14 +199,19 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
 #pragma unroll
                 for (int p = 0; p < H; ++p) X[(2 * p + h) * XS + j] = out[p];  // Y[u][j]
             } else {
+                // Q[j][2p + h]: a row keeps its even coefficients in its first half and its odd ones in the second
+                // (position 64h + p), so that each thread stores its 64 outputs with 128-bit stores; element-wise
+                // stores along a row, with a warp's lanes on 32 different rows, would run into 4-way bank conflicts
+                float4 *dst = reinterpret_cast<float4 *>(X + j * XS + H * h);
 #pragma unroll
-                for (int p = 0; p < H; ++p) X[j * XS + 2 * p + h] = out[p];    // Q[j][v]
+                for (int p4 = 0; p4 < H / 4; ++p4) dst[p4] = make_float4(out[4 * p4], out[4 * p4 + 1], out[4 * p4 + 2], out[4 * p4 + 3]);
             }
             __syncthreads();
         }
 
         // ---- exact top-k ---------------------------------------------------------------------------
-        // thread tid scans the half row [tid/2][64*(tid&1) .. +64): flat indices 64*tid .. 64*tid+63.
+        // thread tid scans one half of row tid/2 as the row pass stored it: the even coefficients (tid even) or the
+        // odd ones (tid odd); element e of its half is coefficient 2e + (tid & 1), flat index 128*(tid/2) + 2e + (tid&1).
         // Fast path (k_eff <= 256): the k_eff-th largest of the 256 per-thread maxima is a lower bound L of
         // the k_eff-th largest coefficient (256 groups: the bound is tight, a few dozen candidates); the
         // candidates are listed in index order and ranked exactly, ties to the lowest index.  Everything
@@ -297,21 +302,33 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                 mask = (tid & 1) ? ((mreg << 16) | (mreg >> 48)) : mreg;
             }
             const unsigned cnt = (unsigned)__popcll(mask);
-            unsigned o = block_exclusive_scan(cnt, warp_tot);
+            const unsigned o = block_exclusive_scan(cnt, warp_tot);
             if (tid == THREADS - 1) s_state[3] = o + cnt;
             __syncthreads();
             const unsigned n_cand = s_state[3];
             use_radix = n_cand > (unsigned)CAP128 || n_cand < (unsigned)k_eff;
             if (!use_radix) {
+                // The list is in index order: inside a row the candidates of the even-coefficient thread (lane 2r)
+                // and of the odd-coefficient thread (lane 2r+1) interleave, so a candidate's place is the row's base
+                // plus the candidates of both threads with a smaller coefficient index.
+                const unsigned plo = __shfl_xor_sync(0xffffffffu, (unsigned)mask, 1);
+                const unsigned phi = __shfl_xor_sync(0xffffffffu, (unsigned)(mask >> 32), 1);
+                const unsigned long long pmask = ((unsigned long long)phi << 32) | plo;
+                const int odd = tid & 1;
+                const unsigned row_base = odd ? o - (unsigned)__popcll(pmask) : o;
                 const float *mine = reinterpret_cast<const float *>(mine4);
-                while (mask) {
-                    const int e = __ffsll((long long)mask) - 1;
-                    mask &= mask - 1ull;
+                unsigned long long left = mask;
+                while (left) {
+                    const int e = __ffsll((long long)left) - 1;
+                    left &= left - 1ull;
+                    const unsigned long long below = (1ull << e) - 1ull;
+                    // partner coefficients before 2e + odd: 2e' + (1 - odd) with e' < e (even thread) or e' <= e (odd thread)
+                    const unsigned long long pbelow = odd ? ((below << 1) | 1ull) : below;
+                    const unsigned at = row_base + (unsigned)__popcll(mask & below) + (unsigned)__popcll(pmask & pbelow);
                     const float val = mine[e];
-                    cand_key[o] = mag_key(val);
-                    cand_val[o] = val;
-                    cand_idx[o] = 64 * tid + e;
-                    ++o;
+                    cand_key[at] = mag_key(val);
+                    cand_val[at] = val;
+                    cand_idx[at] = S * (tid >> 1) + 2 * e + odd;
                 }
                 __syncthreads();
                 // the first warp picks the k_eff largest candidates (list order = index order) and writes the records
@@ -340,7 +357,25 @@ __global__ void __launch_bounds__(THREADS, 2) compress_fast128_kernel(DemoCompre
                 s_state[0] = 0u;
                 s_state[1] = (unsigned)k_eff;
             }
-            // thread tid scans the half row [tid/2][64*(tid&1) .. +64): flat indices 64*tid .. 64*tid+63
+            // this path works on rows in natural order: every thread turns its half row back (coefficient 2e + (tid&1)
+            // from position 64*(tid&1) + e to position 2e + (tid&1)); then thread tid scans the half row
+            // [tid/2][64*(tid&1) .. +64): flat indices 64*tid .. 64*tid+63
+            {
+                float *rowp = X + (tid >> 1) * XS;
+                float tmp[64];
+#pragma unroll
+                for (int i4 = 0; i4 < 16; ++i4) {
+                    const float4 f = reinterpret_cast<const float4 *>(rowp + 64 * (tid & 1))[i4];
+                    tmp[4 * i4 + 0] = f.x;
+                    tmp[4 * i4 + 1] = f.y;
+                    tmp[4 * i4 + 2] = f.z;
+                    tmp[4 * i4 + 3] = f.w;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int e = 0; e < 64; ++e) rowp[2 * e + (tid & 1)] = tmp[e];
+                __syncthreads();
+            }
             const float *mine = X + (tid >> 1) * XS + 64 * (tid & 1);
 #pragma unroll 1
             for (int pass = 0; pass < 4; ++pass) {
