@@ -632,32 +632,38 @@ __global__ void __launch_bounds__(THREADS, 2) decode_fast128_kernel(DemoDecodeAr
             }
             __syncthreads();
         }
-        // two inverse passes (rolled): pass 0 along row j, pass 1 down column j
+        // two inverse passes (rolled): both walk "row j" of the tile with unit stride -- pass 0 leaves its result
+        // transposed, so that the columns pass 1 needs are rows again and every access below has a fixed offset
         float in[H], out[H];
         bool arrived = true;
+        float *ln = St + j * XSD;  // line j
 #pragma unroll 1
         for (int pass = 0; pass < 2; ++pass) {
-            const int line = pass == 0 ? j * XSD : j;   // start of line j
-            const int step = pass == 0 ? 1 : XSD;       // distance between consecutive elements of the line
 #pragma unroll
-            for (int p = 0; p < H; ++p) in[p] = St[line + (2 * p + h) * step];
+            for (int p = 0; p < H; ++p) in[p] = ln[2 * p + h];
             fence_proxy_async();
             __syncthreads();  // every coefficient of the tile has been read
             inverse_half(h, in, out);
             // exchange e / o inside the line: e at elements 0..63, o at 64..127
 #pragma unroll
-            for (int n = 0; n < H; ++n) St[line + (h * H + n) * step] = out[n];
+            for (int n = 0; n < H; ++n) ln[h * H + n] = out[n];
             __syncthreads();
 #pragma unroll
             for (int n = 0; n < H; ++n) {
-                const float other = St[line + ((h ^ 1) * H + n) * step];
+                const float other = ln[(h ^ 1) * H + n];
                 out[n] = h ? other - out[n] : out[n] + other;  // h=0: element n;  h=1: element 127-n
             }
             fence_proxy_async();
             __syncthreads();  // both halves of every line have read their partner's values
             if (pass == 0) {
+                // element n (resp. 127-n) of row j goes to row n (127-n), column j
+                if (h) {
 #pragma unroll
-                for (int n = 0; n < H; ++n) St[line + (h ? (S - 1 - n) : n) * step] = out[n];
+                    for (int n = 0; n < H; ++n) St[(S - 1 - n) * XSD + j] = out[n];
+                } else {
+#pragma unroll
+                    for (int n = 0; n < H; ++n) St[n * XSD + j] = out[n];
+                }
                 __syncthreads();
             } else if (!SIGNS) {
                 if (tid == 0) {
