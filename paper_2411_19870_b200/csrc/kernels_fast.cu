@@ -765,7 +765,9 @@ __host__ __device__ constexpr size_t decode_slot_bytes(bool counts)
 
 // SIGNS: the parameter-server form -- sign(R) goes out as int8 per element, the parameters are neither read
 // nor written (a separate instantiation, so that the update kernel keeps its size).
-template <int S, bool TMAP, int THREADS, bool SIGNS = false>
+// WIDE: the instantiation for fan-ins above one staging batch (sixteen workers at k <= 32): every further batch of a
+// chunk's workers is requested, like the first, while the scatter works on the batch before it.
+template <int S, bool TMAP, int THREADS, bool SIGNS = false, bool WIDE = false>
 __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(DemoDecodeArgs a)
 {
     using C = Cfg<S>;
@@ -825,6 +827,21 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
+    // (WIDE) a further batch of the same chunk: workers w_first .. of the chunk whose records start at off_n
+    auto stage_batch = [&](int buf, int k_n, long long off_n, int w_first) {
+        const int sh = (k_n > 32) ? 6 : 5;
+        DemoRecord *dst = stage_all + buf * STAGE_RECORDS;
+#pragma unroll
+        for (int i = 0; i < STAGE_RECORDS / S; ++i) {
+            const int r = i * S + t, wl = w_first + (r >> sh), j = r & ((1 << sh) - 1);
+            if (wl < a.W && j < k_n)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst + r)),
+                             "l"(a.payloads[wl] + off_n + j)
+                             : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
     const long long stride = (long long)gridDim.x * NCH;
     long long c = (long long)blockIdx.x * NCH + slot;
     int buf = 0;
@@ -861,14 +878,19 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
             if (counts)
                 for (int v = 0; v < S; ++v) Cn[t * S + v] = 0;
         }
-        // next chunk's records on their way (the cursor moves on; this chunk's table entry is in `te`)
-        if (c + stride < a.n_chunks)
-            stage_ahead(buf ^ 1, c + stride);
-        else
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group 1;" ::: "memory");  // this chunk's copies have landed
+        auto stage_next_chunk = [&](int into) {  // (the cursor moves on; this chunk's table entry is in `te`)
+            if (c + stride < a.n_chunks)
+                stage_ahead(into, c + stride);
+            else
+                asm volatile("cp.async.commit_group;" ::: "memory");
+        };
         DemoRecord *stage = stage_all + buf * STAGE_RECORDS;
-        buf ^= 1;
+        if (!WIDE || k_eff > 64) {
+            // next chunk's records on their way
+            stage_next_chunk(buf ^ 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");  // this chunk's copies have landed
+            buf ^= 1;
+        }
         // S = sum over workers in worker order (Decompress&Aggregate).
         if (k_eff <= 64) {
             // Every warp owns the 32 rows of the tile its threads cleared and will transform (rows 32 w .. 32 w + 31
@@ -881,7 +903,19 @@ __global__ void __launch_bounds__(THREADS, 512 / THREADS) decode_fast_kernel(Dem
             const int sh = (k_eff > 32) ? 6 : 5;          // a worker's records take 32 or 64 staging entries
             const int wb = STAGE_RECORDS >> sh;           // workers per batch: 16 or 8
             for (int w0 = 0; w0 < a.W; w0 += wb) {
-                if (w0 > 0) {  // further batches of a large fan-in: fetched on the spot
+                if (WIDE) {
+                    // both warps are done with the previous batch (between chunks the barrier at the end of a chunk
+                    // has seen to that): its buffer takes the batch after this one -- of this chunk's workers or,
+                    // behind the last, the first batch of the slot's next chunk
+                    if (w0 > 0) sb.sync();
+                    if (w0 + wb < a.W)
+                        stage_batch(buf ^ 1, k_eff, rec_off, w0 + wb);
+                    else
+                        stage_next_chunk(buf ^ 1);
+                    asm volatile("cp.async.wait_group 1;" ::: "memory");  // this batch's copies have landed
+                    stage = stage_all + buf * STAGE_RECORDS;
+                    buf ^= 1;
+                } else if (w0 > 0) {  // further batches of a large fan-in: fetched on the spot
                     sb.sync();  // the previous batch has been consumed by both warps
 #pragma unroll 1
                     for (int r = t; r < STAGE_RECORDS; r += S) {
@@ -1090,8 +1124,11 @@ cudaError_t launch_decode(const DemoDecodeArgs &a, int sm_count, cudaStream_t st
     const size_t smem = decode_slot_bytes<S>(a.agg == 2) * NCH;
     if (a.sign_ptrs != nullptr)
         return launch(decode_fast_kernel<S, false, TH, true>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
-    if (a.tmap_x != nullptr)
+    if (a.tmap_x != nullptr) {
+        if (a.W > 16)  // more than one staging batch at k <= 32
+            return launch(decode_fast_kernel<S, true, TH, false, true>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
         return launch(decode_fast_kernel<S, true, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
+    }
     return launch(decode_fast_kernel<S, false, TH>, TH, NCH, smem, a.n_chunks, sm_count, stream, &a);
 }
 
